@@ -1,0 +1,175 @@
+/*
+ * mxfp4.h -- C ABI of the B200 (sm_100a) MXFP4 quantize + block-scaled GEMM library.
+ *
+ * The library implements the hot path of MXFP4 training of transformer linear layers:
+ * both GEMM operands are quantized to OCP MXFP4 (E2M1 elements, one E8M0 power-of-two
+ * scale per 32 contiguous elements along the reduction axis; Appendix A.1, Eq. (1)),
+ * optionally after a 32-point Hadamard rotation along that axis (Appendix A.2), and
+ * multiplied on the FP4 tensor cores (Fprop / Dgrad / Wgrad, Appendix C).
+ *
+ * Conventions for every entry point unless stated otherwise
+ *   - All data pointers are DEVICE pointers owned by the caller.  The library allocates
+ *     no device memory and keeps no reference to a buffer after the call's work is done.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *     enqueue work; they do not synchronise.
+ *   - Return value: MXFP4_OK (0) or a negative MXFP4_ERR_* code.  Argument errors are
+ *     detected on the host before anything is enqueued.  Device-side problems (a bounded
+ *     wait that expired) never trap: the kernel records a status word and returns, and
+ *     mxfp4_check() reports it.
+ *   - A GEMM operand is "K-major": operand[o][k], k contiguous.  Codes hold two elements
+ *     per byte, element k even in bits 3:0 and k odd in bits 7:4.  A code is
+ *     (sign << 3) | magnitude with magnitudes 0..7 = {0, 0.5, 1, 1.5, 2, 3, 4, 6}.
+ *   - A scale byte b means 2^(b - 127).
+ */
+#ifndef MXFP4_H_
+#define MXFP4_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define MXFP4_OK 0
+#define MXFP4_ERR_NULL (-1)      /* a required pointer is NULL                               */
+#define MXFP4_ERR_SHAPE (-2)     /* non-positive size, K not a multiple of 32, ld too small   */
+#define MXFP4_ERR_ALIGN (-3)     /* pointer not 16-byte aligned, or ld not a multiple of 8    */
+#define MXFP4_ERR_ENUM (-4)      /* axis / hadamard_mode / rounding / layout / dtype invalid  */
+#define MXFP4_ERR_WORKSPACE (-5) /* workspace missing or too small                            */
+#define MXFP4_ERR_CUDA (-6)      /* a CUDA runtime/driver call failed (launch, descriptor)    */
+#define MXFP4_ERR_TIMEOUT (-7)   /* a bounded device-side wait expired (reported by check)    */
+#define MXFP4_ERR_DEVICE (-8)    /* not an sm_100 device                                      */
+
+/* enums (plain ints in the ABI) */
+#define MXFP4_AXIS_ROWS 0 /* 32-blocks run down the rows (column-wise 32x1); operand = src^T */
+#define MXFP4_AXIS_COLS 1 /* 32-blocks run along the contiguous axis (row-wise 1x32)         */
+
+#define MXFP4_HADAMARD_NONE 0
+#define MXFP4_HADAMARD_DET 1  /* deterministic 32-point rotation                              */
+#define MXFP4_HADAMARD_RAND 2 /* sign diagonal from `seed`, then the rotation                 */
+
+#define MXFP4_ROUND_RNE 0 /* round to nearest, ties to even                                   */
+#define MXFP4_ROUND_SR 1  /* stochastic rounding, Philox4x32-10 keyed by (seed, element)      */
+
+#define MXFP4_SCALES_CANONICAL 0 /* scales[o][t], row-major, outer x K/32 bytes               */
+#define MXFP4_SCALES_TILED 1     /* 128-row x 4-block tiles of 512 bytes (what the GEMM reads)*/
+
+#define MXFP4_OUT_BF16 0
+#define MXFP4_OUT_FP32 1
+
+#define MXFP4_PASS_FPROP 0
+#define MXFP4_PASS_DGRAD 1
+#define MXFP4_PASS_WGRAD 2
+
+/* Library version (major * 100 + minor). */
+int mxfp4_version(void);
+
+/* Human-readable name of a status code (static storage). */
+const char* mxfp4_status_string(int status);
+
+/* Bytes of packed codes for an operand of `outer` rows and K elements per row: outer*K/2. */
+size_t mxfp4_codes_bytes(int64_t outer, int64_t K);
+
+/*
+ * Bytes of the scale buffer.  Canonical: outer*K/32.  Tiled: whole tiles of 128 rows x 4
+ * blocks, ceil(outer/128) * ceil(K/128) * 512 bytes; the scale of (row o, block t) lives at
+ *   ((o/128) * ceil(K/128) + t/4) * 512 + (o%32)*16 + ((o%128)/32)*4 + (t%4).
+ * Padding rows / blocks hold 0 (the scale of an all-zero block).  Returns 0 on bad input.
+ */
+size_t mxfp4_scales_bytes(int64_t outer, int64_t K, int scale_layout);
+
+/*
+ * mxfp4_quantize -- Eq. (1) of Appendix A.1 with the optional rotation of Appendix A.2,
+ * for row-wise (axis 1) or column-wise (axis 0) 32-blocks (Appendix D).
+ *
+ *   src_bf16     [rows x cols] bf16, row-major, leading dimension ld_src (elements,
+ *                multiple of 8, >= cols); 16-byte aligned.
+ *   axis         MXFP4_AXIS_COLS: operand[o][k] = src[o][k], outer = rows, K = cols.
+ *                MXFP4_AXIS_ROWS: operand[o][k] = src[k][o], outer = cols, K = rows -- the
+ *                transposed operand Dgrad (W^T) and Wgrad (dY^T, X^T) need, written directly
+ *                with no separate transpose pass.
+ *   K must be a multiple of 32.  For MXFP4_AXIS_ROWS, cols must be a multiple of 8.
+ *   hadamard_mode, rounding, seed: each 32-block v becomes H*v (mode 1) or H*(D*v) (mode 2,
+ *                D the +-1 diagonal drawn from `seed`) in fp32 with a fixed five-stage
+ *                butterfly; the block scale is 2^(floor(log2 amax) - 2); elements are rounded
+ *                to E2M1 with saturation at 6.  With MXFP4_ROUND_SR each element uses 8 bits
+ *                of Philox4x32-10(key = seed, counter = (e>>4, 0, operand_tag, 0)), e the
+ *                element's index o*K + k in the operand view.
+ *   operand_tag  decorrelates the stochastic-rounding streams of different operands.
+ *   codes        out, [outer x K/2] bytes, 16-byte aligned.
+ *   scales       out, mxfp4_scales_bytes(outer, K, scale_layout) bytes, 16-byte aligned.
+ * Inputs must be finite.
+ */
+int mxfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis,
+                   int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
+                   void* codes, void* scales, int scale_layout, void* stream);
+
+/*
+ * mxfp4_gemm -- the block-scaled product the linear layers run in place of their FP8 GEMM
+ * (Appendix A.2 last paragraph; operand orientation per Appendix C):
+ *   out[m][n] = alpha * sum_t 2^(sa[m][t]-127) * 2^(sb[n][t]-127) * sum_{k in block t} A[m][k]*B[n][k]
+ * A: [M x K], B: [N x K], both K-major codes with TILED scales (as mxfp4_quantize writes
+ * them).  K multiple of 32.  Products are exact; accumulation is fp32 on the tensor cores.
+ *   alpha        exact power of two in the intended use (2^-5 undoes H*H^T = 32*I).
+ *   out          [M x N] row-major, leading dimension ld_out (elements), bf16 (RNE) or fp32;
+ *                16-byte aligned, ld_out*sizeof(elem) a multiple of 16.
+ *   workspace    unused by the current kernel; may be NULL with workspace_bytes 0.
+ */
+int mxfp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes,
+               const void* b_scales, int64_t M, int64_t N, int64_t K, float alpha, void* out,
+               int out_dtype, int64_t ld_out, void* workspace, size_t workspace_bytes,
+               void* stream);
+
+/*
+ * Workspace (device bytes) the fused linear passes need for the two quantized operands:
+ * codes + tiled scales of both, each region 1024-byte aligned.  pass = MXFP4_PASS_*.
+ */
+size_t mxfp4_linear_workspace_bytes(int64_t T, int64_t in_features, int64_t out_features, int pass);
+
+/*
+ * Fused linear passes (Appendix C).  Each quantizes its two operands along the reduction
+ * axis (same hadamard_mode / rounding / seed for both so that the rotation cancels;
+ * operand_tag 0 for the first operand, 1 for the second) and runs the GEMM with
+ * alpha = 2^-5 when rotated, 1 otherwise.  All matrices row-major and dense (ld = width).
+ *   fprop: Y[T x out]   = X[T x in]    * W[out x in]^T   (both row-wise along `in`)
+ *   dgrad: dX[T x in]   = dY[T x out]  * W[out x in]     (dY row-wise along `out`; W column-wise)
+ *   wgrad: dW[out x in] = dY[T x out]^T * X[T x in]      (both column-wise along tokens)
+ * The reduction size (in / out / T respectively) must be a multiple of 32, all widths
+ * multiples of 8.  workspace >= mxfp4_linear_workspace_bytes(...), 1024-byte aligned.
+ */
+int mxfp4_linear_fprop(const void* X, const void* W, void* Y, int64_t T, int64_t in_features,
+                       int64_t out_features, int hadamard_mode, int rounding, uint64_t seed,
+                       int out_dtype, void* workspace, size_t workspace_bytes, void* stream);
+int mxfp4_linear_dgrad(const void* dY, const void* W, void* dX, int64_t T, int64_t in_features,
+                       int64_t out_features, int hadamard_mode, int rounding, uint64_t seed,
+                       int out_dtype, void* workspace, size_t workspace_bytes, void* stream);
+int mxfp4_linear_wgrad(const void* dY, const void* X, void* dW, int64_t T, int64_t in_features,
+                       int64_t out_features, int hadamard_mode, int rounding, uint64_t seed,
+                       int out_dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Host-buffer form of the three passes: a_host / b_host / out_host are HOST pointers (pinned
+ * memory makes the copies asynchronous).  The call copies both inputs to the caller's device
+ * staging buffers, runs the pass there, copies the result back and returns after the
+ * stream has drained, so out_host is valid on return.
+ *   pass        MXFP4_PASS_*; (a, b, out) = (X, W, Y) / (dY, W, dX) / (dY, X, dW).
+ *   dev_a, dev_b, dev_out   device staging for the two inputs (bf16) and the output.
+ */
+int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* out_host, int64_t T,
+                      int64_t in_features, int64_t out_features, int hadamard_mode, int rounding,
+                      uint64_t seed, int out_dtype, void* dev_a, void* dev_b, void* dev_out,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Synchronises `stream` and returns the sticky device-side status of the current device:
+ * MXFP4_OK, MXFP4_ERR_TIMEOUT (a kernel gave up a bounded wait; its output is invalid) or
+ * MXFP4_ERR_CUDA.  The status word is cleared by the call.
+ */
+int mxfp4_check(void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXFP4_H_ */

@@ -1,0 +1,220 @@
+"""Thin ctypes binding over ``libmxfp4.so`` (the C ABI declared in ``include/mxfp4.h``).
+
+Argument marshalling only: torch provides device memory and the current CUDA stream; every
+step of the path runs inside the library's kernels.  There is no CPU or PyTorch fallback:
+if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+HADAMARD_NONE, HADAMARD_DET, HADAMARD_RAND = 0, 1, 2
+ROUND_RNE, ROUND_SR = 0, 1
+SCALES_CANONICAL, SCALES_TILED = 0, 1
+OUT_BF16, OUT_FP32 = 0, 1
+PASS_FPROP, PASS_DGRAD, PASS_WGRAD = 0, 1, 2
+AXIS_ROWS, AXIS_COLS = 0, 1
+
+EXPORTS = (
+    "mxfp4_version", "mxfp4_status_string", "mxfp4_codes_bytes", "mxfp4_scales_bytes",
+    "mxfp4_quantize", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
+    "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_host", "mxfp4_check",
+)
+
+
+class Mxfp4Error(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what} failed: {status} ({status_string(status)})")
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """Load ``libmxfp4.so`` (must have been built in-tree); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise FileNotFoundError(
+            f"{path} not found: build it with `python -m paper_2605_09825_b200.build` "
+            "(there is no fallback path)")
+    lib = ctypes.CDLL(path)
+    vp, i64, u64, u32, ci, sz = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_uint64, ctypes.c_uint32,
+                                 ctypes.c_int, ctypes.c_size_t)
+    lib.mxfp4_version.argtypes, lib.mxfp4_version.restype = [], ci
+    lib.mxfp4_status_string.argtypes, lib.mxfp4_status_string.restype = [ci], ctypes.c_char_p
+    lib.mxfp4_codes_bytes.argtypes, lib.mxfp4_codes_bytes.restype = [i64, i64], sz
+    lib.mxfp4_scales_bytes.argtypes, lib.mxfp4_scales_bytes.restype = [i64, i64, ci], sz
+    lib.mxfp4_quantize.argtypes = [vp, i64, i64, i64, ci, ci, ci, u64, u32, vp, vp, ci, vp]
+    lib.mxfp4_quantize.restype = ci
+    lib.mxfp4_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, ctypes.c_float, vp, ci, i64, vp, sz, vp]
+    lib.mxfp4_gemm.restype = ci
+    lib.mxfp4_linear_workspace_bytes.argtypes = [i64, i64, i64, ci]
+    lib.mxfp4_linear_workspace_bytes.restype = sz
+    for name in ("mxfp4_linear_fprop", "mxfp4_linear_dgrad", "mxfp4_linear_wgrad"):
+        fn = getattr(lib, name)
+        fn.argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, sz, vp]
+        fn.restype = ci
+    lib.mxfp4_linear_host.argtypes = [ci, vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, vp, vp, vp,
+                                      sz, vp]
+    lib.mxfp4_linear_host.restype = ci
+    lib.mxfp4_check.argtypes, lib.mxfp4_check.restype = [vp], ci
+    _lib = lib
+    return lib
+
+
+def version() -> int:
+    return int(load_library().mxfp4_version())
+
+
+def status_string(status: int) -> str:
+    return load_library().mxfp4_status_string(int(status)).decode()
+
+
+def codes_bytes(outer: int, K: int) -> int:
+    return int(load_library().mxfp4_codes_bytes(outer, K))
+
+
+def scales_bytes(outer: int, K: int, scale_layout: int = SCALES_TILED) -> int:
+    return int(load_library().mxfp4_scales_bytes(outer, K, scale_layout))
+
+
+def linear_workspace_bytes(T: int, in_features: int, out_features: int, pass_: int) -> int:
+    return int(load_library().mxfp4_linear_workspace_bytes(T, in_features, out_features, pass_))
+
+
+def _stream() -> int:
+    return int(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev_ptr(t: torch.Tensor) -> int:
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    return int(t.data_ptr())
+
+
+def _raise(rc: int, what: str):
+    if rc != 0:
+        raise Mxfp4Error(rc, what)
+
+
+def quantize(src: torch.Tensor, axis: int = AXIS_COLS, hadamard_mode: int = HADAMARD_NONE,
+             rounding: int = ROUND_RNE, seed: int = 0, operand_tag: int = 0,
+             scale_layout: int = SCALES_TILED, codes: torch.Tensor | None = None,
+             scales: torch.Tensor | None = None):
+    """``mxfp4_quantize`` on a 2-D bf16 CUDA tensor (rows may be strided: ``ld = stride(0)``).
+
+    Returns ``(codes uint8 [outer, K/2], scales uint8 [scales_bytes])``; output tensors are
+    allocated with torch unless passed in.
+    """
+    if src.dtype != torch.bfloat16 or src.dim() != 2 or src.stride(1) != 1:
+        raise ValueError("src must be a 2-D bf16 tensor with contiguous rows")
+    rows, cols = src.shape
+    outer, K = (rows, cols) if axis == AXIS_COLS else (cols, rows)
+    lib = load_library()
+    if K % 32 != 0 or K <= 0 or outer <= 0:
+        _raise(-2, "mxfp4_quantize")
+    if codes is None:
+        codes = torch.empty((outer, K // 2), dtype=torch.uint8, device=src.device)
+    if scales is None:
+        scales = torch.empty(scales_bytes(outer, K, scale_layout), dtype=torch.uint8, device=src.device)
+    rc = lib.mxfp4_quantize(_dev_ptr(src), rows, cols, src.stride(0), axis, hadamard_mode, rounding,
+                            ctypes.c_uint64(seed), ctypes.c_uint32(operand_tag), _dev_ptr(codes),
+                            _dev_ptr(scales), scale_layout, _stream())
+    _raise(rc, "mxfp4_quantize")
+    return codes, scales
+
+
+def gemm(a_codes: torch.Tensor, a_scales: torch.Tensor, b_codes: torch.Tensor, b_scales: torch.Tensor,
+         alpha: float = 1.0, out_dtype: int = OUT_BF16, out: torch.Tensor | None = None):
+    """``mxfp4_gemm``: ``alpha * A B^T`` from packed codes [M, K/2], [N, K/2] and tiled scales."""
+    M, kh = a_codes.shape
+    N, kh2 = b_codes.shape
+    if kh != kh2:
+        raise ValueError("A and B disagree on K")
+    K = 2 * kh
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32,
+                          device=a_codes.device)
+    rc = load_library().mxfp4_gemm(_dev_ptr(a_codes), _dev_ptr(a_scales), _dev_ptr(b_codes),
+                                   _dev_ptr(b_scales), M, N, K, ctypes.c_float(alpha), _dev_ptr(out),
+                                   out_dtype, out.stride(0), None, 0, _stream())
+    _raise(rc, "mxfp4_gemm")
+    return out
+
+
+def _linear(name: str, pass_: int, a: torch.Tensor, b: torch.Tensor, T: int, in_f: int, out_f: int,
+            out_shape, hadamard_mode, rounding, seed, out_dtype, workspace, out):
+    for t in (a, b):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise ValueError("inputs must be contiguous bf16 tensors")
+    need = linear_workspace_bytes(T, in_f, out_f, pass_)
+    if workspace is None:
+        workspace = torch.empty(max(need, 1), dtype=torch.uint8, device=a.device)
+    if out is None:
+        out = torch.empty(out_shape, dtype=torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32,
+                          device=a.device)
+    fn = getattr(load_library(), name)
+    rc = fn(_dev_ptr(a), _dev_ptr(b), _dev_ptr(out), T, in_f, out_f, hadamard_mode, rounding,
+            ctypes.c_uint64(seed), out_dtype, _dev_ptr(workspace), workspace.numel(), _stream())
+    _raise(rc, name)
+    return out
+
+
+def linear_fprop(X, W, hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0, out_dtype=OUT_BF16,
+                 workspace=None, out=None):
+    """Y [T, out] = X [T, in] W[out, in]^T through ``mxfp4_linear_fprop``."""
+    T, in_f = X.shape
+    out_f = W.shape[0]
+    return _linear("mxfp4_linear_fprop", PASS_FPROP, X, W, T, in_f, out_f, (T, out_f), hadamard_mode,
+                   rounding, seed, out_dtype, workspace, out)
+
+
+def linear_dgrad(dY, W, hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0, out_dtype=OUT_BF16,
+                 workspace=None, out=None):
+    """dX [T, in] = dY [T, out] W [out, in] through ``mxfp4_linear_dgrad``."""
+    T, out_f = dY.shape
+    in_f = W.shape[1]
+    return _linear("mxfp4_linear_dgrad", PASS_DGRAD, dY, W, T, in_f, out_f, (T, in_f), hadamard_mode,
+                   rounding, seed, out_dtype, workspace, out)
+
+
+def linear_wgrad(dY, X, hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0, out_dtype=OUT_BF16,
+                 workspace=None, out=None):
+    """dW [out, in] = dY [T, out]^T X [T, in] through ``mxfp4_linear_wgrad``."""
+    T, out_f = dY.shape
+    in_f = X.shape[1]
+    return _linear("mxfp4_linear_wgrad", PASS_WGRAD, dY, X, T, in_f, out_f, (out_f, in_f),
+                   hadamard_mode, rounding, seed, out_dtype, workspace, out)
+
+
+def linear_host(pass_: int, a_host: torch.Tensor, b_host: torch.Tensor, out_host: torch.Tensor, T: int,
+                in_f: int, out_f: int, dev_a, dev_b, dev_out, workspace, hadamard_mode=HADAMARD_DET,
+                rounding=ROUND_RNE, seed=0, out_dtype=OUT_BF16):
+    """``mxfp4_linear_host``: host (ideally pinned) inputs/outputs, copies inside the call."""
+    for t in (a_host, b_host, out_host):
+        if t.is_cuda:
+            raise ValueError("host tensors expected")
+    rc = load_library().mxfp4_linear_host(
+        pass_, a_host.data_ptr(), b_host.data_ptr(), out_host.data_ptr(), T, in_f, out_f,
+        hadamard_mode, rounding, ctypes.c_uint64(seed), out_dtype, _dev_ptr(dev_a), _dev_ptr(dev_b),
+        _dev_ptr(dev_out), _dev_ptr(workspace), workspace.numel(), _stream())
+    _raise(rc, "mxfp4_linear_host")
+    return out_host
+
+
+def check() -> None:
+    """Synchronise the current stream and raise if a kernel recorded a device-side error."""
+    _raise(load_library().mxfp4_check(_stream()), "mxfp4_check")

@@ -1,0 +1,303 @@
+// Block-scaled MXFP4 GEMM on the 5th-generation tensor cores (the MXFP4 GEMM that replaces the
+// linear layers' FP8 GEMM; operand orientation per Appendix C):
+//   out[m][n] = alpha * sum_t 2^(sa[m][t]-127) 2^(sb[n][t]-127) sum_{k in block t} A[m][k] B[n][k]
+//
+// Persistent, warp-specialised, one CTA per SM, output tile 128 x 256:
+//   warp 0      TMA producer: per K-step of 256 elements loads A (128 rows x 128 B of packed
+//               codes) and B (256 rows x 128 B) in the 128-byte swizzle, plus the matching
+//               scale tiles (512-byte blocks of 128 rows x 4 MX blocks), into a 4-stage ring.
+//   warp 1      MMA issuer: copies the scale tiles shared memory -> TMEM (tcgen05.cp), then
+//               issues four tcgen05.mma kind::mxf4.block_scale (K = 64 each) per stage; the
+//               fp32 accumulator (128 lanes x 256 columns) lives in TMEM.
+//   warps 2..5  epilogue: TMEM -> registers (tcgen05.ld), * alpha, bf16/fp32, global stores.
+// All waits are bounded (see ptx_sm100.cuh).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/mxfp4.h"
+#include "ptx_sm100.cuh"
+#include "tma_host.cuh"
+
+namespace mxfp4 {
+
+constexpr int kGBlockM = 128;
+constexpr int kGBlockN = 256;
+constexpr int kGBlockK = 256;                    // elements per stage = 128 bytes of codes
+constexpr int kGStages = 4;
+constexpr int kGABytes = kGBlockM * 128;         // 16 KB
+constexpr int kGBBytes = kGBlockN * 128;         // 32 KB
+constexpr int kGSfaBytes = 2 * 512;              // 2 K-tiles of 128 elements
+constexpr int kGSfbBytes = 2 * 2 * 512;          // 2 row blocks x 2 K-tiles
+constexpr int kGThreads = 192;
+constexpr uint32_t kGTmemCols = 512;
+constexpr uint32_t kGTmemSfBase = 256;           // accumulator occupies columns 0..255
+constexpr uint32_t kGTmemSfPerBuf = 24;          // 8 columns SFA + 16 columns SFB
+
+struct GemmStage {
+    alignas(1024) uint8_t a[kGABytes];
+    alignas(1024) uint8_t b[kGBBytes];
+    alignas(128) uint8_t sfa[kGSfaBytes];
+    alignas(128) uint8_t sfb[kGSfbBytes];
+};
+
+struct GemmSmem {
+    GemmStage stage[kGStages];
+    alignas(8) uint64_t full[kGStages];
+    uint64_t empty[kGStages];
+    uint64_t tmem_full;
+    uint64_t tmem_empty;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+struct GemmParams {
+    const uint8_t* a_scales;
+    const uint8_t* b_scales;
+    void* out;
+    int64_t ld_out;
+    int32_t M, N, K;
+    int32_t tiles_m, tiles_n;
+    int32_t k_stages;       // ceil(K / 256)
+    int32_t sf_tiles_k;     // ceil(K / 128): 512-byte scale tiles per 128-row block
+    int32_t sf_rows_a;      // ceil(M / 128)
+    int32_t sf_rows_b;      // ceil(N / 128)
+    float alpha;
+    int32_t out_fp32;
+};
+
+// Instruction descriptor of tcgen05.mma kind::mxf4.block_scale: E2M1 x E2M1, E8M0 scales,
+// both operands K-major, M = 128, N = 256.  Scale-factor ids select which byte pair of the
+// 32-bit TMEM scale column an instruction uses.
+__device__ __forceinline__ uint32_t make_idesc_mxf4(uint32_t a_sf_id, uint32_t b_sf_id)
+{
+    uint32_t d = 0;
+    d |= b_sf_id << 4;                 // bits 4..5   B scale-factor id
+    d |= 1u << 7;                      // bits 7..9   A format: E2M1
+    d |= 1u << 10;                     // bits 10..12 B format: E2M1
+    d |= (kGBlockN >> 3) << 17;        // bits 17..22 N / 8
+    d |= 1u << 23;                     // bit 23      scale format: E8M0
+    d |= (kGBlockM >> 4) << 24;        // bits 24..28 M / 16
+    d |= a_sf_id << 29;                // bits 29..30 A scale-factor id
+    return d;
+}
+
+__global__ void __launch_bounds__(kGThreads, 1)
+gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                 const GemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    GemmSmem& sm = *reinterpret_cast<GemmSmem*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int total_tiles = p.tiles_m * p.tiles_n;
+
+    if (threadIdx.x == 0) {
+        sm.abort_flag = 0;
+        for (int s = 0; s < kGStages; ++s) {
+            mbar_init(&sm.full[s], 1);
+            mbar_init(&sm.empty[s], 1);
+        }
+        mbar_init(&sm.tmem_full, 1);
+        mbar_init(&sm.tmem_empty, 4);
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(&sm.tmem_base, kGTmemCols);
+        tmem_relinquish();
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            tma_prefetch_desc(&tm_a);
+            tma_prefetch_desc(&tm_b);
+            int it = 0;
+            bool alive = true;
+            for (int tile = blockIdx.x; alive && tile < total_tiles; tile += gridDim.x) {
+                const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+                for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
+                    const int s = it % kGStages;
+                    const uint32_t round = it / kGStages;
+                    if (round > 0 && !mbar_wait(&sm.empty[s], (round - 1) & 1, &sm.abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    GemmStage& st = sm.stage[s];
+                    const int kt0 = ks * 2;
+                    const int nkt = min(2, p.sf_tiles_k - kt0);
+                    const uint32_t sf_bytes = nkt * 512;
+                    const int nb0 = tn * 2;
+                    const int nnb = min(2, p.sf_rows_b - nb0);
+                    mbar_arrive_expect_tx(&sm.full[s], kGABytes + kGBBytes + sf_bytes * (1 + nnb));
+                    tma_load_2d(st.a, &tm_a, &sm.full[s], ks * 128, tm * kGBlockM);
+                    tma_load_2d(st.b, &tm_b, &sm.full[s], ks * 128, tn * kGBlockN);
+                    bulk_load_1d(st.sfa, p.a_scales + (static_cast<int64_t>(tm) * p.sf_tiles_k + kt0) * 512,
+                                 sf_bytes, &sm.full[s]);
+                    for (int nb = 0; nb < nnb; ++nb)
+                        bulk_load_1d(st.sfb + nb * 1024,
+                                     p.b_scales + (static_cast<int64_t>(nb0 + nb) * p.sf_tiles_k + kt0) * 512,
+                                     sf_bytes, &sm.full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int it = 0, tile_it = 0;
+            bool alive = true;
+            for (int tile = blockIdx.x; alive && tile < total_tiles; tile += gridDim.x, ++tile_it) {
+                if (tile_it > 0 && !mbar_wait(&sm.tmem_empty, (tile_it - 1) & 1, &sm.abort_flag)) break;
+                tcgen05_fence_after();
+                for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
+                    const int s = it % kGStages;
+                    const uint32_t round = it / kGStages;
+                    if (!mbar_wait(&sm.full[s], round & 1, &sm.abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    tcgen05_fence_after();
+                    GemmStage& st = sm.stage[s];
+                    const int valid_k = min(kGBlockK, p.K - ks * kGBlockK);
+                    const int nkt = (valid_k + 127) / 128;
+                    const int nmma = (valid_k + 63) / 64;
+                    const uint32_t sf_tmem = tmem + kGTmemSfBase + (it & 1) * kGTmemSfPerBuf;
+                    for (int kt = 0; kt < nkt; ++kt) {
+                        tcgen05_cp_32x128b_warpx4(sf_tmem + kt * 4,
+                                                  make_smem_desc(smem_u32(st.sfa + kt * 512), 16, 128, 0));
+                        for (int nb = 0; nb < 2; ++nb)
+                            tcgen05_cp_32x128b_warpx4(
+                                sf_tmem + 8 + kt * 8 + nb * 4,
+                                make_smem_desc(smem_u32(st.sfb + nb * 1024 + kt * 512), 16, 128, 0));
+                    }
+                    const uint64_t a_desc = make_smem_desc(smem_u32(st.a), 16, 1024, 2);
+                    const uint64_t b_desc = make_smem_desc(smem_u32(st.b), 16, 1024, 2);
+                    for (int j = 0; j < nmma; ++j) {
+                        const uint32_t sf_id = (j & 1) * 2;
+                        tcgen05_mma_mxf4(tmem, a_desc + 2 * j, b_desc + 2 * j,
+                                         make_idesc_mxf4(sf_id, sf_id), sf_tmem + (j >> 1) * 4,
+                                         sf_tmem + 8 + (j >> 1) * 8, (ks > 0 || j > 0) ? 1u : 0u);
+                    }
+                    tcgen05_commit(&sm.empty[s]);   // stage reusable once these MMAs have read it
+                }
+                if (alive) tcgen05_commit(&sm.tmem_full);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+        int tile_it = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_it) {
+            const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+            if (!mbar_wait(&sm.tmem_full, tile_it & 1, &sm.abort_flag)) break;
+            tcgen05_fence_after();
+            const int64_t row = static_cast<int64_t>(tm) * kGBlockM + quad * 32 + lane;
+            const bool row_ok = row < p.M;
+#pragma unroll 1
+            for (int c = 0; c < kGBlockN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + c * 32, r);
+                tmem_ld_wait();
+                const int64_t col0 = static_cast<int64_t>(tn) * kGBlockN + c * 32;
+                if (!row_ok || col0 >= p.N) continue;
+                if (p.out_fp32) {
+                    float* dst = static_cast<float*>(p.out) + row * p.ld_out + col0;
+                    if (col0 + 32 <= p.N) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            reinterpret_cast<float4*>(dst)[i] =
+                                make_float4(__uint_as_float(r[4 * i]) * p.alpha,
+                                            __uint_as_float(r[4 * i + 1]) * p.alpha,
+                                            __uint_as_float(r[4 * i + 2]) * p.alpha,
+                                            __uint_as_float(r[4 * i + 3]) * p.alpha);
+                    } else {
+                        for (int i = 0; i < 32 && col0 + i < p.N; ++i)
+                            dst[i] = __uint_as_float(r[i]) * p.alpha;
+                    }
+                } else {
+                    __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.out) + row * p.ld_out + col0;
+                    if (col0 + 32 <= p.N) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int h = 0; h < 4; ++h) {
+                                const __nv_bfloat162 v = __floats2bfloat162_rn(
+                                    __uint_as_float(r[8 * i + 2 * h]) * p.alpha,
+                                    __uint_as_float(r[8 * i + 2 * h + 1]) * p.alpha);
+                                w[h] = *reinterpret_cast<const uint32_t*>(&v);
+                            }
+                            reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    } else {
+                        for (int i = 0; i < 32 && col0 + i < p.N; ++i)
+                            dst[i] = __float2bfloat16_rn(__uint_as_float(r[i]) * p.alpha);
+                    }
+                }
+            }
+            // accumulator drained: let the MMA warp start the next tile
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.tmem_empty);
+        }
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        tmem_dealloc(tmem, kGTmemCols);
+    }
+}
+
+static int launch_gemm(const void* a_codes, const void* a_scales, const void* b_codes,
+                       const void* b_scales, int64_t M, int64_t N, int64_t K, float alpha, void* out,
+                       int out_dtype, int64_t ld_out, int sm_count, cudaStream_t stream)
+{
+    CUtensorMap tm_a, tm_b;
+    // codes as bytes: [rows x K/2], box = 128 bytes x (128 | 256) rows, 128-byte swizzle
+    if (!make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a_codes, M, K / 2, K / 2, kGBlockM, 128,
+                      CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b_codes, N, K / 2, K / 2, kGBlockN, 128,
+                      CU_TENSOR_MAP_SWIZZLE_128B))
+        return MXFP4_ERR_CUDA;
+    GemmParams p;
+    p.a_scales = static_cast<const uint8_t*>(a_scales);
+    p.b_scales = static_cast<const uint8_t*>(b_scales);
+    p.out = out;
+    p.ld_out = ld_out;
+    p.M = static_cast<int32_t>(M);
+    p.N = static_cast<int32_t>(N);
+    p.K = static_cast<int32_t>(K);
+    p.tiles_m = static_cast<int32_t>((M + kGBlockM - 1) / kGBlockM);
+    p.tiles_n = static_cast<int32_t>((N + kGBlockN - 1) / kGBlockN);
+    p.k_stages = static_cast<int32_t>((K + kGBlockK - 1) / kGBlockK);
+    p.sf_tiles_k = static_cast<int32_t>((K + 127) / 128);
+    p.sf_rows_a = static_cast<int32_t>((M + 127) / 128);
+    p.sf_rows_b = static_cast<int32_t>((N + 127) / 128);
+    p.alpha = alpha;
+    p.out_fp32 = out_dtype == MXFP4_OUT_FP32;
+    const int64_t total = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
+    if (total > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    const size_t smem = sizeof(GemmSmem) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(gemm_mxf4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess)
+            return MXFP4_ERR_CUDA;
+        attr_set = true;
+    }
+    const int grid = static_cast<int>(total < sm_count ? total : sm_count);
+    gemm_mxf4_kernel<<<grid, kGThreads, smem, stream>>>(tm_a, tm_b, p);
+    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+}  // namespace mxfp4

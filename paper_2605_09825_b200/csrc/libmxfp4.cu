@@ -1,0 +1,331 @@
+// C ABI of the library (see include/mxfp4.h).  Single translation unit: the kernels live in
+// the headers included below.  Host code here only validates arguments, builds TMA tensor
+// maps and launches; every step of the path runs in the kernels.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "../../include/mxfp4.h"
+#include "ptx_sm100.cuh"
+#include "tma_host.cuh"
+#include "quantize_kernel.cuh"
+#include "gemm_kernel.cuh"
+
+namespace mxfp4 {
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int cc_major = 0;
+    bool ok = false;
+};
+
+static const DeviceInfo& device_info()
+{
+    static DeviceInfo info[64];
+    static bool init[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (!init[dev]) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) == cudaSuccess) {
+            info[dev].sm_count = prop.multiProcessorCount;
+            info[dev].cc_major = prop.major;
+            info[dev].ok = true;
+        }
+        init[dev] = true;
+    }
+    return info[dev];
+}
+
+// Host copy of the counter-based generator, used only for the 32-bit sign mask of the
+// randomized rotation (counter (0,0,0,1), key = seed).
+static uint32_t host_sign_mask(uint64_t seed)
+{
+    uint32_t c[4] = {0, 0, 0, 1};
+    uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = 0xD2511F53ull * c[0], p1 = 0xCD9E8D57ull * c[2];
+        const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c[1] ^ k0;
+        const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c[3] ^ k1;
+        c[0] = n0; c[1] = static_cast<uint32_t>(p1); c[2] = n2; c[3] = static_cast<uint32_t>(p0);
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    return c[0];
+}
+
+template <int AXIS, int HMODE, int SR>
+static int launch_quantize(const CUtensorMap& tm_src, const CUtensorMap& tm_codes,
+                           const QuantParams& p, int grid, cudaStream_t stream)
+{
+    const size_t smem = sizeof(QuantSmem) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(quantize_kernel<AXIS, HMODE, SR>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess)
+            return MXFP4_ERR_CUDA;
+        attr_set = true;
+    }
+    quantize_kernel<AXIS, HMODE, SR><<<grid, kQThreads, smem, stream>>>(tm_src, tm_codes, p);
+    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+template <int AXIS>
+static int dispatch_quantize(int hmode, int sr, const CUtensorMap& a, const CUtensorMap& b,
+                             const QuantParams& p, int grid, cudaStream_t st)
+{
+    switch (hmode * 2 + sr) {
+        case 0: return launch_quantize<AXIS, 0, 0>(a, b, p, grid, st);
+        case 1: return launch_quantize<AXIS, 0, 1>(a, b, p, grid, st);
+        case 2: return launch_quantize<AXIS, 1, 0>(a, b, p, grid, st);
+        case 3: return launch_quantize<AXIS, 1, 1>(a, b, p, grid, st);
+        case 4: return launch_quantize<AXIS, 2, 0>(a, b, p, grid, st);
+        default: return launch_quantize<AXIS, 2, 1>(a, b, p, grid, st);
+    }
+}
+
+static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace mxfp4
+
+using namespace mxfp4;
+
+extern "C" {
+
+int mxfp4_version(void) { return 100; }
+
+const char* mxfp4_status_string(int status)
+{
+    switch (status) {
+        case MXFP4_OK: return "ok";
+        case MXFP4_ERR_NULL: return "null pointer";
+        case MXFP4_ERR_SHAPE: return "bad shape";
+        case MXFP4_ERR_ALIGN: return "bad alignment";
+        case MXFP4_ERR_ENUM: return "bad enum value";
+        case MXFP4_ERR_WORKSPACE: return "workspace missing or too small";
+        case MXFP4_ERR_CUDA: return "CUDA call failed";
+        case MXFP4_ERR_TIMEOUT: return "device-side wait timed out";
+        case MXFP4_ERR_DEVICE: return "not an sm_100 device";
+        default: return "unknown status";
+    }
+}
+
+size_t mxfp4_codes_bytes(int64_t outer, int64_t K)
+{
+    if (outer <= 0 || K <= 0 || K % 32 != 0) return 0;
+    return static_cast<size_t>(outer) * static_cast<size_t>(K / 2);
+}
+
+size_t mxfp4_scales_bytes(int64_t outer, int64_t K, int scale_layout)
+{
+    if (outer <= 0 || K <= 0 || K % 32 != 0) return 0;
+    if (scale_layout == MXFP4_SCALES_CANONICAL)
+        return static_cast<size_t>(outer) * static_cast<size_t>(K / 32);
+    if (scale_layout == MXFP4_SCALES_TILED)
+        return static_cast<size_t>((outer + 127) / 128) * static_cast<size_t>((K + 127) / 128) * 512;
+    return 0;
+}
+
+int mxfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis,
+                   int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
+                   void* codes, void* scales, int scale_layout, void* stream)
+{
+    if (!src_bf16 || !codes || !scales) return MXFP4_ERR_NULL;
+    if (axis != 0 && axis != 1) return MXFP4_ERR_ENUM;
+    if (hadamard_mode < 0 || hadamard_mode > 2 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
+    if (scale_layout != 0 && scale_layout != 1) return MXFP4_ERR_ENUM;
+    if (rows <= 0 || cols <= 0 || ld_src < cols) return MXFP4_ERR_SHAPE;
+    const int64_t outer = axis ? rows : cols;
+    const int64_t K = axis ? cols : rows;
+    if (K % 32 != 0) return MXFP4_ERR_SHAPE;
+    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (!aligned16(src_bf16) || !aligned16(codes) || !aligned16(scales)) return MXFP4_ERR_ALIGN;
+    if (ld_src % 8 != 0) return MXFP4_ERR_ALIGN;
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return MXFP4_ERR_CUDA;
+    if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
+
+    CUtensorMap tm_src, tm_codes;
+    const bool ok_src =
+        axis == 1 ? make_tmap_2d(&tm_src, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, src_bf16, rows, cols,
+                                 ld_src * 2, 128, 64, CU_TENSOR_MAP_SWIZZLE_128B)
+                  : make_tmap_2d(&tm_src, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, src_bf16, rows, cols,
+                                 ld_src * 2, 128, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+    const bool ok_codes = make_tmap_2d(&tm_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, outer,
+                                       K / 2, K / 2, 128, 64, CU_TENSOR_MAP_SWIZZLE_64B);
+    if (!ok_src || !ok_codes) return MXFP4_ERR_CUDA;
+
+    QuantParams p;
+    p.scales = static_cast<uint8_t*>(scales);
+    p.outer = outer;
+    p.K = K;
+    p.nt = K / 32;
+    p.tiles_o = static_cast<int32_t>((outer + kQTileO - 1) / kQTileO);
+    p.tiles_k = static_cast<int32_t>((K + kQTileK - 1) / kQTileK);
+    p.seed_lo = static_cast<uint32_t>(seed);
+    p.seed_hi = static_cast<uint32_t>(seed >> 32);
+    p.tag = operand_tag;
+    p.sign_mask = hadamard_mode == MXFP4_HADAMARD_RAND ? host_sign_mask(seed) : 0u;
+    p.scale_layout = scale_layout;
+    const int64_t total = static_cast<int64_t>(p.tiles_o) * p.tiles_k;
+    if (total > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    const int grid = static_cast<int>(total < dev.sm_count ? total : dev.sm_count);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return axis == 1 ? dispatch_quantize<1>(hadamard_mode, rounding, tm_src, tm_codes, p, grid, st)
+                     : dispatch_quantize<0>(hadamard_mode, rounding, tm_src, tm_codes, p, grid, st);
+}
+
+int mxfp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes,
+               const void* b_scales, int64_t M, int64_t N, int64_t K, float alpha, void* out,
+               int out_dtype, int64_t ld_out, void* workspace, size_t workspace_bytes,
+               void* stream)
+{
+    (void)workspace;
+    (void)workspace_bytes;
+    if (!a_codes || !a_scales || !b_codes || !b_scales || !out) return MXFP4_ERR_NULL;
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 32 != 0 || ld_out < N) return MXFP4_ERR_SHAPE;
+    if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (!aligned16(a_codes) || !aligned16(a_scales) || !aligned16(b_codes) || !aligned16(b_scales) ||
+        !aligned16(out))
+        return MXFP4_ERR_ALIGN;
+    const int64_t esz = out_dtype == MXFP4_OUT_BF16 ? 2 : 4;
+    if ((ld_out * esz) % 16 != 0) return MXFP4_ERR_ALIGN;
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return MXFP4_ERR_CUDA;
+    if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
+    return launch_gemm(a_codes, a_scales, b_codes, b_scales, M, N, K, alpha, out, out_dtype, ld_out,
+                       dev.sm_count, static_cast<cudaStream_t>(stream));
+}
+
+// Workspace layout of a fused pass: [A codes][A scales][B codes][B scales], each region
+// rounded up to 1024 bytes.
+static void linear_dims(int pass, int64_t T, int64_t in_f, int64_t out_f, int64_t* M, int64_t* N,
+                        int64_t* K)
+{
+    if (pass == MXFP4_PASS_FPROP) { *M = T; *N = out_f; *K = in_f; }
+    else if (pass == MXFP4_PASS_DGRAD) { *M = T; *N = in_f; *K = out_f; }
+    else { *M = out_f; *N = in_f; *K = T; }
+}
+
+size_t mxfp4_linear_workspace_bytes(int64_t T, int64_t in_features, int64_t out_features, int pass)
+{
+    if (pass < 0 || pass > 2 || T <= 0 || in_features <= 0 || out_features <= 0) return 0;
+    int64_t M, N, K;
+    linear_dims(pass, T, in_features, out_features, &M, &N, &K);
+    if (K % 32 != 0) return 0;
+    return round_up(mxfp4_codes_bytes(M, K), 1024) + round_up(mxfp4_scales_bytes(M, K, 1), 1024) +
+           round_up(mxfp4_codes_bytes(N, K), 1024) + round_up(mxfp4_scales_bytes(N, K, 1), 1024);
+}
+
+static int linear_pass(int pass, const void* a_src, const void* b_src, void* out, int64_t T,
+                       int64_t in_f, int64_t out_f, int hmode, int rounding, uint64_t seed,
+                       int out_dtype, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!a_src || !b_src || !out) return MXFP4_ERR_NULL;
+    if (T <= 0 || in_f <= 0 || out_f <= 0) return MXFP4_ERR_SHAPE;
+    if (hmode < 0 || hmode > 2 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
+    int64_t M, N, K;
+    linear_dims(pass, T, in_f, out_f, &M, &N, &K);
+    if (K % 32 != 0 || in_f % 8 != 0 || out_f % 8 != 0) return MXFP4_ERR_SHAPE;
+    const size_t need = mxfp4_linear_workspace_bytes(T, in_f, out_f, pass);
+    if (!workspace || workspace_bytes < need) return MXFP4_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 1023u) return MXFP4_ERR_ALIGN;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    uint8_t* a_codes = ws;
+    uint8_t* a_scales = a_codes + round_up(mxfp4_codes_bytes(M, K), 1024);
+    uint8_t* b_codes = a_scales + round_up(mxfp4_scales_bytes(M, K, 1), 1024);
+    uint8_t* b_scales = b_codes + round_up(mxfp4_codes_bytes(N, K), 1024);
+
+    // (rows, cols, axis) of each source in its own row-major shape
+    int64_t ar, ac, br, bc;
+    int a_axis, b_axis;
+    if (pass == MXFP4_PASS_FPROP) {          // A = X [T x in] row-wise, B = W [out x in] row-wise
+        ar = T; ac = in_f; a_axis = 1; br = out_f; bc = in_f; b_axis = 1;
+    } else if (pass == MXFP4_PASS_DGRAD) {   // A = dY [T x out] row-wise, B = W [out x in] column-wise
+        ar = T; ac = out_f; a_axis = 1; br = out_f; bc = in_f; b_axis = 0;
+    } else {                                 // A = dY [T x out] column-wise, B = X [T x in] column-wise
+        ar = T; ac = out_f; a_axis = 0; br = T; bc = in_f; b_axis = 0;
+    }
+    int rc = mxfp4_quantize(a_src, ar, ac, ac, a_axis, hmode, rounding, seed, 0u, a_codes, a_scales,
+                            MXFP4_SCALES_TILED, stream);
+    if (rc != MXFP4_OK) return rc;
+    rc = mxfp4_quantize(b_src, br, bc, bc, b_axis, hmode, rounding, seed, 1u, b_codes, b_scales,
+                        MXFP4_SCALES_TILED, stream);
+    if (rc != MXFP4_OK) return rc;
+    const float alpha = hmode != MXFP4_HADAMARD_NONE ? 0.03125f : 1.0f;
+    return mxfp4_gemm(a_codes, a_scales, b_codes, b_scales, M, N, K, alpha, out, out_dtype, N,
+                      nullptr, 0, stream);
+}
+
+int mxfp4_linear_fprop(const void* X, const void* W, void* Y, int64_t T, int64_t in_features,
+                       int64_t out_features, int hadamard_mode, int rounding, uint64_t seed,
+                       int out_dtype, void* workspace, size_t workspace_bytes, void* stream)
+{
+    return linear_pass(MXFP4_PASS_FPROP, X, W, Y, T, in_features, out_features, hadamard_mode,
+                       rounding, seed, out_dtype, workspace, workspace_bytes, stream);
+}
+
+int mxfp4_linear_dgrad(const void* dY, const void* W, void* dX, int64_t T, int64_t in_features,
+                       int64_t out_features, int hadamard_mode, int rounding, uint64_t seed,
+                       int out_dtype, void* workspace, size_t workspace_bytes, void* stream)
+{
+    return linear_pass(MXFP4_PASS_DGRAD, dY, W, dX, T, in_features, out_features, hadamard_mode,
+                       rounding, seed, out_dtype, workspace, workspace_bytes, stream);
+}
+
+int mxfp4_linear_wgrad(const void* dY, const void* X, void* dW, int64_t T, int64_t in_features,
+                       int64_t out_features, int hadamard_mode, int rounding, uint64_t seed,
+                       int out_dtype, void* workspace, size_t workspace_bytes, void* stream)
+{
+    return linear_pass(MXFP4_PASS_WGRAD, dY, X, dW, T, in_features, out_features, hadamard_mode,
+                       rounding, seed, out_dtype, workspace, workspace_bytes, stream);
+}
+
+int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* out_host, int64_t T,
+                      int64_t in_features, int64_t out_features, int hadamard_mode, int rounding,
+                      uint64_t seed, int out_dtype, void* dev_a, void* dev_b, void* dev_out,
+                      void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (pass < 0 || pass > 2) return MXFP4_ERR_ENUM;
+    if (!a_host || !b_host || !out_host || !dev_a || !dev_b || !dev_out) return MXFP4_ERR_NULL;
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
+    if (T <= 0 || in_features <= 0 || out_features <= 0) return MXFP4_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // source shapes: (a, b, out) = (X, W, Y) / (dY, W, dX) / (dY, X, dW)
+    const size_t a_elems = static_cast<size_t>(T) * (pass == MXFP4_PASS_FPROP ? in_features : out_features);
+    const size_t b_elems = pass == MXFP4_PASS_WGRAD ? static_cast<size_t>(T) * in_features
+                                                    : static_cast<size_t>(out_features) * in_features;
+    int64_t M, N, K;
+    linear_dims(pass, T, in_features, out_features, &M, &N, &K);
+    const size_t out_bytes = static_cast<size_t>(M) * N * (out_dtype == MXFP4_OUT_BF16 ? 2 : 4);
+    if (cudaMemcpyAsync(dev_a, a_host, a_elems * 2, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dev_b, b_host, b_elems * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return MXFP4_ERR_CUDA;
+    const int rc = linear_pass(pass, dev_a, dev_b, dev_out, T, in_features, out_features,
+                               hadamard_mode, rounding, seed, out_dtype, workspace, workspace_bytes,
+                               stream);
+    if (rc != MXFP4_OK) return rc;
+    if (cudaMemcpyAsync(out_host, dev_out, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return MXFP4_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+int mxfp4_check(void* stream)
+{
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return MXFP4_ERR_CUDA;
+    int status = 0;
+    if (cudaMemcpyFromSymbol(&status, g_device_status, sizeof(int)) != cudaSuccess)
+        return MXFP4_ERR_CUDA;
+    if (status != 0) {
+        const int zero = 0;
+        cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int));
+    }
+    return status;
+}
+
+}  // extern "C"

@@ -1,0 +1,77 @@
+"""The C-ABI library builds, loads and exports every symbol the header declares; argument
+errors are reported on the host before any device work.  No GPU needed."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2605_09825_b200 import api, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return api.load_library()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "mxfp4.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mxfp4_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(lib):
+    names = _declared_symbols()
+    assert set(names) == set(api.EXPORTS)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_version_and_status_strings(lib):
+    assert api.version() >= 100
+    assert api.status_string(0) == "ok"
+    for code in range(-8, 0):
+        assert api.status_string(code) not in ("ok", "unknown status")
+
+
+def test_size_helpers(lib):
+    assert api.codes_bytes(256, 512) == 256 * 256
+    assert api.scales_bytes(256, 512, api.SCALES_CANONICAL) == 256 * 16
+    assert api.scales_bytes(256, 512, api.SCALES_TILED) == 2 * 4 * 512
+    assert api.scales_bytes(300, 160, api.SCALES_TILED) == 3 * 2 * 512   # padded to whole tiles
+    assert api.codes_bytes(4, 48) == 0 and api.scales_bytes(4, 48, 1) == 0
+    assert api.scales_bytes(4, 64, 7) == 0
+    # fprop at T=256, in=512, out=256: two operands of 256 x 512
+    want = 2 * (256 * 256 + 2 * 4 * 512)
+    assert api.linear_workspace_bytes(256, 512, 256, api.PASS_FPROP) == want
+    assert api.linear_workspace_bytes(256, 512, 256, 5) == 0
+
+
+def test_argument_errors_come_back_as_status_codes(lib):
+    buf = ctypes.create_string_buffer(1 << 16)
+    base = ctypes.addressof(buf)
+    p = (base + 15) & ~15
+    q = lib.mxfp4_quantize
+    assert q(None, 32, 32, 32, 1, 0, 0, 0, 0, p, p, 0, None) == -1            # NULL
+    assert q(p, 32, 32, 32, 2, 0, 0, 0, 0, p, p, 0, None) == -4               # axis
+    assert q(p, 32, 32, 32, 1, 3, 0, 0, 0, p, p, 0, None) == -4               # hadamard mode
+    assert q(p, 32, 32, 32, 1, 0, 2, 0, 0, p, p, 0, None) == -4               # rounding
+    assert q(p, 32, 32, 32, 1, 0, 0, 0, 0, p, p, 9, None) == -4               # layout
+    assert q(p, 32, 48, 48, 1, 0, 0, 0, 0, p, p, 0, None) == -2               # K % 32
+    assert q(p, 48, 32, 32, 0, 0, 0, 0, 0, p, p, 0, None) == -2               # K = rows % 32
+    assert q(p, 32, 64, 32, 1, 0, 0, 0, 0, p, p, 0, None) == -2               # ld < cols
+    assert q(p + 2, 32, 32, 32, 1, 0, 0, 0, 0, p, p, 0, None) == -3           # alignment
+    assert q(p, 32, 32, 36, 1, 0, 0, 0, 0, p, p, 0, None) == -3               # ld % 8
+    g = lib.mxfp4_gemm
+    assert g(None, p, p, p, 128, 128, 128, 1.0, p, 0, 128, None, 0, None) == -1
+    assert g(p, p, p, p, 128, 128, 100, 1.0, p, 0, 128, None, 0, None) == -2
+    assert g(p, p, p, p, 128, 128, 128, 1.0, p, 3, 128, None, 0, None) == -4
+    assert g(p, p, p, p, 128, 128, 128, 1.0, p, 0, 64, None, 0, None) == -2   # ld_out < N
+    assert g(p, p, p, p, 128, 100, 128, 1.0, p, 0, 100, None, 0, None) == -3  # ld_out * 2 % 16
+    f = lib.mxfp4_linear_fprop
+    assert f(p, p, p, 128, 128, 128, 1, 0, 0, 0, None, 0, None) == -5         # no workspace
+    assert f(p, p, p, 128, 100, 128, 1, 0, 0, 0, p, 1 << 15, None) == -2      # in % 32
+    assert f(None, p, p, 128, 128, 128, 1, 0, 0, 0, p, 1 << 15, None) == -1

@@ -1,0 +1,149 @@
+"""CUDA block-scaled GEMM and the fused linear passes vs the CPU oracle, through the C ABI.
+
+Tolerance (stated by the benchmark spec for fp32 outputs): |out - ref| <= 1e-5 * sum|products|; bf16
+outputs add half a bf16 ulp of the reference.  Products of E2M1 values and power-of-two scales
+are exact, so only the fp32 accumulation order differs from the fp64 reference.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import assert_gemm_close, random_bits, to_dev
+from paper_2605_09825_b200 import api, synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _run_gemm(ac, asc, bc, bsc, alpha, out_dtype):
+    out = api.gemm(_dev(ac), _dev(oracle.scales_to_tiled(asc)), _dev(bc), _dev(oracle.scales_to_tiled(bsc)),
+                   alpha, out_dtype)
+    api.check()
+    return out.float().cpu().numpy()
+
+
+def _random_operands(rng, M, N, K, lo=118, hi=136):
+    ac = rng.integers(0, 256, (M, K // 2), dtype=np.uint8)
+    bc = rng.integers(0, 256, (N, K // 2), dtype=np.uint8)
+    asc = rng.integers(lo, hi, (M, K // 32), dtype=np.uint8)
+    bsc = rng.integers(lo, hi, (N, K // 32), dtype=np.uint8)
+    return ac, asc, bc, bsc
+
+
+def test_all_ones_counts_k():
+    M, N, K = 128, 256, 256
+    ac = np.full((M, K // 2), 0x22, np.uint8)
+    bc = np.full((N, K // 2), 0x22, np.uint8)
+    asc = np.full((M, K // 32), 127, np.uint8)
+    bsc = np.full((N, K // 32), 127, np.uint8)
+    out = _run_gemm(ac, asc, bc, bsc, 1.0, api.OUT_FP32)
+    assert (out == K).all()
+
+
+def test_scale_indexing_by_row_and_block():
+    # unit codes; every (row, block) of A and B carries its own exponent, so any mix-up of
+    # rows, 32-row groups, blocks or operands changes the result
+    M, N, K = 256, 512, 512
+    ac = np.full((M, K // 2), 0x22, np.uint8)
+    bc = np.full((N, K // 2), 0x22, np.uint8)
+    rng = np.random.default_rng(3)
+    asc = rng.integers(120, 134, (M, K // 32), dtype=np.uint8)
+    bsc = rng.integers(120, 134, (N, K // 32), dtype=np.uint8)
+    out = _run_gemm(ac, asc, bc, bsc, 1.0, api.OUT_FP32)
+    ref, S = oracle.gemm(ac, asc, bc, bsc)
+    assert_gemm_close(out, ref, S, False, "scale indexing")
+
+
+def test_one_hot_codes_locate_every_k():
+    M, N, K = 128, 256, 512
+    rng = np.random.default_rng(4)
+    ac = np.zeros((M, K // 2), np.uint8)
+    bc = np.full((N, K // 2), 0x22, np.uint8)
+    ks = rng.integers(0, K, M)
+    ac[np.arange(M), ks // 2] = np.where(ks % 2 == 0, 0x06, 0x60).astype(np.uint8)   # 4.0 at k
+    # B holds a different value per k so that the product names the k that was hit
+    vals = rng.integers(1, 8, (N, K)).astype(np.uint8)
+    bc = (vals[:, 0::2] | (vals[:, 1::2] << 4)).astype(np.uint8)
+    asc = np.full((M, K // 32), 127, np.uint8)
+    bsc = np.full((N, K // 32), 127, np.uint8)
+    out = _run_gemm(ac, asc, bc, bsc, 1.0, api.OUT_FP32)
+    ref, _ = oracle.gemm(ac, asc, bc, bsc)
+    assert (out == ref).all()
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 256), (256, 256, 512), (384, 768, 1024), (200, 328, 416),
+                                   (1, 8, 32), (129, 264, 96), (520, 1000, 2080)])
+@pytest.mark.parametrize("out_dtype", [api.OUT_FP32, api.OUT_BF16])
+def test_random_operands_full_compare(M, N, K, out_dtype):
+    rng = np.random.default_rng(M * 31 + N * 7 + K)
+    ac, asc, bc, bsc = _random_operands(rng, M, N, K)
+    out = _run_gemm(ac, asc, bc, bsc, 0.03125, out_dtype)
+    ref, S = oracle.gemm(ac, asc, bc, bsc, alpha=0.03125)
+    assert_gemm_close(out, ref, S, out_dtype == api.OUT_BF16, f"gemm {M}x{N}x{K}")
+
+
+def test_bf16_output_is_the_rounded_fp32_output():
+    rng = np.random.default_rng(9)
+    ac, asc, bc, bsc = _random_operands(rng, 256, 512, 512)
+    f = _run_gemm(ac, asc, bc, bsc, 1.0, api.OUT_FP32)
+    b = _run_gemm(ac, asc, bc, bsc, 1.0, api.OUT_BF16)
+    assert (torch.from_numpy(f).to(torch.bfloat16).float().numpy() == b).all()
+
+
+def test_gemm_is_deterministic_and_respects_ld_out():
+    rng = np.random.default_rng(10)
+    M, N, K = 256, 264, 512
+    ac, asc, bc, bsc = _random_operands(rng, M, N, K)
+    args = (_dev(ac), _dev(oracle.scales_to_tiled(asc)), _dev(bc), _dev(oracle.scales_to_tiled(bsc)))
+    big = torch.full((M, 512), 777.0, dtype=torch.float32, device="cuda")
+    api.gemm(*args, 1.0, api.OUT_FP32, out=big[:, :N])
+    once = api.gemm(*args, 1.0, api.OUT_FP32)
+    api.check()
+    assert (big[:, :N] == once).all() and (big[:, N:] == 777.0).all()
+
+
+def test_config1_fprop_full_output():
+    t = synth.config1()
+    X, W = to_dev(t["X"]), to_dev(t["W"])
+    for hmode in (0, 1, 2):
+        y = api.linear_fprop(X, W, hmode, 0, 7, api.OUT_FP32)
+        api.check()
+        ref, S = oracle.linear_fprop(t["X"], t["W"], hmode, 0, 7)
+        assert_gemm_close(y.cpu().numpy(), ref, S, False, f"config 1 fprop mode {hmode}")
+
+
+@pytest.mark.parametrize("hmode,rnd", [(0, 0), (1, 0), (2, 0), (0, 1)])
+def test_three_passes_small_layer(hmode, rnd):
+    rng = np.random.default_rng(40 + hmode)
+    T, IN, OUT = 384, 512, 320
+    Xb, Wb, dYb = random_bits(rng, T, IN, 2), random_bits(rng, OUT, IN, 2), random_bits(rng, T, OUT, 2)
+    X, W, dY = to_dev(Xb), to_dev(Wb), to_dev(dYb)
+    for out_dtype in (api.OUT_FP32, api.OUT_BF16):
+        bf = out_dtype == api.OUT_BF16
+        y = api.linear_fprop(X, W, hmode, rnd, 7, out_dtype)
+        dx = api.linear_dgrad(dY, W, hmode, rnd, 7, out_dtype)
+        dw = api.linear_wgrad(dY, X, hmode, rnd, 7, out_dtype)
+        api.check()
+        assert_gemm_close(y.float().cpu().numpy(), *oracle.linear_fprop(Xb, Wb, hmode, rnd, 7), bf, "fprop")
+        assert_gemm_close(dx.float().cpu().numpy(), *oracle.linear_dgrad(dYb, Wb, hmode, rnd, 7), bf, "dgrad")
+        assert_gemm_close(dw.float().cpu().numpy(), *oracle.linear_wgrad(dYb, Xb, hmode, rnd, 7), bf, "wgrad")
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    rng = np.random.default_rng(50)
+    T, IN, OUT = 256, 256, 384
+    Xb, Wb = random_bits(rng, T, IN, 2), random_bits(rng, OUT, IN, 2)
+    Xh = torch.from_numpy(Xb.view(np.int16)).view(torch.bfloat16).pin_memory()
+    Wh = torch.from_numpy(Wb.view(np.int16)).view(torch.bfloat16).pin_memory()
+    Yh = torch.empty((T, OUT), dtype=torch.bfloat16).pin_memory()
+    dX, dW_, dY = (torch.empty_like(Xh, device="cuda"), torch.empty_like(Wh, device="cuda"),
+                   torch.empty((T, OUT), dtype=torch.bfloat16, device="cuda"))
+    ws = torch.empty(api.linear_workspace_bytes(T, IN, OUT, api.PASS_FPROP), dtype=torch.uint8, device="cuda")
+    api.linear_host(api.PASS_FPROP, Xh, Wh, Yh, T, IN, OUT, dX, dW_, dY, ws)
+    want = api.linear_fprop(to_dev(Xb), to_dev(Wb))
+    api.check()
+    assert (Yh.cuda() == want).all()

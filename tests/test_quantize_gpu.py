@@ -1,0 +1,131 @@
+"""CUDA quantizer vs the CPU oracle: codes and scales bit-exact, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import gpu_quantize, random_bits, to_dev
+from paper_2605_09825_b200 import api, synth
+
+pytestmark = pytest.mark.gpu
+
+VARIANTS = [(0, 0), (1, 0), (2, 0), (0, 1), (1, 1), (2, 1)]   # (hadamard_mode, rounding)
+
+
+def _check(bits, axis, hmode, rnd, seed=7, tag=1, layout=api.SCALES_TILED):
+    codes, scales, raw = gpu_quantize(bits, axis, hmode, rnd, seed, tag, layout)
+    want_codes, want_scales = oracle.quantize(bits, axis, hmode, rnd, seed, tag)
+    assert codes.shape == want_codes.shape
+    bad = np.argwhere(scales != want_scales)
+    assert bad.size == 0, f"scales differ at {bad[:5].tolist()}: {scales[tuple(bad[0])]} vs {want_scales[tuple(bad[0])]}"
+    bad = np.argwhere(codes != want_codes)
+    assert bad.size == 0, (f"{len(bad)} code bytes differ, first at {bad[:5].tolist()}: "
+                           f"{codes[tuple(bad[0])]:#x} vs {want_codes[tuple(bad[0])]:#x}")
+    return raw
+
+
+@pytest.mark.parametrize("hmode,rnd", VARIANTS)
+@pytest.mark.parametrize("axis", [1, 0])
+def test_config1_tiny(axis, hmode, rnd):
+    t = synth.config1()
+    _check(t["X"], axis, hmode, rnd)
+    _check(t["W"], axis, hmode, rnd, tag=0)
+
+
+@pytest.mark.parametrize("hmode,rnd", VARIANTS)
+@pytest.mark.parametrize("axis", [1, 0])
+@pytest.mark.parametrize("rows,cols", [(32, 32), (1, 64), (96, 160), (300, 416), (1000, 1184), (520, 2048)])
+def test_ragged_shapes_span_tiles_and_tails(rows, cols, axis, hmode, rnd):
+    if axis == 0 and (rows % 32 or cols % 8):
+        pytest.skip("column-wise blocks need rows % 32 == 0 and cols % 8 == 0")
+    if axis == 0 and rows == 1:
+        pytest.skip("K = rows")
+    rng = np.random.default_rng(rows * 7919 + cols)
+    bits = random_bits(rng, rows, cols)
+    raw = _check(bits, axis, hmode, rnd)
+    # padding rows / blocks of the tiled scale buffer hold 0
+    outer, K = (rows, cols) if axis == 1 else (cols, rows)
+    used = np.zeros(raw.size, dtype=bool)
+    o = np.arange(outer)[:, None]
+    t = np.arange(K // 32)[None, :]
+    off = ((o // 128) * ((K // 32 + 3) // 4) + t // 4) * 512 + (o % 32) * 16 + ((o % 128) // 32) * 4 + t % 4
+    used[off] = True
+    assert (raw[~used] == 0).all()
+
+
+def test_one_row_axis1():
+    rng = np.random.default_rng(5)
+    _check(random_bits(rng, 1, 64), 1, 1, 0)
+    _check(random_bits(rng, 3, 32), 1, 1, 1)
+
+
+@pytest.mark.parametrize("axis", [1, 0])
+def test_canonical_scale_layout(axis):
+    rng = np.random.default_rng(17)
+    bits = random_bits(rng, 288, 352)
+    _check(bits, axis, 1, 0, layout=api.SCALES_CANONICAL)
+
+
+def test_strided_source_rows():
+    rng = np.random.default_rng(19)
+    full = random_bits(rng, 200, 512)
+    dev = to_dev(full)
+    view = dev[:, 64:64 + 256]                       # ld = 512, cols = 256, base 128-byte aligned
+    for axis in (1,):
+        codes, scales = api.quantize(view, axis, 1, 0)
+        api.check()
+        want = oracle.quantize(np.ascontiguousarray(full[:, 64:320]), axis, 1, 0)
+        assert (codes.cpu().numpy() == want[0]).all()
+        assert (oracle.scales_from_tiled(scales.cpu().numpy(), 200, 8) == want[1]).all()
+
+
+def test_every_bf16_pattern_and_special_blocks():
+    # all finite bf16 patterns, each as the single non-zero element of a block, plus zero and
+    # negative-zero blocks: exercises sub-normal maxima, the scale clamp and signed zeros
+    pats = np.array([p for p in range(1 << 16) if ((p >> 7) & 0xFF) != 0xFF], dtype=np.uint16)
+    bits = np.zeros((len(pats) + 2, 32), dtype=np.uint16)
+    bits[np.arange(len(pats)), pats % 32] = pats
+    bits[-1, :] = 0x8000
+    for hmode in (0, 1):
+        _check(bits, 1, hmode, 0)
+        _check(bits, 1, hmode, 1)
+
+
+def test_rounding_ties_and_saturation_on_device():
+    vals = np.array([6.0, 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, -0.25, -0.75, -1.25, -1.75, -2.5,
+                     -3.5, -5.0, 7.5, -7.5, 0.0, -0.0, 0.1, -0.1, 5.5, -5.5] + [0.0] * 9, dtype=np.float32)
+    bits = (vals.view(np.uint32) >> 16).astype(np.uint16)[None, :]
+    _check(bits, 1, 0, 0)
+
+
+def test_results_are_reproducible_run_to_run():
+    t = synth.config1()
+    a = gpu_quantize(t["X"], 0, 1, 1, 7, 0)
+    b = gpu_quantize(t["X"], 0, 1, 1, 7, 0)
+    assert (a[0] == b[0]).all() and (a[2] == b[2]).all()
+
+
+def test_canary_bytes_around_outputs_stay_untouched():
+    rng = np.random.default_rng(23)
+    bits = random_bits(rng, 200, 288)
+    src = to_dev(bits)
+    for axis in (1, 0):
+        outer, K = (200, 288) if axis == 1 else (288, 200 // 8 * 8)
+        if axis == 0:
+            src0 = to_dev(bits[:192])
+            outer, K = 288, 192
+        nc, ns = api.codes_bytes(outer, K), api.scales_bytes(outer, K)
+        pad = 4096
+        cbuf = torch.full((nc + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda")
+        sbuf = torch.full((ns + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda")
+        api.quantize(src if axis == 1 else src0, axis, 1, 0,
+                     codes=cbuf[pad:pad + nc].view(outer, K // 2), scales=sbuf[pad:pad + ns])
+        api.check()
+        for buf, n in ((cbuf, nc), (sbuf, ns)):
+            assert (buf[:pad] == 0xA5).all() and (buf[pad + n:] == 0xA5).all()
+
+
+@pytest.mark.parametrize("name,axis", [("X", 1), ("W", 1)])
+def test_config2_full_size(name, axis):
+    t = synth.config2()
+    _check(t[name], axis, 1, 0, seed=0, tag=0)
