@@ -130,7 +130,8 @@ def quantize(src: torch.Tensor, axis: int = AXIS_COLS, hadamard_mode: int = HADA
         codes = torch.empty((outer, K // 2), dtype=torch.uint8, device=src.device)
     if scales is None:
         scales = torch.empty(scales_bytes(outer, K, scale_layout), dtype=torch.uint8, device=src.device)
-    rc = lib.mxfp4_quantize(_dev_ptr(src), rows, cols, src.stride(0), axis, hadamard_mode, rounding,
+    ld = src.stride(0) if rows > 1 else cols   # a single row's stride is arbitrary in torch
+    rc = lib.mxfp4_quantize(_dev_ptr(src), rows, cols, ld, axis, hadamard_mode, rounding,
                             ctypes.c_uint64(seed), ctypes.c_uint32(operand_tag), _dev_ptr(codes),
                             _dev_ptr(scales), scale_layout, _stream())
     _raise(rc, "mxfp4_quantize")
