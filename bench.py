@@ -1,0 +1,436 @@
+#!/usr/bin/env python
+"""Benchmark of the MXFP4 linear-layer hot path on B200.
+
+One "step" is one pass of the whole hot path -- Hadamard + quantize of both operands and the
+block-scaled GEMM, for Fprop, Dgrad and Wgrad of every linear of the workload -- over one batch
+of seeded synthetic tensors shaped like Llama-3.1-8B layers.  The default workload is the full
+layer linear stack at 16384 tokens (12 fused passes = 24 quantize launches + 12 GEMMs), the one
+configuration that exercises every step of the path; ``--workload qkv|gate_up|down`` selects
+the single-linear configurations.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload W] [--impl ours|reference]
+
+Prints ONE JSON line.  ``value`` is whole-job TFLOP/s (2*M*N*K per GEMM, quantize time
+included) with inputs resident in HBM; ``e2e`` is the same metric through the host-buffer
+entry point with the host<->device copies inside the timed region; ``roofline`` describes the
+dominant kernel (the GEMM) from per-launch CUDA-event timings taken in this run;
+``cpu_baseline`` times the CPU oracle on a bounded sample of the same workload.
+With ``--impl reference`` the CPU oracle itself is the timed arm.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "MXFP4 linear-layer TFLOP/s incl. Hadamard+quantize (Fprop+Dgrad+Wgrad)"
+UNIT = "TFLOP/s"
+
+WORKLOADS = {
+    # name: (tokens, [linear names])
+    "layer_stack": (16384, ["qkv", "o", "gate_up", "down"]),
+    "qkv": (8192, ["qkv"]),
+    "gate_up": (8192, ["gate_up"]),
+    "down": (8192, ["down"]),
+}
+
+
+def workload_label(name: str, tokens: int) -> str:
+    if name == "layer_stack":
+        return ("Llama-3.1-8B layer linear stack (QKV, O, gate+up, down) x (Fprop, Dgrad, Wgrad), "
+                f"{tokens} tokens, deterministic H32, RNE")
+    return f"Llama-3.1-8B {name} linear x (Fprop, Dgrad, Wgrad), {tokens} tokens, deterministic H32, RNE"
+
+
+def pass_dims(pass_: int, T: int, in_f: int, out_f: int):
+    if pass_ == 0:
+        return T, out_f, in_f
+    if pass_ == 1:
+        return T, in_f, out_f
+    return out_f, in_f, T
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-i", str(self.index), "-lms", "20"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append((time.time(), ln.strip()))
+
+    def stop(self, t_begin=None, t_end=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+
+        def parse(lines):
+            mhz, mx, watts, reasons = [], None, [], set()
+            for _, ln in lines:
+                f = [x.strip() for x in ln.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    mhz.append(float(f[1]))
+                    mx = float(f[2])
+                    watts.append(float(f[3]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, f[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            return mhz, mx, watts, reasons
+
+        inside = [x for x in self.lines
+                  if t_begin is None or (t_begin <= x[0] <= (t_end or x[0]) + 0.05)]
+        window = "timed region"
+        if not inside:            # region shorter than one sampling period: use the whole run
+            inside, window = self.lines, "whole run (timed region shorter than a sample)"
+        mhz, mx, watts, reasons = parse(inside)
+        return {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": mx,
+                "power_w_max": max(watts) if watts else None, "reasons": sorted(reasons),
+                "samples": len(mhz), "window": window}
+
+
+def aggregate_over_ranks(elapsed_ms: float, world: int) -> float:
+    """Max of the per-rank device times (all ranks run the same work: weak scaling replicas)."""
+    import torch
+    import torch.distributed as dist
+    if world <= 1 or not dist.is_initialized():
+        return elapsed_ms
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# --------------------------------------------------------------------------- oracle arm
+def oracle_sample(steps: int, warmup: int):
+    """Time the CPU oracle on a bounded sample: the QKV Fprop restricted to 2048 tokens."""
+    import oracle
+    from paper_2605_09825_b200 import synth
+    tokens = 2048
+    t = synth.linear_tensors("qkv", tokens, 2, ("X", "W"))
+    flops = 2.0 * tokens * 6144 * 4096
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.linear_fprop(t["X"], t["W"], 1, 0, 0)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    mean = sum(times) / len(times)
+    return {"value": flops / mean / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"QKV Fprop (quantize X [{tokens}x4096] and W [6144x4096] with H32, fp64 GEMM) "
+                      f"restricted to {tokens} tokens; {len(times)} runs, mean {mean:.2f} s"}, mean
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 3))
+    warm = min(args.warmup, 1)
+    base, mean = oracle_sample(steps, warm)
+    tokens, _ = WORKLOADS[args.workload]
+    line = {
+        "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT,
+        "n_gpus": args.gpus, "steps": steps, "warmup": warm, "ms_per_step": mean * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "e2m1 x e2m1 -> f64",
+        "data": "synthetic", "config": {"workload": workload_label(args.workload, tokens),
+                                        "note": "CPU oracle on a bounded sample of this workload"},
+        "cpu_baseline": base,
+        "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- CUDA arm
+def run_ours(args):
+    import torch
+    from paper_2605_09825_b200 import api, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    api.load_library()
+    peaks = load_peaks()
+    tokens, names = WORKLOADS[args.workload]
+    hmode, rnd, seed = api.HADAMARD_DET, api.ROUND_RNE, 0
+
+    # ---- inputs: seeded synthetic, generated on the host, then resident in HBM
+    host, dev_in = {}, {}
+    for n in names:
+        t = synth.linear_tensors(n, tokens, 5)
+        host[n] = {k: torch.from_numpy(v.view(np.int16)).view(torch.bfloat16) for k, v in t.items()}
+        dev_in[n] = {k: v.cuda() for k, v in host[n].items()}
+    dims = {n: synth.LLAMA8B_LINEARS[n] for n in names}   # (out, in)
+    max_out = max(max(tokens * o, tokens * i, o * i) for o, i in dims.values())
+    out_buf = torch.empty(max_out, dtype=torch.bfloat16, device="cuda")
+    ws_bytes = max(api.linear_workspace_bytes(tokens, i, o, p) for o, i in dims.values() for p in range(3))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    lib = api.load_library()
+    stream = torch.cuda.current_stream()
+    sptr = int(stream.cuda_stream)
+
+    passes = []   # (linear, pass, a, b, M, N, K)
+    for n in names:
+        o, i = dims[n]
+        d = dev_in[n]
+        passes.append((n, 0, d["X"], d["W"]) + pass_dims(0, tokens, i, o))
+        passes.append((n, 1, d["dY"], d["W"]) + pass_dims(1, tokens, i, o))
+        passes.append((n, 2, d["dY"], d["X"]) + pass_dims(2, tokens, i, o))
+    flops_per_step = sum(2.0 * M * N * K for (_, _, _, _, M, N, K) in passes)
+    fused = [lib.mxfp4_linear_fprop, lib.mxfp4_linear_dgrad, lib.mxfp4_linear_wgrad]
+
+    def step():
+        for (n, p, a, b, M, N, K) in passes:
+            o, i = dims[n]
+            rc = fused[p](a.data_ptr(), b.data_ptr(), out_buf.data_ptr(), tokens, i, o, hmode, rnd, seed,
+                          api.OUT_BF16, ws.data_ptr(), ws_bytes, sptr)
+            if rc != 0:
+                raise api.Mxfp4Error(rc, "fused linear pass")
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step()
+    api.check()
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    t_begin = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    sync_all()
+    t_end = time.time()
+    elapsed_ms = aggregate_over_ranks(e0.elapsed_time(e1), world)
+    api.check()
+
+    # ---- the same step, decomposed, with CUDA events around every launch (roofline inputs)
+    def a_b_axes(p):
+        return ((1, 1), (1, 0), (0, 0))[p]
+
+    gemm_ms = gemm_flops = quant_ms = quant_bytes = 0.0
+    for rep in range(2):
+        evs = []
+        for (n, p, a, b, M, N, K) in passes:
+            ax_a, ax_b = a_b_axes(p)
+            ac = ws[: M * K // 2].view(M, K // 2)
+            off = (M * K // 2 + 255) // 256 * 256
+            asz = api.scales_bytes(M, K)
+            a_s = ws[off: off + asz]
+            off = off + (asz + 255) // 256 * 256
+            bc = ws[off: off + N * K // 2].view(N, K // 2)
+            off = off + (N * K // 2 + 255) // 256 * 256
+            b_s = ws[off: off + api.scales_bytes(N, K)]
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            ev[0].record(stream)
+            api.quantize(a, ax_a, hmode, rnd, seed, 0, codes=ac, scales=a_s)
+            ev[1].record(stream)
+            api.quantize(b, ax_b, hmode, rnd, seed, 1, codes=bc, scales=b_s)
+            ev[2].record(stream)
+            api.gemm(ac, a_s, bc, b_s, 1.0 / 32, api.OUT_BF16, out=out_buf[: M * N].view(M, N))
+            ev[3].record(stream)
+            evs.append((ev, M, N, K))
+        torch.cuda.synchronize()
+        if rep == 0:
+            continue   # first decomposed pass is a warm-up
+        for ev, M, N, K in evs:
+            quant_ms += ev[0].elapsed_time(ev[1]) + ev[1].elapsed_time(ev[2])
+            quant_bytes += (M + N) * K * 2.53125
+            gemm_ms += ev[2].elapsed_time(ev[3])
+            gemm_flops += 2.0 * M * N * K
+    clocks = sampler.stop(t_begin, t_end)
+    api.check()
+
+    n_gemm = len(passes)
+    fp4_peak = 4.0 * peaks["bf16_tflops_sustained"]
+    gemm_tflops = gemm_flops / (gemm_ms * 1e-3) / 1e12
+    roofline = {
+        "kernel": "gemm_mxf4_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak,
+        "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak, "traffic": None,
+        "peak_source": f"4 x sustained cuBLAS bf16 ({peaks['source']}); burst would be "
+                       f"{4.0 * peaks['bf16_tflops']:.0f}, nominal dense FP4 9000",
+        "flops_per_launch": gemm_flops / n_gemm, "avg_launch_ms": gemm_ms / n_gemm,
+    }
+    quant_gbs = quant_bytes / (quant_ms * 1e-3) / 1e9
+    quantize_info = {"kernel": "quantize_kernel", "bound": "hbm", "achieved": quant_gbs,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"],
+                     "bytes_per_element": 2.53125, "avg_launch_ms": quant_ms / (2 * n_gemm)}
+
+    # ---- end to end: host buffers in, host buffer out, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        pin = {n: {k: v.pin_memory() for k, v in host[n].items()} for n in names}
+        out_host = torch.empty(max_out, dtype=torch.bfloat16).pin_memory()
+        stage_a = torch.empty(max(tokens * max(o, i) for o, i in dims.values()), dtype=torch.bfloat16, device="cuda")
+        stage_b = torch.empty(max(max(tokens * i, o * i) for o, i in dims.values()), dtype=torch.bfloat16, device="cuda")
+        h2d = d2h = 0
+        for (n, p, a, b, M, N, K) in passes:
+            h2d += (a.numel() + b.numel()) * 2
+            d2h += M * N * 2
+
+        def e2e_step():
+            for (n, p, a, b, M, N, K) in passes:
+                o, i = dims[n]
+                ah = pin[n]["X" if p == 0 else "dY"]
+                bh = pin[n]["X" if p == 2 else "W"]
+                rc = lib.mxfp4_linear_host(p, ah.data_ptr(), bh.data_ptr(), out_host.data_ptr(), tokens, i, o,
+                                           hmode, rnd, seed, api.OUT_BF16, stage_a.data_ptr(), stage_b.data_ptr(),
+                                           out_buf.data_ptr(), ws.data_ptr(), ws_bytes, sptr)
+                if rc != 0:
+                    raise api.Mxfp4Error(rc, "mxfp4_linear_host")
+
+        e2e_step()
+        n_e2e = max(1, min(args.steps, 3))
+        sync_all()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            e2e_step()
+        sync_all()
+        e2e_ms = aggregate_over_ranks((time.perf_counter() - t0) * 1e3, world)
+        e2e = {"value": world * flops_per_step * n_e2e / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
+               "ms_per_step": e2e_ms / n_e2e,
+               "note": "mxfp4_linear_host per pass: pinned host inputs copied in, result copied out, "
+                       "stream drained each call"}
+
+    # ---- context: cuBLAS bf16 and FP8 on the same GEMM shapes (not the target)
+    context = {}
+    if not args.no_context:
+        try:
+            def time_fn(fn, reps=3):
+                fn()
+                torch.cuda.synchronize()
+                a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a0.record()
+                for _ in range(reps):
+                    fn()
+                a1.record()
+                torch.cuda.synchronize()
+                return a0.elapsed_time(a1) / reps
+            bf_ms = f8_ms = 0.0
+            for (n, p, a, b, M, N, K) in passes:
+                A = torch.randn(M, K, device="cuda", dtype=torch.bfloat16)
+                B = torch.randn(N, K, device="cuda", dtype=torch.bfloat16)
+                bf_ms += time_fn(lambda: torch.matmul(A, B.t()))
+                A8, B8 = A.to(torch.float8_e4m3fn), B.to(torch.float8_e4m3fn)
+                one = torch.ones((), device="cuda", dtype=torch.float32)
+                f8_ms += time_fn(lambda: torch._scaled_mm(A8, B8.t(), scale_a=one, scale_b=one,
+                                                          out_dtype=torch.bfloat16))
+                del A, B, A8, B8
+            context = {"cublas_bf16_tflops": flops_per_step / (bf_ms * 1e-3) / 1e12,
+                       "cublas_fp8_tflops": flops_per_step / (f8_ms * 1e-3) / 1e12,
+                       "note": "GEMMs only (no quantize/cast time), same 12 shapes"}
+        except Exception as exc:   # context only
+            context = {"error": repr(exc)[:200]}
+
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    cpu_base = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu_base, _ = oracle_sample(2, 1)   # about 15 s of host time
+
+    ms_per_step = elapsed_ms / args.steps
+    line = {
+        "metric": METRIC, "value": world * flops_per_step / (ms_per_step * 1e-3) / 1e12, "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "e2m1 (mxfp4) x e2m1, f32 accumulate",
+        "data": "synthetic",
+        "config": {"workload": workload_label(args.workload, tokens), "passes_per_step": len(passes),
+                   "flops_per_step": flops_per_step, "out_dtype": "bf16",
+                   "l2": "inputs larger than L2 (several GB per step), no flush needed",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "roofline": roofline, "quantize": quantize_info,
+        "frac_of_nominal_fp4_peak": world and (flops_per_step / (ms_per_step * 1e-3) / 1e12) / 9000.0,
+        "cpu_baseline": cpu_base, "e2e": e2e, "gpu_launches": 3 * len(passes) * args.steps,
+        "clocks": clocks, "context": context,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="layer_stack", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-context", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

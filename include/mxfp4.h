@@ -124,7 +124,7 @@ int mxfp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes,
 
 /*
  * Workspace (device bytes) the fused linear passes need for the two quantized operands:
- * codes + tiled scales of both, each region 1024-byte aligned.  pass = MXFP4_PASS_*.
+ * codes + tiled scales of both, each region 256-byte aligned.  pass = MXFP4_PASS_*.
  */
 size_t mxfp4_linear_workspace_bytes(int64_t T, int64_t in_features, int64_t out_features, int pass);
 
@@ -137,7 +137,7 @@ size_t mxfp4_linear_workspace_bytes(int64_t T, int64_t in_features, int64_t out_
  *   dgrad: dX[T x in]   = dY[T x out]  * W[out x in]     (dY row-wise along `out`; W column-wise)
  *   wgrad: dW[out x in] = dY[T x out]^T * X[T x in]      (both column-wise along tokens)
  * The reduction size (in / out / T respectively) must be a multiple of 32, all widths
- * multiples of 8.  workspace >= mxfp4_linear_workspace_bytes(...), 1024-byte aligned.
+ * multiples of 8.  workspace >= mxfp4_linear_workspace_bytes(...), 256-byte aligned.
  */
 int mxfp4_linear_fprop(const void* X, const void* W, void* Y, int64_t T, int64_t in_features,
                        int64_t out_features, int hadamard_mode, int rounding, uint64_t seed,

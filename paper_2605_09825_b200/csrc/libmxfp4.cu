@@ -203,7 +203,7 @@ int mxfp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes,
 }
 
 // Workspace layout of a fused pass: [A codes][A scales][B codes][B scales], each region
-// rounded up to 1024 bytes.
+// rounded up to 256 bytes.
 static void linear_dims(int pass, int64_t T, int64_t in_f, int64_t out_f, int64_t* M, int64_t* N,
                         int64_t* K)
 {
@@ -218,8 +218,8 @@ size_t mxfp4_linear_workspace_bytes(int64_t T, int64_t in_features, int64_t out_
     int64_t M, N, K;
     linear_dims(pass, T, in_features, out_features, &M, &N, &K);
     if (K % 32 != 0) return 0;
-    return round_up(mxfp4_codes_bytes(M, K), 1024) + round_up(mxfp4_scales_bytes(M, K, 1), 1024) +
-           round_up(mxfp4_codes_bytes(N, K), 1024) + round_up(mxfp4_scales_bytes(N, K, 1), 1024);
+    return round_up(mxfp4_codes_bytes(M, K), 256) + round_up(mxfp4_scales_bytes(M, K, 1), 256) +
+           round_up(mxfp4_codes_bytes(N, K), 256) + round_up(mxfp4_scales_bytes(N, K, 1), 256);
 }
 
 static int linear_pass(int pass, const void* a_src, const void* b_src, void* out, int64_t T,
@@ -234,12 +234,12 @@ static int linear_pass(int pass, const void* a_src, const void* b_src, void* out
     if (K % 32 != 0 || in_f % 8 != 0 || out_f % 8 != 0) return MXFP4_ERR_SHAPE;
     const size_t need = mxfp4_linear_workspace_bytes(T, in_f, out_f, pass);
     if (!workspace || workspace_bytes < need) return MXFP4_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(workspace) & 1023u) return MXFP4_ERR_ALIGN;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MXFP4_ERR_ALIGN;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     uint8_t* a_codes = ws;
-    uint8_t* a_scales = a_codes + round_up(mxfp4_codes_bytes(M, K), 1024);
-    uint8_t* b_codes = a_scales + round_up(mxfp4_scales_bytes(M, K, 1), 1024);
-    uint8_t* b_scales = b_codes + round_up(mxfp4_codes_bytes(N, K), 1024);
+    uint8_t* a_scales = a_codes + round_up(mxfp4_codes_bytes(M, K), 256);
+    uint8_t* b_codes = a_scales + round_up(mxfp4_scales_bytes(M, K, 1), 256);
+    uint8_t* b_scales = b_codes + round_up(mxfp4_codes_bytes(N, K), 256);
 
     // (rows, cols, axis) of each source in its own row-major shape
     int64_t ar, ac, br, bc;
