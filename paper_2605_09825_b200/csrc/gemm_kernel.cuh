@@ -6,10 +6,15 @@
 //   warp 0      TMA producer: per K-step of 256 elements loads A (128 rows x 128 B of packed
 //               codes) and B (256 rows x 128 B) in the 128-byte swizzle, plus the matching
 //               scale tiles (512-byte blocks of 128 rows x 4 MX blocks), into a 4-stage ring.
-//   warp 1      MMA issuer: copies the scale tiles shared memory -> TMEM (tcgen05.cp), then
-//               issues four tcgen05.mma kind::mxf4.block_scale (K = 64 each) per stage; the
-//               fp32 accumulator (128 lanes x 256 columns) lives in TMEM.
-//   warps 2..5  epilogue: TMEM -> registers (tcgen05.ld), * alpha, bf16/fp32, global stores.
+//   warp 1      MMA issuer: copies the scale tiles shared memory -> TMEM (tcgen05.cp) one
+//               stage ahead of the math, then issues four tcgen05.mma kind::mxf4.block_scale
+//               (K = 64 each) per stage; the fp32 accumulator (128 lanes x 256 columns) lives
+//               in TMEM.
+//   warps 2..9  epilogue: each warp pulls its 32 rows x 128 columns out of TMEM with four
+//               back-to-back tcgen05.ld, hands the accumulator back to the MMA warp at once,
+//               and only then scales by alpha, converts and stores (bf16 through a small
+//               swizzled shared-memory staging buffer so that global stores are coalesced),
+//               overlapping with the next tile's main loop.
 // All waits are bounded (see ptx_sm100.cuh).
 #pragma once
 
@@ -32,20 +37,18 @@ constexpr int kGABytes = kGBlockM * 128;         // 16 KB
 constexpr int kGBBytes = kGBlockN * 128;         // 32 KB
 constexpr int kGSfaBytes = 2 * 512;              // 2 K-tiles of 128 elements
 constexpr int kGSfbBytes = 2 * 2 * 512;          // 2 row blocks x 2 K-tiles
-constexpr int kGThreads = 192;
+constexpr int kGEpiWarps = 8;
+constexpr int kGThreads = 64 + 32 * kGEpiWarps;
 constexpr uint32_t kGTmemCols = 512;
 constexpr uint32_t kGTmemSfBase = 256;           // accumulator occupies columns 0..255
 constexpr uint32_t kGTmemSfPerBuf = 24;          // 8 columns SFA + 16 columns SFB
 
-struct GemmStage {
-    alignas(1024) uint8_t a[kGABytes];
-    alignas(1024) uint8_t b[kGBBytes];
-    alignas(128) uint8_t sfa[kGSfaBytes];
-    alignas(128) uint8_t sfb[kGSfbBytes];
-};
-
 struct GemmSmem {
-    GemmStage stage[kGStages];
+    alignas(1024) uint8_t a[kGStages][kGABytes];
+    alignas(1024) uint8_t b[kGStages][kGBBytes];
+    alignas(128) uint8_t sfa[kGStages][kGSfaBytes];
+    alignas(128) uint8_t sfb[kGStages][kGSfbBytes];
+    alignas(128) uint8_t out_stage[kGEpiWarps][32 * 64];   // 32 rows x 32 bf16 per warp
     alignas(8) uint64_t full[kGStages];
     uint64_t empty[kGStages];
     uint64_t tmem_full;
@@ -63,7 +66,6 @@ struct GemmParams {
     int32_t tiles_m, tiles_n;
     int32_t k_stages;       // ceil(K / 256)
     int32_t sf_tiles_k;     // ceil(K / 128): 512-byte scale tiles per 128-row block
-    int32_t sf_rows_a;      // ceil(M / 128)
     int32_t sf_rows_b;      // ceil(N / 128)
     float alpha;
     int32_t out_fp32;
@@ -85,6 +87,20 @@ __device__ __forceinline__ uint32_t make_idesc_mxf4(uint32_t a_sf_id, uint32_t b
     return d;
 }
 
+// Scale tiles of ring stage `s` -> TMEM scale buffer `sf_tmem` (SFA: 4 columns per K-tile;
+// SFB: 8 columns per K-tile, 4 per 128-row block).
+__device__ __forceinline__ void copy_scales_to_tmem(GemmSmem& sm, int s, uint32_t sf_tmem, int nkt)
+{
+    for (int kt = 0; kt < nkt; ++kt) {
+        tcgen05_cp_32x128b_warpx4(sf_tmem + kt * 4,
+                                  make_smem_desc(smem_u32(&sm.sfa[s][kt * 512]), 16, 128, 0));
+#pragma unroll
+        for (int nb = 0; nb < 2; ++nb)
+            tcgen05_cp_32x128b_warpx4(sf_tmem + 8 + kt * 8 + nb * 4,
+                                      make_smem_desc(smem_u32(&sm.sfb[s][nb * 1024 + kt * 512]), 16, 128, 0));
+    }
+}
+
 __global__ void __launch_bounds__(kGThreads, 1)
 gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                  const GemmParams p)
@@ -95,6 +111,7 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int total_tiles = p.tiles_m * p.tiles_n;
+    const int my_tiles = blockIdx.x < total_tiles ? (total_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
 
     if (threadIdx.x == 0) {
         sm.abort_flag = 0;
@@ -103,7 +120,7 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             mbar_init(&sm.empty[s], 1);
         }
         mbar_init(&sm.tmem_full, 1);
-        mbar_init(&sm.tmem_empty, 4);
+        mbar_init(&sm.tmem_empty, kGEpiWarps);
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -131,19 +148,18 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                         alive = false;
                         break;
                     }
-                    GemmStage& st = sm.stage[s];
                     const int kt0 = ks * 2;
                     const int nkt = min(2, p.sf_tiles_k - kt0);
                     const uint32_t sf_bytes = nkt * 512;
                     const int nb0 = tn * 2;
                     const int nnb = min(2, p.sf_rows_b - nb0);
                     mbar_arrive_expect_tx(&sm.full[s], kGABytes + kGBBytes + sf_bytes * (1 + nnb));
-                    tma_load_2d(st.a, &tm_a, &sm.full[s], ks * 128, tm * kGBlockM);
-                    tma_load_2d(st.b, &tm_b, &sm.full[s], ks * 128, tn * kGBlockN);
-                    bulk_load_1d(st.sfa, p.a_scales + (static_cast<int64_t>(tm) * p.sf_tiles_k + kt0) * 512,
+                    tma_load_2d(sm.a[s], &tm_a, &sm.full[s], ks * 128, tm * kGBlockM);
+                    tma_load_2d(sm.b[s], &tm_b, &sm.full[s], ks * 128, tn * kGBlockN);
+                    bulk_load_1d(sm.sfa[s], p.a_scales + (static_cast<int64_t>(tm) * p.sf_tiles_k + kt0) * 512,
                                  sf_bytes, &sm.full[s]);
                     for (int nb = 0; nb < nnb; ++nb)
-                        bulk_load_1d(st.sfb + nb * 1024,
+                        bulk_load_1d(&sm.sfb[s][nb * 1024],
                                      p.b_scales + (static_cast<int64_t>(nb0 + nb) * p.sf_tiles_k + kt0) * 512,
                                      sf_bytes, &sm.full[s]);
                 }
@@ -152,34 +168,41 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            int it = 0, tile_it = 0;
-            bool alive = true;
-            for (int tile = blockIdx.x; alive && tile < total_tiles; tile += gridDim.x, ++tile_it) {
+            const int total_it = my_tiles * p.k_stages;
+            bool alive = total_it > 0;
+            // scales of the very first stage; afterwards each iteration copies the next one's
+            if (alive) {
+                alive = mbar_wait(&sm.full[0], 0, &sm.abort_flag);
+                if (alive) {
+                    tcgen05_fence_after();
+                    copy_scales_to_tmem(sm, 0, tmem + kGTmemSfBase, (min(kGBlockK, p.K) + 127) / 128);
+                }
+            }
+            int it = 0;
+            for (int tile_it = 0; alive && tile_it < my_tiles; ++tile_it) {
                 if (tile_it > 0 && !mbar_wait(&sm.tmem_empty, (tile_it - 1) & 1, &sm.abort_flag)) break;
                 tcgen05_fence_after();
                 for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
                     const int s = it % kGStages;
-                    const uint32_t round = it / kGStages;
-                    if (!mbar_wait(&sm.full[s], round & 1, &sm.abort_flag)) {
-                        alive = false;
-                        break;
-                    }
-                    tcgen05_fence_after();
-                    GemmStage& st = sm.stage[s];
-                    const int valid_k = min(kGBlockK, p.K - ks * kGBlockK);
-                    const int nkt = (valid_k + 127) / 128;
-                    const int nmma = (valid_k + 63) / 64;
                     const uint32_t sf_tmem = tmem + kGTmemSfBase + (it & 1) * kGTmemSfPerBuf;
-                    for (int kt = 0; kt < nkt; ++kt) {
-                        tcgen05_cp_32x128b_warpx4(sf_tmem + kt * 4,
-                                                  make_smem_desc(smem_u32(st.sfa + kt * 512), 16, 128, 0));
-                        for (int nb = 0; nb < 2; ++nb)
-                            tcgen05_cp_32x128b_warpx4(
-                                sf_tmem + 8 + kt * 8 + nb * 4,
-                                make_smem_desc(smem_u32(st.sfb + nb * 1024 + kt * 512), 16, 128, 0));
+                    if (it + 1 < total_it) {
+                        // next stage's scales go to the other TMEM scale buffer while this
+                        // stage's MMAs run
+                        const int s1 = (it + 1) % kGStages;
+                        if (!mbar_wait(&sm.full[s1], ((it + 1) / kGStages) & 1, &sm.abort_flag)) {
+                            alive = false;
+                            break;
+                        }
+                        tcgen05_fence_after();
+                        const int ks1 = (ks + 1 == p.k_stages) ? 0 : ks + 1;
+                        const int vk1 = min(kGBlockK, p.K - ks1 * kGBlockK);
+                        copy_scales_to_tmem(sm, s1, tmem + kGTmemSfBase + ((it + 1) & 1) * kGTmemSfPerBuf,
+                                            (vk1 + 127) / 128);
                     }
-                    const uint64_t a_desc = make_smem_desc(smem_u32(st.a), 16, 1024, 2);
-                    const uint64_t b_desc = make_smem_desc(smem_u32(st.b), 16, 1024, 2);
+                    const int valid_k = min(kGBlockK, p.K - ks * kGBlockK);
+                    const int nmma = (valid_k + 63) / 64;
+                    const uint64_t a_desc = make_smem_desc(smem_u32(sm.a[s]), 16, 1024, 2);
+                    const uint64_t b_desc = make_smem_desc(smem_u32(sm.b[s]), 16, 1024, 2);
                     for (int j = 0; j < nmma; ++j) {
                         const uint32_t sf_id = (j & 1) * 2;
                         tcgen05_mma_mxf4(tmem, a_desc + 2 * j, b_desc + 2 * j,
@@ -193,60 +216,89 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
+        const int ew = warp - 2;
         const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+        const int half = ew >> 2;                  // which 128 accumulator columns
+        uint8_t* stg = sm.out_stage[ew];
         int tile_it = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_it) {
             const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
             if (!mbar_wait(&sm.tmem_full, tile_it & 1, &sm.abort_flag)) break;
             tcgen05_fence_after();
-            const int64_t row = static_cast<int64_t>(tm) * kGBlockM + quad * 32 + lane;
-            const bool row_ok = row < p.M;
-#pragma unroll 1
-            for (int c = 0; c < kGBlockN / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld_32x32b_x32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + c * 32, r);
-                tmem_ld_wait();
-                const int64_t col0 = static_cast<int64_t>(tn) * kGBlockN + c * 32;
-                if (!row_ok || col0 >= p.N) continue;
-                if (p.out_fp32) {
+            uint32_t r[4][32];
+            const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + half * 128;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(taddr + c * 32, r[c]);
+            tmem_ld_wait();
+            // the accumulator is in registers: release TMEM before converting and storing
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.tmem_empty);
+
+            const int64_t row0 = static_cast<int64_t>(tm) * kGBlockM + quad * 32;
+            const int64_t colbase = static_cast<int64_t>(tn) * kGBlockN + half * 128;
+            if (p.out_fp32) {
+                const int64_t row = row0 + lane;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int64_t col0 = colbase + c * 32;
+                    if (row >= p.M || col0 >= p.N) continue;
                     float* dst = static_cast<float*>(p.out) + row * p.ld_out + col0;
                     if (col0 + 32 <= p.N) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
                             reinterpret_cast<float4*>(dst)[i] =
-                                make_float4(__uint_as_float(r[4 * i]) * p.alpha,
-                                            __uint_as_float(r[4 * i + 1]) * p.alpha,
-                                            __uint_as_float(r[4 * i + 2]) * p.alpha,
-                                            __uint_as_float(r[4 * i + 3]) * p.alpha);
+                                make_float4(__uint_as_float(r[c][4 * i]) * p.alpha,
+                                            __uint_as_float(r[c][4 * i + 1]) * p.alpha,
+                                            __uint_as_float(r[c][4 * i + 2]) * p.alpha,
+                                            __uint_as_float(r[c][4 * i + 3]) * p.alpha);
                     } else {
-                        for (int i = 0; i < 32 && col0 + i < p.N; ++i)
-                            dst[i] = __uint_as_float(r[i]) * p.alpha;
-                    }
-                } else {
-                    __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.out) + row * p.ld_out + col0;
-                    if (col0 + 32 <= p.N) {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int h = 0; h < 4; ++h) {
-                                const __nv_bfloat162 v = __floats2bfloat162_rn(
-                                    __uint_as_float(r[8 * i + 2 * h]) * p.alpha,
-                                    __uint_as_float(r[8 * i + 2 * h + 1]) * p.alpha);
-                                w[h] = *reinterpret_cast<const uint32_t*>(&v);
-                            }
-                            reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[0], w[1], w[2], w[3]);
-                        }
-                    } else {
-                        for (int i = 0; i < 32 && col0 + i < p.N; ++i)
-                            dst[i] = __float2bfloat16_rn(__uint_as_float(r[i]) * p.alpha);
+                        for (int i = 0; i < 32; ++i)
+                            if (col0 + i < p.N) dst[i] = __uint_as_float(r[c][i]) * p.alpha;
                     }
                 }
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    // own row (= lane), 32 columns -> 64 bytes, 16-byte chunk q stored at
+                    // q ^ ((lane >> 1) & 3) so that both the row-wise writes and the
+                    // 8-rows-per-instruction reads below are bank-conflict free
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int h = 0; h < 4; ++h) {
+                            const __nv_bfloat162 v = __floats2bfloat162_rn(
+                                __uint_as_float(r[c][8 * q + 2 * h]) * p.alpha,
+                                __uint_as_float(r[c][8 * q + 2 * h + 1]) * p.alpha);
+                            w[h] = *reinterpret_cast<const uint32_t*>(&v);
+                        }
+                        *reinterpret_cast<uint4*>(stg + lane * 64 + ((q ^ ((lane >> 1) & 3)) * 16)) =
+                            make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                    __syncwarp();
+                    const int64_t col0 = colbase + c * 32 + (lane & 3) * 8;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int rr = i * 8 + (lane >> 2);
+                        const uint4 v = *reinterpret_cast<const uint4*>(
+                            stg + rr * 64 + (((lane & 3) ^ ((rr >> 1) & 3)) * 16));
+                        const int64_t row = row0 + rr;
+                        if (row < p.M && col0 < p.N) {
+                            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.out) + row * p.ld_out + col0;
+                            if (col0 + 8 <= p.N) {
+                                *reinterpret_cast<uint4*>(dst) = v;
+                            } else {
+                                const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+                                for (int k = 0; k < 8; ++k)
+                                    if (col0 + k < p.N) dst[k] = e[k];
+                            }
+                        }
+                    }
+                    __syncwarp();
+                }
             }
-            // accumulator drained: let the MMA warp start the next tile
-            tcgen05_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.tmem_empty);
         }
     }
 
@@ -281,7 +333,6 @@ static int launch_gemm(const void* a_codes, const void* a_scales, const void* b_
     p.tiles_n = static_cast<int32_t>((N + kGBlockN - 1) / kGBlockN);
     p.k_stages = static_cast<int32_t>((K + kGBlockK - 1) / kGBlockK);
     p.sf_tiles_k = static_cast<int32_t>((K + 127) / 128);
-    p.sf_rows_a = static_cast<int32_t>((M + 127) / 128);
     p.sf_rows_b = static_cast<int32_t>((N + 127) / 128);
     p.alpha = alpha;
     p.out_fp32 = out_dtype == MXFP4_OUT_FP32;
