@@ -3,19 +3,22 @@
 //   out[m][n] = alpha * sum_t 2^(sa[m][t]-127) 2^(sb[n][t]-127) sum_{k in block t} A[m][k] B[n][k]
 //
 // Persistent, warp-specialised, one CTA per SM, output tile 128 x 256:
-//   warp 0      TMA producer: per K-step of 256 elements loads A (128 rows x 128 B of packed
+//   warp 12      TMA producer: per K-step of 256 elements loads A (128 rows x 128 B of packed
 //               codes) and B (256 rows x 128 B) in the 128-byte swizzle, plus the matching
 //               scale tiles (512-byte blocks of 128 rows x 4 MX blocks), into a 4-stage ring.
-//   warp 1      MMA issuer: copies the scale tiles shared memory -> TMEM (tcgen05.cp) one
-//               stage ahead of the math, then issues four tcgen05.mma kind::mxf4.block_scale
-//               (K = 64 each) per stage; the fp32 accumulator (128 lanes x 256 columns) lives
-//               in TMEM.
-//   warps 2..9  epilogue: each warp pulls its 32 rows x 128 columns out of TMEM with four
+//   warps 0..3   scale warps (one per TMEM lane quadrant): read each stage's scale tiles from
+//                shared memory and write them into that stage's TMEM scale columns with
+//                tcgen05.st.  (A tcgen05.cp would do the same copy, but each one occupies the
+//                tensor pipe for about as long as an MMA and six are needed per stage.)
+//   warps 4..11  epilogue: each warp pulls its 32 rows x 128 columns out of TMEM with four
 //               back-to-back tcgen05.ld, hands the accumulator back to the MMA warp at once,
 //               and only then scales by alpha, converts and stores (bf16 through a small
 //               swizzled shared-memory staging buffer so that global stores are coalesced),
 //               overlapping with the next tile's main loop.
-// All waits are bounded (see ptx_sm100.cuh).
+//   warp 13      MMA issuer: four tcgen05.mma kind::mxf4.block_scale (K = 64 each) per stage;
+//                the fp32 accumulator (128 lanes x 256 columns) lives in TMEM.
+// Registers are rebalanced with setmaxnreg: the epilogue warps hold 128 accumulator values
+// per thread, the other roles need few.  All waits are bounded (see ptx_sm100.cuh).
 #pragma once
 
 #include <cuda.h>
@@ -38,10 +41,12 @@ constexpr int kGBBytes = kGBlockN * 128;         // 32 KB
 constexpr int kGSfaBytes = 2 * 512;              // 2 K-tiles of 128 elements
 constexpr int kGSfbBytes = 2 * 2 * 512;          // 2 row blocks x 2 K-tiles
 constexpr int kGEpiWarps = 8;
-constexpr int kGThreads = 64 + 32 * kGEpiWarps;
+constexpr int kGProducerWarp = 12;
+constexpr int kGMmaWarp = 13;
+constexpr int kGThreads = 512;                   // 4 warpgroups: scales | epilogue x2 | producer+MMA
 constexpr uint32_t kGTmemCols = 512;
 constexpr uint32_t kGTmemSfBase = 256;           // accumulator occupies columns 0..255
-constexpr uint32_t kGTmemSfPerBuf = 24;          // 8 columns SFA + 16 columns SFB
+constexpr uint32_t kGTmemSfPerBuf = 24;          // per stage: 8 columns SFA + 16 columns SFB
 
 struct GemmSmem {
     alignas(1024) uint8_t a[kGStages][kGABytes];
@@ -51,6 +56,7 @@ struct GemmSmem {
     alignas(128) uint8_t out_stage[kGEpiWarps][32 * 64];   // 32 rows x 32 bf16 per warp
     alignas(8) uint64_t full[kGStages];
     uint64_t empty[kGStages];
+    uint64_t sf_ready[kGStages];
     uint64_t tmem_full;
     uint64_t tmem_empty;
     uint32_t tmem_base;
@@ -87,20 +93,6 @@ __device__ __forceinline__ uint32_t make_idesc_mxf4(uint32_t a_sf_id, uint32_t b
     return d;
 }
 
-// Scale tiles of ring stage `s` -> TMEM scale buffer `sf_tmem` (SFA: 4 columns per K-tile;
-// SFB: 8 columns per K-tile, 4 per 128-row block).
-__device__ __forceinline__ void copy_scales_to_tmem(GemmSmem& sm, int s, uint32_t sf_tmem, int nkt)
-{
-    for (int kt = 0; kt < nkt; ++kt) {
-        tcgen05_cp_32x128b_warpx4(sf_tmem + kt * 4,
-                                  make_smem_desc(smem_u32(&sm.sfa[s][kt * 512]), 16, 128, 0));
-#pragma unroll
-        for (int nb = 0; nb < 2; ++nb)
-            tcgen05_cp_32x128b_warpx4(sf_tmem + 8 + kt * 8 + nb * 4,
-                                      make_smem_desc(smem_u32(&sm.sfb[s][nb * 1024 + kt * 512]), 16, 128, 0));
-    }
-}
-
 __global__ void __launch_bounds__(kGThreads, 1)
 gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                  const GemmParams p)
@@ -118,12 +110,13 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         for (int s = 0; s < kGStages; ++s) {
             mbar_init(&sm.full[s], 1);
             mbar_init(&sm.empty[s], 1);
+            mbar_init(&sm.sf_ready[s], 4);
         }
         mbar_init(&sm.tmem_full, 1);
         mbar_init(&sm.tmem_empty, kGEpiWarps);
         fence_barrier_init();
     }
-    if (warp == 1) {
+    if (warp == kGMmaWarp) {
         tmem_alloc(&sm.tmem_base, kGTmemCols);
         tmem_relinquish();
     }
@@ -132,8 +125,11 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     tcgen05_fence_after();
     const uint32_t tmem = sm.tmem_base;
 
-    if (warp == 0) {
+    // register budget per role (whole warpgroups): 4*32*(56 + 2*192 + 56) = 63488 <= 65536;
+    // every warp of a warpgroup executes the same setmaxnreg at the top of its role
+    if (warp == kGProducerWarp) {
         // ------------------------------------------------------------ TMA producer
+        setmaxnreg_dec<56>();
         if (lane == 0) {
             tma_prefetch_desc(&tm_a);
             tma_prefetch_desc(&tm_b);
@@ -165,40 +161,26 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == kGMmaWarp) {
         // ------------------------------------------------------------ MMA issuer
+        setmaxnreg_dec<56>();
         if (lane == 0) {
-            const int total_it = my_tiles * p.k_stages;
-            bool alive = total_it > 0;
-            // scales of the very first stage; afterwards each iteration copies the next one's
-            if (alive) {
-                alive = mbar_wait(&sm.full[0], 0, &sm.abort_flag);
-                if (alive) {
-                    tcgen05_fence_after();
-                    copy_scales_to_tmem(sm, 0, tmem + kGTmemSfBase, (min(kGBlockK, p.K) + 127) / 128);
-                }
-            }
             int it = 0;
+            bool alive = true;
             for (int tile_it = 0; alive && tile_it < my_tiles; ++tile_it) {
                 if (tile_it > 0 && !mbar_wait(&sm.tmem_empty, (tile_it - 1) & 1, &sm.abort_flag)) break;
                 tcgen05_fence_after();
                 for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
                     const int s = it % kGStages;
-                    const uint32_t sf_tmem = tmem + kGTmemSfBase + (it & 1) * kGTmemSfPerBuf;
-                    if (it + 1 < total_it) {
-                        // next stage's scales go to the other TMEM scale buffer while this
-                        // stage's MMAs run
-                        const int s1 = (it + 1) % kGStages;
-                        if (!mbar_wait(&sm.full[s1], ((it + 1) / kGStages) & 1, &sm.abort_flag)) {
-                            alive = false;
-                            break;
-                        }
-                        tcgen05_fence_after();
-                        const int ks1 = (ks + 1 == p.k_stages) ? 0 : ks + 1;
-                        const int vk1 = min(kGBlockK, p.K - ks1 * kGBlockK);
-                        copy_scales_to_tmem(sm, s1, tmem + kGTmemSfBase + ((it + 1) & 1) * kGTmemSfPerBuf,
-                                            (vk1 + 127) / 128);
+                    const uint32_t parity = (it / kGStages) & 1;
+                    // codes landed in shared memory, scales landed in this stage's TMEM columns
+                    if (!mbar_wait(&sm.full[s], parity, &sm.abort_flag) ||
+                        !mbar_wait(&sm.sf_ready[s], parity, &sm.abort_flag)) {
+                        alive = false;
+                        break;
                     }
+                    tcgen05_fence_after();
+                    const uint32_t sf_tmem = tmem + kGTmemSfBase + s * kGTmemSfPerBuf;
                     const int valid_k = min(kGBlockK, p.K - ks * kGBlockK);
                     const int nmma = (valid_k + 63) / 64;
                     const uint64_t a_desc = make_smem_desc(smem_u32(sm.a[s]), 16, 1024, 2);
@@ -209,14 +191,44 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                                          make_idesc_mxf4(sf_id, sf_id), sf_tmem + (j >> 1) * 4,
                                          sf_tmem + 8 + (j >> 1) * 8, (ks > 0 || j > 0) ? 1u : 0u);
                     }
-                    tcgen05_commit(&sm.empty[s]);   // stage reusable once these MMAs have read it
+                    // frees the shared-memory stage and its TMEM scale columns together
+                    tcgen05_commit(&sm.empty[s]);
                 }
                 if (alive) tcgen05_commit(&sm.tmem_full);
             }
         }
-    } else {
+    } else if (warp < 4) {
+        // ------------------------------------------------------------ scale warps
+        // Lane r of every quadrant must hold, per 128-row x 4-block scale tile, the 16 bytes at
+        // offset 16*r of that tile: four 32-bit columns = rows r, r+32, r+64, r+96.  Stage s
+        // owns TMEM columns [s*24, s*24+24): SFA K-tiles 0,1 | SFB K-tile 0 (row blocks 0,1) |
+        // SFB K-tile 1.  The columns are free again once the producer has seen empty[s], which
+        // happens before full[s] can complete, so waiting on full[s] is enough.
+        setmaxnreg_dec<56>();
+        const int total_it = my_tiles * p.k_stages;
+        const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+        for (int it = 0; it < total_it; ++it) {
+            const int s = it % kGStages;
+            if (!mbar_wait(&sm.full[s], (it / kGStages) & 1, &sm.abort_flag)) break;
+            const uint4 a0 = *reinterpret_cast<const uint4*>(&sm.sfa[s][lane * 16]);
+            const uint4 a1 = *reinterpret_cast<const uint4*>(&sm.sfa[s][512 + lane * 16]);
+            const uint4 b00 = *reinterpret_cast<const uint4*>(&sm.sfb[s][lane * 16]);
+            const uint4 b01 = *reinterpret_cast<const uint4*>(&sm.sfb[s][1024 + lane * 16]);
+            const uint4 b10 = *reinterpret_cast<const uint4*>(&sm.sfb[s][512 + lane * 16]);
+            const uint4 b11 = *reinterpret_cast<const uint4*>(&sm.sfb[s][1536 + lane * 16]);
+            const uint32_t t = tmem + lane_base + kGTmemSfBase + s * kGTmemSfPerBuf;
+            tmem_st_32x32b_x8(t, a0, a1);
+            tmem_st_32x32b_x8(t + 8, b00, b01);
+            tmem_st_32x32b_x8(t + 16, b10, b11);
+            tmem_st_wait();
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.sf_ready[s]);
+        }
+    } else if (warp < 12) {
         // ------------------------------------------------------------ epilogue warps
-        const int ew = warp - 2;
+        setmaxnreg_inc<192>();
+        const int ew = warp - 4;
         const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
         const int half = ew >> 2;                  // which 128 accumulator columns
         uint8_t* stg = sm.out_stage[ew];
@@ -302,9 +314,13 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         }
     }
 
+    else {
+        setmaxnreg_dec<56>();   // idle warps of the producer/MMA warpgroup
+    }
+
     tcgen05_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kGMmaWarp) {
         tcgen05_fence_after();
         tmem_dealloc(tmem, kGTmemCols);
     }
