@@ -37,7 +37,8 @@ _lib = None
 
 
 def library_path() -> str:
-    return _build.LIB_PATH
+    """Path of the shared library; ``MXFP4_LIBRARY`` overrides the in-tree build."""
+    return os.environ.get("MXFP4_LIBRARY") or _build.LIB_PATH
 
 
 def load_library() -> ctypes.CDLL:

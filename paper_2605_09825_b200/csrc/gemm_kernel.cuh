@@ -25,6 +25,10 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#ifdef MXFP4_PROBE
+#include <stdlib.h>
+#include <stdio.h>
+#endif
 
 #include "../../include/mxfp4.h"
 #include "ptx_sm100.cuh"
@@ -75,6 +79,10 @@ struct GemmParams {
     int32_t sf_rows_b;      // ceil(N / 128)
     float alpha;
     int32_t out_fp32;
+#ifdef MXFP4_PROBE
+    int32_t debug;
+    long long* probe_out;
+#endif
 };
 
 // Instruction descriptor of tcgen05.mma kind::mxf4.block_scale: E2M1 x E2M1, E8M0 scales,
@@ -124,6 +132,10 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem = sm.tmem_base;
+#ifdef MXFP4_PROBE
+    long long pc0 = 0; unsigned long long pg0 = 0;
+    if (threadIdx.x == 0 && blockIdx.x == 0) { pc0 = clock64(); asm volatile("mov.u64 %0, %globaltimer;" : "=l"(pg0)); }
+#endif
 
     // register budget per role (whole warpgroups): 4*32*(56 + 2*192 + 56) = 63488 <= 65536;
     // every warp of a warpgroup executes the same setmaxnreg at the top of its role
@@ -168,6 +180,9 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             int it = 0;
             bool alive = true;
             for (int tile_it = 0; alive && tile_it < my_tiles; ++tile_it) {
+#ifdef MXFP4_PROBE
+                if (!(p.debug & 1))
+#endif
                 if (tile_it > 0 && !mbar_wait(&sm.tmem_empty, (tile_it - 1) & 1, &sm.abort_flag)) break;
                 tcgen05_fence_after();
                 for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
@@ -175,7 +190,11 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                     const uint32_t parity = (it / kGStages) & 1;
                     // codes landed in shared memory, scales landed in this stage's TMEM columns
                     if (!mbar_wait(&sm.full[s], parity, &sm.abort_flag) ||
+#ifdef MXFP4_PROBE
+                        (!(p.debug & 2) && !mbar_wait(&sm.sf_ready[s], parity, &sm.abort_flag))) {
+#else
                         !mbar_wait(&sm.sf_ready[s], parity, &sm.abort_flag)) {
+#endif
                         alive = false;
                         break;
                     }
@@ -320,6 +339,9 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 
     tcgen05_fence_before();
     __syncthreads();
+#ifdef MXFP4_PROBE
+    if (threadIdx.x == 0 && blockIdx.x == 0) { unsigned long long g1; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g1)); p.probe_out[0] = clock64() - pc0; p.probe_out[1] = (long long)(g1 - pg0); }
+#endif
     if (warp == kGMmaWarp) {
         tcgen05_fence_after();
         tmem_dealloc(tmem, kGTmemCols);
@@ -352,6 +374,9 @@ static int launch_gemm(const void* a_codes, const void* a_scales, const void* b_
     p.sf_rows_b = static_cast<int32_t>((N + 127) / 128);
     p.alpha = alpha;
     p.out_fp32 = out_dtype == MXFP4_OUT_FP32;
+#ifdef MXFP4_PROBE
+    { const char* e = getenv("MXFP4_GEMM_DEBUG"); p.debug = e ? atoi(e) : 0; static long long* buf = nullptr; if (!buf) cudaMalloc(&buf, 64); p.probe_out = buf; }
+#endif
     const int64_t total = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
     if (total > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
     const size_t smem = sizeof(GemmSmem) + 1024;
@@ -364,6 +389,9 @@ static int launch_gemm(const void* a_codes, const void* a_scales, const void* b_
     }
     const int grid = static_cast<int>(total < sm_count ? total : sm_count);
     gemm_mxf4_kernel<<<grid, kGThreads, smem, stream>>>(tm_a, tm_b, p);
+#ifdef MXFP4_PROBE
+    if (getenv("MXFP4_GEMM_CLOCK")) { long long h[2]; cudaStreamSynchronize(stream); cudaMemcpy(h, p.probe_out, 16, cudaMemcpyDeviceToHost); fprintf(stderr, "probe: %lld cycles in %lld ns -> %.0f MHz\n", h[0], h[1], h[0] * 1e3 / h[1]); }
+#endif
     return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
