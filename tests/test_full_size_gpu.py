@@ -1,0 +1,70 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times (fused
+passes, bf16 outputs, deterministic H32 + RNE and the config-4 variants): quantized operands
+bit-exact against the oracle on whole tensors, GEMM outputs on sampled rows the oracle computes
+one by one (first and last 128-row tile edges plus seeded random rows, all columns)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import assert_gemm_close, to_dev
+from paper_2605_09825_b200 import api, synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _rows(M, seed, n_random=24):
+    rng = np.random.default_rng(seed)
+    fixed = [0, 1, 31, 32, 127, 128, M - 129, M - 128, M - 1]
+    return np.unique(np.concatenate([np.array(fixed), rng.integers(0, M, n_random)])).astype(np.int64)
+
+
+def _check_pass(pass_, a_bits, b_bits, hmode, rnd, seed, what):
+    a, b = to_dev(a_bits), to_dev(b_bits)
+    fn = (api.linear_fprop, api.linear_dgrad, api.linear_wgrad)[pass_]
+    ofn = (oracle.linear_fprop, oracle.linear_dgrad, oracle.linear_wgrad)[pass_]
+    out = fn(a, b, hmode, rnd, seed, api.OUT_BF16)
+    api.check()
+    M = out.shape[0]
+    rows = _rows(M, 1234 + pass_)
+    ref, S = ofn(a_bits, b_bits, hmode, rnd, seed, rows=rows)
+    got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy()
+    assert_gemm_close(got, ref, S, True, what)
+    del out
+
+
+def _check_quant(bits, axis, hmode, rnd, seed, tag):
+    codes, scales = api.quantize(to_dev(bits), axis, hmode, rnd, seed, tag)
+    api.check()
+    wc, ws = oracle.quantize(bits, axis, hmode, rnd, seed, tag)
+    outer, K = wc.shape[0], wc.shape[1] * 2
+    assert (codes.cpu().numpy() == wc).all()
+    assert (oracle.scales_from_tiled(scales.cpu().numpy(), outer, K // 32) == ws).all()
+
+
+def test_config2_qkv_fprop():
+    t = synth.config2()
+    _check_pass(0, t["X"], t["W"], 1, 0, 0, "config 2 fprop")
+
+
+def test_config3_gate_up_fprop_and_dgrad():
+    t = synth.config3()
+    _check_pass(0, t["X"], t["W"], 1, 0, 0, "config 3 fprop")
+    _check_pass(1, t["dY"], t["W"], 1, 0, 0, "config 3 dgrad")
+    _check_quant(t["dY"], 1, 1, 0, 0, 0)        # the largest operand of the path, row-wise
+    _check_quant(t["W"], 0, 1, 0, 0, 1)         # W^T for Dgrad, column-wise
+
+
+@pytest.mark.parametrize("hmode,rnd", [(1, 0), (2, 0), (0, 1)])
+def test_config4_down_wgrad_variants(hmode, rnd):
+    t = synth.config4()
+    _check_pass(2, t["dY"], t["X"], hmode, rnd, 7, f"config 4 wgrad mode {hmode} rounding {rnd}")
+    _check_quant(t["X"], 0, hmode, rnd, 7, 1)   # X^T [14336 x 8192], column-wise, whole tensor
+
+
+@pytest.mark.parametrize("name", ["qkv", "o", "gate_up", "down"])
+def test_config5_layer_stack_16384_tokens(name):
+    t = synth.linear_tensors(name, 16384, 5)
+    _check_pass(0, t["X"], t["W"], 1, 0, 0, f"config 5 {name} fprop")
+    _check_pass(1, t["dY"], t["W"], 1, 0, 0, f"config 5 {name} dgrad")
+    _check_pass(2, t["dY"], t["X"], 1, 0, 0, f"config 5 {name} wgrad")
