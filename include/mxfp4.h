@@ -41,6 +41,7 @@ extern "C" {
 #define MXFP4_ERR_CUDA (-6)      /* a CUDA runtime/driver call failed (launch, descriptor)    */
 #define MXFP4_ERR_TIMEOUT (-7)   /* a bounded device-side wait expired (reported by check)    */
 #define MXFP4_ERR_DEVICE (-8)    /* not an sm_100 device                                      */
+#define MXFP4_ERR_STATIC_LIMIT (-9) /* mxfp4_linear_static: problem exceeds the built-in scratch */
 
 /* enums (plain ints in the ABI) */
 #define MXFP4_AXIS_ROWS 0 /* 32-blocks run down the rows (column-wise 32x1); operand = src^T */
@@ -161,6 +162,38 @@ int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* ou
                       int64_t in_features, int64_t out_features, int hadamard_mode, int rounding,
                       uint64_t seed, int out_dtype, void* dev_a, void* dev_b, void* dev_out,
                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * mxfp4_linear_static -- the fused passes for callers that cannot allocate device memory.
+ * (The paper has no counterpart to this entry point; it exists for integration only.)
+ *
+ * Who needs it: code that runs where neither cudaMalloc nor the host framework's allocator may
+ * be called -- for example a callback inside a runtime that has handed all device memory to
+ * its own arena (cudaMalloc would fail or fragment it), a latency-critical serving loop that
+ * cannot afford cudaMalloc's implicit device synchronisation, or a plugin that is given
+ * input/output buffers but no allocator handle.  Such callers still pass the inputs and the
+ * output; only the scratch for the two quantized operands comes from the library.
+ *
+ * How: the scratch is a fixed array of MXFP4_STATIC_SCRATCH_BYTES that is part of the library
+ * image, so every GPU that loads the library holds that much memory until the process exits.
+ * The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ *
+ *   pass, (a, b, out), T, in_features, out_features, hadamard_mode, rounding, seed, out_dtype:
+ *       exactly as mxfp4_linear_fprop / _dgrad / _wgrad (pass = MXFP4_PASS_*), same results.
+ *   Limit: mxfp4_linear_workspace_bytes(T, in, out, pass) must not exceed
+ *       MXFP4_STATIC_SCRATCH_BYTES; larger problems return MXFP4_ERR_STATIC_LIMIT and nothing
+ *       is enqueued (use the workspace-taking entry points for those).
+ *   First call on a device: looks up the array's device address (once per device, with that
+ *       device current).  Make that first call before any stream capture begins.
+ *   Sharing: every call on a device uses the same array and finds the previous call's
+ *       contents in it.  Nothing needs clearing -- each call rewrites all bytes it later reads --
+ *       but two calls that overlap on the GPU (different streams, or concurrent host threads
+ *       without ordering) race on the array.  Issue them on one stream or order them with events.
+ */
+#define MXFP4_STATIC_SCRATCH_BYTES (16 * 1024 * 1024)
+int mxfp4_linear_static(int pass, const void* a, const void* b, void* out, int64_t T,
+                        int64_t in_features, int64_t out_features, int hadamard_mode, int rounding,
+                        uint64_t seed, int out_dtype, void* stream);
 
 /*
  * Synchronises `stream` and returns the sticky device-side status of the current device:

@@ -23,8 +23,10 @@ AXIS_ROWS, AXIS_COLS = 0, 1
 EXPORTS = (
     "mxfp4_version", "mxfp4_status_string", "mxfp4_codes_bytes", "mxfp4_scales_bytes",
     "mxfp4_quantize", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
-    "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_host", "mxfp4_check",
+    "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_host", "mxfp4_linear_static",
+    "mxfp4_check",
 )
+STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
 
 class Mxfp4Error(RuntimeError):
@@ -71,6 +73,8 @@ def load_library() -> ctypes.CDLL:
     lib.mxfp4_linear_host.argtypes = [ci, vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, vp, vp, vp,
                                       sz, vp]
     lib.mxfp4_linear_host.restype = ci
+    lib.mxfp4_linear_static.argtypes = [ci, vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp]
+    lib.mxfp4_linear_static.restype = ci
     lib.mxfp4_check.argtypes, lib.mxfp4_check.restype = [vp], ci
     _lib = lib
     return lib
@@ -215,6 +219,31 @@ def linear_host(pass_: int, a_host: torch.Tensor, b_host: torch.Tensor, out_host
         _dev_ptr(dev_out), _dev_ptr(workspace), workspace.numel(), _stream())
     _raise(rc, "mxfp4_linear_host")
     return out_host
+
+
+def linear_static(pass_: int, a: torch.Tensor, b: torch.Tensor, T: int, in_f: int, out_f: int,
+                  hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0, out_dtype=OUT_BF16,
+                  out: torch.Tensor | None = None):
+    """``mxfp4_linear_static``: a fused pass whose scratch is the library's built-in array.
+
+    For callers that may not allocate device memory: the caller provides inputs and (here,
+    optionally) the output; the library allocates nothing.  Problems whose scratch need exceeds
+    ``STATIC_SCRATCH_BYTES`` are rejected with status -9.  Calls share one array per device, so
+    overlapping calls on different streams race; the first call on a device should come before
+    any stream capture.
+    """
+    for t in (a, b):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise ValueError("inputs must be contiguous bf16 tensors")
+    shape = {PASS_FPROP: (T, out_f), PASS_DGRAD: (T, in_f), PASS_WGRAD: (out_f, in_f)}[pass_]
+    if out is None:
+        out = torch.empty(shape, dtype=torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32,
+                          device=a.device)
+    rc = load_library().mxfp4_linear_static(pass_, _dev_ptr(a), _dev_ptr(b), _dev_ptr(out), T, in_f, out_f,
+                                            hadamard_mode, rounding, ctypes.c_uint64(seed), out_dtype,
+                                            _stream())
+    _raise(rc, "mxfp4_linear_static")
+    return out
 
 
 def check() -> None:

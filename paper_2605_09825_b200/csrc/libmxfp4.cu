@@ -110,6 +110,7 @@ const char* mxfp4_status_string(int status)
         case MXFP4_ERR_CUDA: return "CUDA call failed";
         case MXFP4_ERR_TIMEOUT: return "device-side wait timed out";
         case MXFP4_ERR_DEVICE: return "not an sm_100 device";
+        case MXFP4_ERR_STATIC_LIMIT: return "problem needs more scratch than the built-in array holds";
         default: return "unknown status";
     }
 }
@@ -313,6 +314,49 @@ int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* ou
     if (cudaMemcpyAsync(out_host, dev_out, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return MXFP4_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free variant of the fused passes.  The scratch the passes need (the two quantized
+// operands) lives in this file-scope device array instead of a caller-supplied workspace.  In
+// host code the array's name is only a stand-in for the symbol, not a device address, so the
+// address is fetched once per device with cudaGetSymbolAddress and cached.
+static __device__ __align__(256) uint8_t g_static_scratch[MXFP4_STATIC_SCRATCH_BYTES];
+
+static int static_scratch_address(uint8_t** out)
+{
+    static uint8_t* cached[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
+    if (!cached[dev]) {
+        uint8_t* ptr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess || !ptr)
+            return MXFP4_ERR_CUDA;
+        cached[dev] = ptr;
+    }
+    *out = cached[dev];
+    return MXFP4_OK;
+}
+
+int mxfp4_linear_static(int pass, const void* a, const void* b, void* out, int64_t T,
+                        int64_t in_features, int64_t out_features, int hadamard_mode, int rounding,
+                        uint64_t seed, int out_dtype, void* stream)
+{
+    if (pass < 0 || pass > 2) return MXFP4_ERR_ENUM;
+    if (T <= 0 || in_features <= 0 || out_features <= 0) return MXFP4_ERR_SHAPE;
+    int64_t M, N, K;
+    linear_dims(pass, T, in_features, out_features, &M, &N, &K);
+    if (K % 32 != 0) return MXFP4_ERR_SHAPE;
+    const size_t need = mxfp4_linear_workspace_bytes(T, in_features, out_features, pass);
+    if (need == 0) return MXFP4_ERR_SHAPE;
+    if (need > static_cast<size_t>(MXFP4_STATIC_SCRATCH_BYTES)) return MXFP4_ERR_STATIC_LIMIT;
+    uint8_t* scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != MXFP4_OK) return rc;
+    // Nothing in the scratch has to start at zero: the two quantize launches of this call
+    // rewrite every code byte and every scale tile (padding included) the GEMM will read.
+    return linear_pass(pass, a, b, out, T, in_features, out_features, hadamard_mode, rounding, seed,
+                       out_dtype, scratch, MXFP4_STATIC_SCRATCH_BYTES, stream);
 }
 
 int mxfp4_check(void* stream)
