@@ -4,7 +4,8 @@
 // Work unit: a tile of 128 operand rows x 128 elements along K (4 MX blocks).  A producer warp
 // streams source tiles into a ring of shared-memory stages with TMA; 512 consumer threads each
 // own one 32-element block per tile: the whole block sits in the thread's registers, so the
-// five butterfly stages, the block maximum and the rounding need no cross-lane traffic.
+// five butterfly stages (as packed fp32x2 operations), the block maximum and the rounding
+// need no cross-lane traffic.
 // Results leave through shared memory: packed codes as a 128 x 64-byte tile written by a TMA
 // store (which also clips ragged edges), scales as one contiguous 512-byte tile.
 //
@@ -50,33 +51,84 @@ struct QuantParams {
     int32_t scale_layout;    // 0 canonical, 1 tiled
 };
 
-// In-register 32-point Walsh-Hadamard transform, stages h = 1, 2, 4, 8, 16; every output is
-// one fp32 add or subtract (no FMA contraction can occur: there are no multiplies).
-__device__ __forceinline__ void fwht32(float (&v)[32])
+// Packed fp32 pairs: sm_100 adds, subtracts and multiplies two independent fp32 values held in
+// one 64-bit register with a single instruction (each lane is an ordinary IEEE fp32
+// round-to-nearest operation, so results are bit-identical to the scalar form).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+
+__device__ __forceinline__ void unpack2(uint64_t p, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// max(|a|, |b|, |c|) in one instruction.
+__device__ __forceinline__ float max3_abs(float a, float b, float c)
+{
+    float r;
+    asm("max.abs.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// In-register 32-point Walsh-Hadamard transform of v[0..31] held as 16 pairs
+// P[i] = (v[2i], v[2i+1]).  Stage h = 1 was applied by the caller while forming the pairs
+// (its partners share a pair); stages h = 2, 4, 8, 16 pair whole registers, so each packed
+// add/sub does two butterflies.  Same five stages, same order, one fp32 rounding per output.
+__device__ __forceinline__ void fwht32_stages_2_to_16(uint64_t (&P)[16])
 {
 #pragma unroll
-    for (int h = 1; h < 32; h <<= 1) {
+    for (int hp = 1; hp < 16; hp <<= 1) {
 #pragma unroll
-        for (int i = 0; i < 32; i += 2 * h) {
+        for (int i = 0; i < 16; i += 2 * hp) {
 #pragma unroll
-            for (int j = i; j < i + h; ++j) {
-                const float a = v[j], b = v[j + h];
-                v[j] = __fadd_rn(a, b);
-                v[j + h] = __fsub_rn(a, b);
+            for (int j = i; j < i + hp; ++j) {
+                const uint64_t a = P[j], b = P[j + hp];
+                P[j] = add2(a, b);
+                P[j + hp] = sub2(a, b);
             }
         }
     }
 }
 
-// Two E2M1 codes from two floats, round-to-nearest-even, saturating: `lo` lands in bits 3:0.
-__device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
+// Eight E2M1 codes (one 32-bit word of packed output) from eight floats, round-to-nearest-even,
+// saturating; v0 lands in bits 3:0, v7 in bits 31:28.
+__device__ __forceinline__ uint32_t cvt_e2m1x8(float v0, float v1, float v2, float v3, float v4,
+                                               float v5, float v6, float v7)
 {
-    uint16_t r;
-    asm("{\n\t.reg .b8 t;\n\t"
-        "cvt.rn.satfinite.e2m1x2.f32 t, %1, %2;\n\t"
-        "cvt.u16.u8 %0, t;\n\t}"
-        : "=h"(r)
-        : "f"(hi), "f"(lo));
+    uint32_t r;
+    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
+        "mov.b32 %0, {b0, b1, b2, b3};\n\t}"
+        : "=r"(r)
+        : "f"(v0), "f"(v1), "f"(v2), "f"(v3), "f"(v4), "f"(v5), "f"(v6), "f"(v7));
     return r;
 }
 
@@ -155,7 +207,17 @@ quantize_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constan
 
         const bool ok = mbar_wait(&sm.full[s], round & 1, &sm.abort_flag);
 
-        float v[32];
+        // the block as 16 packed pairs P[i] = (v[2i], v[2i+1]); the sign diagonal and the first
+        // butterfly stage (whose partners are the two halves of a pair) are applied on the way in
+        uint64_t P[16];
+        auto make_pair = [&](int i, uint32_t lo_bits, uint32_t hi_bits) {
+            if (HMODE == 2) {
+                lo_bits ^= (p.sign_mask << (31 - 2 * i)) & 0x80000000u;
+                hi_bits ^= (p.sign_mask << (30 - 2 * i)) & 0x80000000u;
+            }
+            const float a = __uint_as_float(lo_bits), b = __uint_as_float(hi_bits);
+            P[i] = HMODE != 0 ? pack2(__fadd_rn(a, b), __fsub_rn(a, b)) : pack2(a, b);
+        };
         if (ok) {
             if (AXIS == 1) {
                 const uint8_t* base = &sm.stage[s][(kb >> 1) * (kQStageBytes / 2) + o * 128];
@@ -165,53 +227,49 @@ quantize_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constan
                     const uint4 q = *reinterpret_cast<const uint4*>(base + chunk);
                     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        v[8 * j + 2 * i] = __uint_as_float(w[i] << 16);
-                        v[8 * j + 2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-                    }
+                    for (int i = 0; i < 4; ++i) make_pair(4 * j + i, w[i] * 65536u, w[i] & 0xFFFF0000u);
                 }
             } else {
                 const uint16_t* base =
                     reinterpret_cast<const uint16_t*>(&sm.stage[s][0]) + (kb * 32) * 128 + o;
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    v[j] = __uint_as_float(static_cast<uint32_t>(base[j * 128]) << 16);
+                for (int i = 0; i < 16; ++i)
+                    make_pair(i, static_cast<uint32_t>(base[(2 * i) * 128]) * 65536u,
+                              static_cast<uint32_t>(base[(2 * i + 1) * 128]) * 65536u);
             }
         } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = 0.0f;
+            for (int i = 0; i < 16; ++i) P[i] = 0ull;
         }
         // the stage is in registers now: hand it back to the producer
         __syncwarp();
         if ((tid & 31) == 0) mbar_arrive(&sm.empty[s]);
 
-        if (HMODE == 2) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                v[j] = __uint_as_float(__float_as_uint(v[j]) ^ ((p.sign_mask << (31 - j)) & 0x80000000u));
-        }
-        if (HMODE != 0) fwht32(v);
+        if (HMODE != 0) fwht32_stages_2_to_16(P);
 
-        float amax = 0.0f;
+        float v[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) amax = fmaxf(amax, fabsf(v[j]));
+        for (int i = 0; i < 16; ++i) unpack2(P[i], v[2 * i], v[2 * i + 1]);
+        float amax = max3_abs(v[0], v[1], v[2]);
+#pragma unroll
+        for (int j = 3; j < 31; j += 2) amax = max3_abs(amax, v[j], v[j + 1]);
+        amax = fmaxf(amax, fabsf(v[31]));
         const uint32_t E = __float_as_uint(amax) >> 23;
         const uint32_t byte = E > 2u ? E - 2u : 0u;   // E <= 255 keeps byte <= 253 < 255
         const float mult = __uint_as_float((254u - byte) << 23);
+        const uint64_t mult2 = pack2(mult, mult);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint64_t sp = mul2(P[i], mult2);
+            unpack2(sp, v[2 * i], v[2 * i + 1]);       // v now holds the scaled values
+        }
 
         uint32_t packed[4];
         if (SR == 0) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t w = 0;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float lo = __fmul_rn(v[8 * q + 2 * i], mult);
-                    const float hi = __fmul_rn(v[8 * q + 2 * i + 1], mult);
-                    w |= cvt_e2m1x2(lo, hi) << (8 * i);
-                }
-                packed[q] = w;
-            }
+            for (int q = 0; q < 4; ++q)
+                packed[q] = cvt_e2m1x8(v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4],
+                                       v[8 * q + 5], v[8 * q + 6], v[8 * q + 7]);
         } else {
             const uint64_t e0 = static_cast<uint64_t>(to * kQTileO + o) * static_cast<uint64_t>(p.K) +
                                 static_cast<uint64_t>((tk * 4 + kb) * 32);
@@ -230,7 +288,7 @@ quantize_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constan
                         const int j = half * 16 + q * 8 + i;       // element in the block
                         const int e = q * 8 + i;                   // element in the 16-group
                         const uint32_t u8 = (r[e >> 2] >> (8 * (e & 3))) & 0xFFu;
-                        w |= sr_e2m1(__fmul_rn(v[j], mult), u8) << (4 * i);
+                        w |= sr_e2m1(v[j], u8) << (4 * i);
                     }
                     packed[half * 2 + q] = w;
                 }
