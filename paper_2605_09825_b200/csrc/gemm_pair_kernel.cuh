@@ -1,31 +1,40 @@
-// Block-scaled MXFP4 GEMM, CTA-pair version (tcgen05 cta_group::2): two CTAs of a cluster share
-// one 256 x 256 output tile.  Each CTA loads its own 128 rows of A and its own 128 rows of B per
-// K-step (32 KB instead of the 48 KB a lone 128 x 256 tile needs), which is what matters once the
-// L2 -> shared-memory operand feed, not the tensor pipe, bounds the kernel.  No TMA multicast is
-// used: every CTA fetches its own operands; only barrier signals cross the pair.
+// Block-scaled MXFP4 GEMM on the 5th-generation tensor cores (the MXFP4 GEMM that replaces the
+// linear layers' FP8 GEMM; operand orientation per Appendix C):
 //
 //   out[m][n] = alpha * sum_t 2^(sa[m][t]-127) 2^(sb[n][t]-127) sum_{k in block t} A[m][k] B[n][k]
 //
-// Roles per CTA (512 threads, four warpgroups; same split as the single-CTA kernel):
-//   warps 0..3   scale warps: shared memory -> this CTA's TMEM scale columns (tcgen05.st)
-//   warps 4..11  epilogue: this CTA's 128 rows x 256 columns of the accumulator
-//   warp 12      TMA producer: A half, B half (completion counted on the LEADER's barrier),
-//                scale tiles (local barrier)
-//   warp 13      MMA issuer -- only in the leader CTA (cluster rank 0); its commits arrive on
-//                the barriers of both CTAs
-// Barrier ownership: full / sf_ready / tmem_empty are consumed by the leader's MMA thread, so
-// the peer's producers, scale warps and epilogue warps arrive on the leader's copies; empty and
-// tmem_full are signalled in both CTAs by a multicast tcgen05.commit; sf_full is local.
+// CTA-pair kernel (tcgen05 cta_group::2): the two CTAs of a cluster share one 256 x 256 output
+// tile.  Each CTA loads its own 128 rows of A and its own 128 rows of B (64 KB per K-step of 512
+// elements, against the 96 KB a lone 128 x 256 tile would need), because the L2 -> shared-memory
+// operand feed, not the tensor pipe, is what bounds an FP4 GEMM here.  No TMA multicast is used:
+// every CTA fetches its own operands; only barrier signals cross the pair.
+//
+// Roles per CTA (512 threads, four warpgroups; registers rebalanced with setmaxnreg):
+//   warps 0..3   scale warps (one per TMEM lane quadrant): shared memory -> this CTA's TMEM scale
+//                columns with tcgen05.st.  (tcgen05.cp would do the same copy, but measured here
+//                each one holds the tensor pipe for 70-85 cycles whatever its shape, and a
+//                K-step needs twelve of them against 1024 cycles of MMA.)
+//   warps 4..11  epilogue: this CTA's 128 rows x 256 columns of the accumulator; four
+//                back-to-back tcgen05.ld per warp, accumulator handed back at once, then
+//                alpha, conversion and stores overlap the next tile's main loop.
+//   warp 12      TMA producer: A and B halves (completion counted on the LEADER's barrier) and
+//                the scale tiles (local barrier), 3-stage ring.
+//   warp 13      MMA issuer, leader CTA (cluster rank 0) only: eight
+//                tcgen05.mma.cta_group::2.kind::mxf4.block_scale (256 x 256 x 64) per stage; its
+//                commits arrive on the barriers of both CTAs.
+// The issuing warps run their loops in warp-uniform control flow and issue through
+// elect.sync, so descriptors stay in uniform registers; the MMA warp tests the next stage's
+// barriers before it issues the current stage's MMAs, which hides the barrier round trip.
+// Barrier ownership: full / sf_ready / tmem_empty are consumed by the leader's MMA warp, so the
+// peer's producer, scale warps and epilogue warps arrive on the leader's copies (relaxed: they
+// publish no ordinary memory writes); empty and tmem_full are signalled in both CTAs by a
+// multicast tcgen05.commit; sf_full is local.  All waits are bounded (see ptx_sm100.cuh).
 #pragma once
 
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
-#ifdef MXFP4_PROBE
-#include <stdio.h>
-#include <stdlib.h>
-#endif
 
 #include "../../include/mxfp4.h"
 #include "ptx_sm100.cuh"
@@ -37,26 +46,25 @@ constexpr int kPHalfM = 128;                     // rows of A (and of the accumu
 constexpr int kPHalfN = 128;                     // rows of B per CTA
 constexpr int kPTileM = 256;
 constexpr int kPTileN = 256;
-constexpr int kPBlockK = 256;                    // elements per stage = 128 bytes of codes
-constexpr int kPStages = 5;
-constexpr int kPABytes = kPHalfM * 128;          // 16 KB
-constexpr int kPBBytes = kPHalfN * 128;          // 16 KB
-constexpr int kPSfaBytes = 2 * 512;              // own 128 rows x 2 K-tiles
-constexpr int kPSfbBytes = 2 * 2 * 512;          // both 128-row blocks of B x 2 K-tiles
+constexpr int kPBlockK = 512;                    // elements per stage: two 128-byte swizzled boxes
+constexpr int kPStages = 3;
+constexpr int kPBoxBytes = 128 * 128;            // 128 rows x 128 bytes of codes = 16 KB
+constexpr int kPSfaBytes = 4 * 512;              // own 128 rows x 4 K-tiles of 128 elements
+constexpr int kPSfbBytes = 2 * 4 * 512;          // both 128-row blocks of B x 4 K-tiles
 constexpr int kPEpiWarps = 8;
 constexpr int kPProducerWarp = 12;
 constexpr int kPMmaWarp = 13;
 constexpr int kPThreads = 512;
 constexpr uint32_t kPTmemCols = 512;
-constexpr uint32_t kPTmemSfBase = 256;
-constexpr uint32_t kPTmemSfPerBuf = 24;
+constexpr uint32_t kPTmemSfBase = 256;           // accumulator occupies columns 0..255
+constexpr uint32_t kPTmemSfPerBuf = 48;          // per stage: 16 columns SFA + 32 columns SFB
 
 struct GemmPairSmem {
-    alignas(1024) uint8_t a[kPStages][kPABytes];
-    alignas(1024) uint8_t b[kPStages][kPBBytes];
+    alignas(1024) uint8_t a[kPStages][2][kPBoxBytes];     // [stage][K half][128 rows x 128 B]
+    alignas(1024) uint8_t b[kPStages][2][kPBoxBytes];
     alignas(128) uint8_t sfa[kPStages][kPSfaBytes];
-    alignas(128) uint8_t sfb[kPStages][kPSfbBytes];
-    alignas(128) uint8_t out_stage[kPEpiWarps][32 * 64];
+    alignas(128) uint8_t sfb[kPStages][kPSfbBytes];       // [row block][K-tile][512]
+    alignas(128) uint8_t out_stage[kPEpiWarps][32 * 32];  // 32 rows x 16 bf16 per warp
     alignas(8) uint64_t full[kPStages];      // leader's copy is the live one
     uint64_t sf_full[kPStages];              // local
     uint64_t sf_ready[kPStages];             // leader's copy is the live one
@@ -74,29 +82,27 @@ struct GemmPairParams {
     int64_t ld_out;
     int32_t M, N, K;
     int32_t tiles_m, tiles_n;   // 256 x 256 pair tiles
-    int32_t k_stages;
+    int32_t k_stages;           // ceil(K / 512)
     int32_t sf_tiles_k;         // ceil(K / 128)
     int32_t sf_rows_a;          // ceil(M / 128)
     int32_t sf_rows_b;          // ceil(N / 128)
     float alpha;
     int32_t out_fp32;
-#ifdef MXFP4_PROBE
-    long long* probe_out;
-    int32_t debug;
-#endif
 };
 
-// Instruction descriptor for the pair MMA: M = 256 (128 per CTA), N = 256.
+// Instruction descriptor of the pair MMA: E2M1 x E2M1, E8M0 scales, both operands K-major,
+// M = 256 (128 per CTA), N = 256.  Scale-factor ids select which byte pair of the 32-bit TMEM
+// scale column an instruction uses.
 __device__ __forceinline__ uint32_t make_idesc_mxf4_pair(uint32_t a_sf_id, uint32_t b_sf_id)
 {
     uint32_t d = 0;
-    d |= b_sf_id << 4;
-    d |= 1u << 7;                      // A format E2M1
-    d |= 1u << 10;                     // B format E2M1
-    d |= (kPTileN >> 3) << 17;         // N / 8
-    d |= 1u << 23;                     // scale format E8M0
-    d |= (kPTileM >> 4) << 24;         // M / 16
-    d |= a_sf_id << 29;
+    d |= b_sf_id << 4;                 // bits 4..5   B scale-factor id
+    d |= 1u << 7;                      // bits 7..9   A format: E2M1
+    d |= 1u << 10;                     // bits 10..12 B format: E2M1
+    d |= (kPTileN >> 3) << 17;         // bits 17..22 N / 8
+    d |= 1u << 23;                     // bit 23      scale format: E8M0
+    d |= (kPTileM >> 4) << 24;         // bits 24..28 M / 16
+    d |= a_sf_id << 29;                // bits 29..30 A scale-factor id
     return d;
 }
 
@@ -138,38 +144,41 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
     tcgen05_fence_after();
     const uint32_t tmem = sm.tmem_base;
 
+    // register budget per role (whole warpgroups): 4*32*(56 + 2*192 + 56) = 63488 <= 65536;
+    // every warp of a warpgroup executes the same setmaxnreg at the top of its role
     if (warp == kPProducerWarp) {
         // ------------------------------------------------------------ TMA producer
         setmaxnreg_dec<56>();
-        {
-            // the whole warp walks the loop (uniform control flow keeps addresses and
-            // descriptors in uniform registers); one elected lane issues the copies
-            if (lane == 0) {
-                tma_prefetch_desc(&tm_a);
-                tma_prefetch_desc(&tm_b);
-            }
-            int it = 0;
-            bool alive = true;
-            for (int t = 0; alive && t < my_tiles; ++t) {
-                const int tile = cluster_id + t * n_clusters;
-                const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-                const int a_row_tile = tm * 2 + static_cast<int>(rank);     // 128-row scale tile of A
-                for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
-                    const int s = it % kPStages;
-                    const uint32_t round = it / kPStages;
-                    if (round > 0 && !mbar_wait(&sm.empty[s], (round - 1) & 1, &sm.abort_flag)) {
-                        alive = false;
-                        break;
-                    }
-                    if (elect_one_sync()) {
+        if (lane == 0) {
+            tma_prefetch_desc(&tm_a);
+            tma_prefetch_desc(&tm_b);
+        }
+        int it = 0;
+        bool alive = true;
+        for (int t = 0; alive && t < my_tiles; ++t) {
+            const int tile = cluster_id + t * n_clusters;
+            const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+            const int a_row_tile = tm * 2 + static_cast<int>(rank);     // 128-row scale tile of A
+            for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
+                const int s = it % kPStages;
+                const uint32_t round = it / kPStages;
+                if (round > 0 && !mbar_wait(&sm.empty[s], (round - 1) & 1, &sm.abort_flag)) {
+                    alive = false;
+                    break;
+                }
+                if (elect_one_sync()) {
                     // codes: counted on the leader's full barrier
                     const uint32_t full_leader = map_to_cta(smem_u32(&sm.full[s]), 0);
-                    mbar_arrive_expect_tx_cluster(full_leader, kPABytes + kPBBytes);
-                    tma_load_2d_pair(sm.a[s], &tm_a, full_leader, ks * 128, tm * kPTileM + rank * kPHalfM);
-                    tma_load_2d_pair(sm.b[s], &tm_b, full_leader, ks * 128, tn * kPTileN + rank * kPHalfN);
-                    // scales: local
-                    const int kt0 = ks * 2;
-                    const int nkt = min(2, p.sf_tiles_k - kt0);
+                    mbar_arrive_expect_tx_cluster(full_leader, 4 * kPBoxBytes);
+                    const int32_t xa = ks * (kPBlockK / 2);
+                    const int32_t ya = tm * kPTileM + rank * kPHalfM, yb = tn * kPTileN + rank * kPHalfN;
+                    tma_load_2d_pair(sm.a[s][0], &tm_a, full_leader, xa, ya);
+                    tma_load_2d_pair(sm.b[s][0], &tm_b, full_leader, xa, yb);
+                    tma_load_2d_pair(sm.a[s][1], &tm_a, full_leader, xa + 128, ya);
+                    tma_load_2d_pair(sm.b[s][1], &tm_b, full_leader, xa + 128, yb);
+                    // scales: local barrier
+                    const int kt0 = ks * 4;
+                    const int nkt = min(4, p.sf_tiles_k - kt0);
                     const uint32_t sf_bytes = nkt * 512;
                     const int has_a = a_row_tile < p.sf_rows_a ? 1 : 0;
                     const int nb0 = tn * 2;
@@ -180,122 +189,100 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                                      p.a_scales + (static_cast<int64_t>(a_row_tile) * p.sf_tiles_k + kt0) * 512,
                                      sf_bytes, &sm.sf_full[s]);
                     for (int nb = 0; nb < nnb; ++nb)
-                        bulk_load_1d(&sm.sfb[s][nb * 1024],
+                        bulk_load_1d(&sm.sfb[s][nb * 2048],
                                      p.b_scales + (static_cast<int64_t>(nb0 + nb) * p.sf_tiles_k + kt0) * 512,
                                      sf_bytes, &sm.sf_full[s]);
-                    }
-                    __syncwarp();
                 }
+                __syncwarp();
             }
         }
     } else if (warp == kPMmaWarp) {
         // ------------------------------------------------------------ MMA issuer (leader only)
         setmaxnreg_dec<56>();
-        if (rank == 0) {
-            // whole warp in uniform control flow; one elected lane issues MMAs and commits
+        if (rank == 0 && total_it > 0) {
             int it = 0;
             bool alive = true;
+            // readiness of the current stage as seen by the test issued one stage earlier
+            bool rdy_full = false, rdy_sf = false;
             for (int tile_it = 0; alive && tile_it < my_tiles; ++tile_it) {
                 if (tile_it > 0 && !mbar_wait(&sm.tmem_empty, (tile_it - 1) & 1, &sm.abort_flag)) break;
-                tcgen05_fence_after();
                 for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
                     const int s = it % kPStages;
                     const uint32_t parity = (it / kPStages) & 1;
-#ifdef MXFP4_PROBE
-                    long long pt0 = clock64();
-                    bool okw = mbar_wait(&sm.full[s], parity, &sm.abort_flag);
-                    long long pt1 = clock64();
-                    okw = okw && ((p.debug & 2) || mbar_wait(&sm.sf_ready[s], parity, &sm.abort_flag));
-                    long long pt2 = clock64();
-                    if (blockIdx.x == 0 && it >= 64 && it < 128) {
-                        p.probe_out[8 + (it - 64) * 3] = pt0; p.probe_out[8 + (it - 64) * 3 + 1] = pt1; p.probe_out[8 + (it - 64) * 3 + 2] = pt2;
-                    }
-                    if (!okw) { alive = false; break; }
-#else
-                    if (!mbar_wait(&sm.full[s], parity, &sm.abort_flag) ||
-                        !mbar_wait(&sm.sf_ready[s], parity, &sm.abort_flag)) {
+                    // codes landed in both CTAs' shared memory; scales landed in both CTAs' TMEM
+                    if ((!rdy_full && !mbar_wait(&sm.full[s], parity, &sm.abort_flag)) ||
+                        (!rdy_sf && !mbar_wait(&sm.sf_ready[s], parity, &sm.abort_flag))) {
                         alive = false;
                         break;
                     }
-#endif
                     tcgen05_fence_after();
+                    if (it + 1 < total_it) {
+                        const int s1 = (it + 1) % kPStages;
+                        const uint32_t parity1 = ((it + 1) / kPStages) & 1;
+                        rdy_full = mbar_test_wait(&sm.full[s1], parity1);
+                        rdy_sf = mbar_test_wait(&sm.sf_ready[s1], parity1);
+                    }
                     const uint32_t sf_tmem = tmem + kPTmemSfBase + s * kPTmemSfPerBuf;
                     const int valid_k = min(kPBlockK, p.K - ks * kPBlockK);
                     const int nmma = (valid_k + 63) / 64;
-                    const uint64_t a_desc = make_smem_desc(smem_u32(sm.a[s]), 16, 1024, 2);
-                    const uint64_t b_desc = make_smem_desc(smem_u32(sm.b[s]), 16, 1024, 2);
                     if (elect_one_sync()) {
-                    for (int j = 0; j < nmma; ++j) {
-                        const uint32_t sf_id = (j & 1) * 2;
-                        tcgen05_mma_mxf4_pair(tmem, a_desc + 2 * j, b_desc + 2 * j,
-                                              make_idesc_mxf4_pair(sf_id, sf_id), sf_tmem + (j >> 1) * 4,
-                                              sf_tmem + 8 + (j >> 1) * 8, (ks > 0 || j > 0) ? 1u : 0u);
-#ifdef MXFP4_PROBE
-                        if (blockIdx.x == 0 && it >= 64 && it < 128) p.probe_out[600 + (it - 64) * 5 + j] = clock64();
-#endif
-                    }
-                    tcgen05_commit_pair(&sm.empty[s], 3);     // stage + scale columns free, both CTAs
-#ifdef MXFP4_PROBE
-                    if (blockIdx.x == 0 && it >= 64 && it < 128) p.probe_out[600 + (it - 64) * 5 + 4] = clock64();
-#endif
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (j < nmma) {
+                                // K half j>>2 (its own 128-byte swizzled box), 32 bytes per K = 64
+                                const uint64_t a_desc =
+                                    make_smem_desc(smem_u32(sm.a[s][j >> 2]) + (j & 3) * 32, 16, 1024, 2);
+                                const uint64_t b_desc =
+                                    make_smem_desc(smem_u32(sm.b[s][j >> 2]) + (j & 3) * 32, 16, 1024, 2);
+                                const uint32_t sf_id = (j & 1) * 2;
+                                tcgen05_mma_mxf4_pair(tmem, a_desc, b_desc, make_idesc_mxf4_pair(sf_id, sf_id),
+                                                      sf_tmem + (j >> 1) * 4, sf_tmem + 16 + (j >> 1) * 8,
+                                                      (ks > 0 || j > 0) ? 1u : 0u);
+                            }
+                        }
+                        // frees the shared-memory stage and its TMEM scale columns in both CTAs
+                        tcgen05_commit_pair(&sm.empty[s], 3);
                     }
                     __syncwarp();
                 }
-                __syncwarp();
                 if (alive && elect_one_sync()) tcgen05_commit_pair(&sm.tmem_full, 3);
                 __syncwarp();
             }
         }
     } else if (warp < 4) {
         // ------------------------------------------------------------ scale warps
+        // Lane r of every quadrant must hold, per 128-row x 4-block scale tile, the 16 bytes at
+        // offset 16*r of that tile: four 32-bit columns = rows r, r+32, r+64, r+96.  Stage s
+        // owns TMEM columns [s*48, s*48+48): SFA K-tiles 0..3 (4 columns each) | SFB K-tiles
+        // 0..3 (8 columns each: row blocks 0, 1).  The columns are free again once the producer
+        // has seen empty[s], which happens before sf_full[s] can complete.
         setmaxnreg_dec<56>();
         const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
-#ifdef MXFP4_PROBE
-        if (!(p.debug & 8))
-#endif
+        const uint32_t sf_ready_leader_base = map_to_cta(smem_u32(&sm.sf_ready[0]), 0);
         for (int it = 0; it < total_it; ++it) {
             const int s = it % kPStages;
-#ifdef MXFP4_PROBE
-            long long q0 = clock64();
-#endif
             if (!mbar_wait(&sm.sf_full[s], (it / kPStages) & 1, &sm.abort_flag)) break;
-#ifdef MXFP4_PROBE
-            long long q1 = clock64();
-#endif
-            const uint4 a0 = *reinterpret_cast<const uint4*>(&sm.sfa[s][lane * 16]);
-            const uint4 a1 = *reinterpret_cast<const uint4*>(&sm.sfa[s][512 + lane * 16]);
-            const uint4 b00 = *reinterpret_cast<const uint4*>(&sm.sfb[s][lane * 16]);
-            const uint4 b01 = *reinterpret_cast<const uint4*>(&sm.sfb[s][1024 + lane * 16]);
-            const uint4 b10 = *reinterpret_cast<const uint4*>(&sm.sfb[s][512 + lane * 16]);
-            const uint4 b11 = *reinterpret_cast<const uint4*>(&sm.sfb[s][1536 + lane * 16]);
             const uint32_t t = tmem + lane_base + kPTmemSfBase + s * kPTmemSfPerBuf;
-            tmem_st_32x32b_x8(t, a0, a1);
-            tmem_st_32x32b_x8(t + 8, b00, b01);
-            tmem_st_32x32b_x8(t + 16, b10, b11);
-#ifdef MXFP4_PROBE
-            long long q2 = clock64();
-#endif
+            const uint8_t* sa = &sm.sfa[s][lane * 16];
+            const uint8_t* sb = &sm.sfb[s][lane * 16];
+            tmem_st_32x32b_x8(t, *reinterpret_cast<const uint4*>(sa), *reinterpret_cast<const uint4*>(sa + 512));
+            tmem_st_32x32b_x8(t + 8, *reinterpret_cast<const uint4*>(sa + 1024),
+                              *reinterpret_cast<const uint4*>(sa + 1536));
+#pragma unroll
+            for (int kt = 0; kt < 4; ++kt)
+                tmem_st_32x32b_x8(t + 16 + kt * 8, *reinterpret_cast<const uint4*>(sb + kt * 512),
+                                  *reinterpret_cast<const uint4*>(sb + 2048 + kt * 512));
             tmem_st_wait();
-#ifdef MXFP4_PROBE
-            long long q3 = clock64();
-#endif
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sm.sf_ready[s]), 0));
-#ifdef MXFP4_PROBE
-            if (blockIdx.x == 0 && warp == 0 && lane == 0 && it >= 64 && it < 128) {
-                long long q4 = clock64();
-                long long* o = p.probe_out + 256 + (it - 64) * 5;
-                o[0] = q0; o[1] = q1; o[2] = q2; o[3] = q3; o[4] = q4;
-            }
-#endif
+            if (lane == 0) mbar_arrive_cluster(sf_ready_leader_base + s * 8);
         }
     } else if (warp < 12) {
         // ------------------------------------------------------------ epilogue warps
         setmaxnreg_inc<192>();
         const int ew = warp - 4;
-        const int quad = warp & 3;
-        const int half = ew >> 2;
+        const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+        const int half = ew >> 2;                  // which 128 accumulator columns
         uint8_t* stg = sm.out_stage[ew];
         const uint32_t tmem_empty_leader = map_to_cta(smem_u32(&sm.tmem_empty), 0);
         for (int tile_it = 0; tile_it < my_tiles; ++tile_it) {
@@ -308,15 +295,13 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(taddr + c * 32, r[c]);
             tmem_ld_wait();
+            // the accumulator is in registers: release TMEM before converting and storing
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
 
             const int64_t row0 = static_cast<int64_t>(tm) * kPTileM + rank * kPHalfM + quad * 32;
             const int64_t colbase = static_cast<int64_t>(tn) * kPTileN + half * 128;
-#ifdef MXFP4_PROBE
-            if (p.debug & 4) continue;
-#endif
             if (p.out_fp32) {
                 const int64_t row = row0 + lane;
 #pragma unroll
@@ -340,27 +325,30 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                 }
             } else {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 8; ++c) {
+                    // own row (= lane), 16 columns -> 32 bytes; the two 16-byte chunks of a row
+                    // are swapped on alternate groups of four rows so that row-wise writes and
+                    // the 16-rows-per-instruction reads below stay bank-conflict free
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
+                    for (int q = 0; q < 2; ++q) {
                         uint32_t w[4];
 #pragma unroll
                         for (int h = 0; h < 4; ++h) {
                             const __nv_bfloat162 v = __floats2bfloat162_rn(
-                                __uint_as_float(r[c][8 * q + 2 * h]) * p.alpha,
-                                __uint_as_float(r[c][8 * q + 2 * h + 1]) * p.alpha);
+                                __uint_as_float(r[c >> 1][(c & 1) * 16 + 8 * q + 2 * h]) * p.alpha,
+                                __uint_as_float(r[c >> 1][(c & 1) * 16 + 8 * q + 2 * h + 1]) * p.alpha);
                             w[h] = *reinterpret_cast<const uint32_t*>(&v);
                         }
-                        *reinterpret_cast<uint4*>(stg + lane * 64 + ((q ^ ((lane >> 1) & 3)) * 16)) =
+                        *reinterpret_cast<uint4*>(stg + lane * 32 + ((q ^ ((lane >> 2) & 1)) * 16)) =
                             make_uint4(w[0], w[1], w[2], w[3]);
                     }
                     __syncwarp();
-                    const int64_t col0 = colbase + c * 32 + (lane & 3) * 8;
+                    const int64_t col0 = colbase + c * 16 + (lane & 1) * 8;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int rr = i * 8 + (lane >> 2);
+                    for (int i = 0; i < 2; ++i) {
+                        const int rr = i * 16 + (lane >> 1);
                         const uint4 v = *reinterpret_cast<const uint4*>(
-                            stg + rr * 64 + (((lane & 3) ^ ((rr >> 1) & 3)) * 16));
+                            stg + rr * 32 + (((lane & 1) ^ ((rr >> 2) & 1)) * 16));
                         const int64_t row = row0 + rr;
                         if (row < p.M && col0 < p.N) {
                             __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.out) + row * p.ld_out + col0;
@@ -396,6 +384,7 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
                             int out_dtype, int64_t ld_out, int sm_count, cudaStream_t stream)
 {
     CUtensorMap tm_a, tm_b;
+    // codes as bytes: [rows x K/2], box = 128 bytes x 128 rows, 128-byte swizzle
     if (!make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a_codes, M, K / 2, K / 2, kPHalfM, 128,
                       CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b_codes, N, K / 2, K / 2, kPHalfN, 128,
@@ -417,9 +406,6 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     p.sf_rows_b = static_cast<int32_t>((N + 127) / 128);
     p.alpha = alpha;
     p.out_fp32 = out_dtype == MXFP4_OUT_FP32;
-#ifdef MXFP4_PROBE
-    { static long long* buf = nullptr; if (!buf) cudaMalloc(&buf, 8192); p.probe_out = buf; const char* e = getenv("MXFP4_GEMM_DEBUG"); p.debug = e ? atoi(e) : 0; }
-#endif
     const int64_t total = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
     if (total > 0x3FFFFFFF) return MXFP4_ERR_SHAPE;
     const size_t smem = sizeof(GemmPairSmem) + 1024;
@@ -433,9 +419,6 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     const int max_clusters = sm_count / 2;
     const int clusters = static_cast<int>(total < max_clusters ? total : max_clusters);
     gemm_mxf4_pair_kernel<<<2 * clusters, kPThreads, smem, stream>>>(tm_a, tm_b, p);
-#ifdef MXFP4_PROBE
-    if (getenv("MXFP4_GEMM_TRACE")) { static long long h[1024]; cudaStreamSynchronize(stream); cudaMemcpy(h, p.probe_out, 8192, cudaMemcpyDeviceToHost); for (int i = 1; i < 64; ++i) { long long* o = h + 256 + i * 5; fprintf(stderr, "scale it %d: loop gap %lld | wait sf_full %lld | lds+st issue %lld | wait::st %lld | arrive %lld\n", 64 + i, o[0] - o[-1], o[1] - o[0], o[2] - o[1], o[3] - o[2], o[4] - o[3]); } for (int i = 0; i < 64; ++i) { long long* o = h + 600 + i * 5; fprintf(stderr, "issue it %d: mma0 %lld mma1 %lld mma2 %lld mma3 %lld commit %lld\n", 64 + i, o[0] - h[8 + i * 3 + 2], o[1] - o[0], o[2] - o[1], o[3] - o[2], o[4] - o[3]); } for (int i = 0; i < 64; ++i) fprintf(stderr, "it %d: since prev issue %lld | wait full %lld | wait sf %lld\n", 64 + i, i ? h[8 + i * 3] - h[8 + (i - 1) * 3 + 2] : 0, h[8 + i * 3 + 1] - h[8 + i * 3], h[8 + i * 3 + 2] - h[8 + i * 3 + 1]); }
-#endif
     return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 

@@ -5,13 +5,11 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <string.h>
-#include <stdlib.h>
 
 #include "../../include/mxfp4.h"
 #include "ptx_sm100.cuh"
 #include "tma_host.cuh"
 #include "quantize_kernel.cuh"
-#include "gemm_kernel.cuh"
 #include "gemm_pair_kernel.cuh"
 
 namespace mxfp4 {
@@ -201,12 +199,6 @@ int mxfp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes,
     const DeviceInfo& dev = device_info();
     if (!dev.ok) return MXFP4_ERR_CUDA;
     if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
-    {
-        const char* e = getenv("MXFP4_GEMM_KERNEL");   // temporary selector while the pair kernel is validated
-        if (e && e[0] == '1')
-            return launch_gemm(a_codes, a_scales, b_codes, b_scales, M, N, K, alpha, out, out_dtype, ld_out,
-                               dev.sm_count, static_cast<cudaStream_t>(stream));
-    }
     return launch_gemm_pair(a_codes, a_scales, b_codes, b_scales, M, N, K, alpha, out, out_dtype, ld_out,
                             dev.sm_count, static_cast<cudaStream_t>(stream));
 }
