@@ -3,24 +3,27 @@
 //
 //   out[m][n] = alpha * sum_t 2^(sa[m][t]-127) 2^(sb[n][t]-127) sum_{k in block t} A[m][k] B[n][k]
 //
-// CTA-pair kernel (tcgen05 cta_group::2): the two CTAs of a cluster share one 256 x 256 output
-// tile.  Each CTA loads its own 128 rows of A and its own 128 rows of B (64 KB per K-step of 512
-// elements, against the 96 KB a lone 128 x 256 tile would need), because the L2 -> shared-memory
-// operand feed, not the tensor pipe, is what bounds an FP4 GEMM here.  No TMA multicast is used:
-// every CTA fetches its own operands; only barrier signals cross the pair.
+// CTA-pair kernel (tcgen05 cta_group::2): the two CTAs of a cluster share one 256 x 384 output
+// tile (two 256 x 192 MMAs per K = 64).  Each CTA loads its own 128 rows of A and its own
+// 2 x 96 rows of B: 40 KB per K-step of 256 elements for 128 x 384 outputs, against the 48 KB a
+// lone 128 x 256 tile needs for two thirds of that -- the L2 -> shared-memory operand feed
+// (about 10.5 TB/s on this part), not the tensor pipe, is what bounds an FP4 GEMM here, and the
+// 512 TMEM columns are exactly used up: 384 accumulator + 4 x 32 scale columns.  No TMA
+// multicast is used: every CTA fetches its own operands; only barrier signals cross the pair.
 //
 // Roles per CTA (512 threads, four warpgroups; registers rebalanced with setmaxnreg):
 //   warps 0..3   scale warps (one per TMEM lane quadrant): shared memory -> this CTA's TMEM scale
 //                columns with tcgen05.st.  (tcgen05.cp would do the same copy, but measured here
 //                each one holds the tensor pipe for 70-85 cycles whatever its shape, and a
-//                K-step needs twelve of them against 1024 cycles of MMA.)
-//   warps 4..11  epilogue: this CTA's 128 rows x 256 columns of the accumulator; four
-//                back-to-back tcgen05.ld per warp, accumulator handed back at once, then
-//                alpha, conversion and stores overlap the next tile's main loop.
-//   warp 12      TMA producer: A and B halves (completion counted on the LEADER's barrier) and
-//                the scale tiles (local barrier), 3-stage ring.
+//                K-step needs eight of them against 768 cycles of MMA.)
+//   warps 4..11  epilogue: this CTA's 128 rows x 384 columns of the accumulator, 32 rows x 192
+//                columns per warp in two rounds of three tcgen05.ld; the accumulator is handed
+//                back as soon as the second round has landed, then alpha, conversion and stores
+//                overlap the next tile's main loop.
+//   warp 12      TMA producer: A half and two B sub-tiles (completion counted on the LEADER's
+//                barrier) and the scale tiles (local barrier), 4-stage ring.
 //   warp 13      MMA issuer, leader CTA (cluster rank 0) only: eight
-//                tcgen05.mma.cta_group::2.kind::mxf4.block_scale (256 x 256 x 64) per stage; its
+//                tcgen05.mma.cta_group::2.kind::mxf4.block_scale (256 x 192 x 64) per stage; its
 //                commits arrive on the barriers of both CTAs.
 // The issuing warps run their loops in warp-uniform control flow and issue through
 // elect.sync, so descriptors stay in uniform registers; the MMA warp tests the next stage's
@@ -43,26 +46,28 @@
 namespace mxfp4 {
 
 constexpr int kPHalfM = 128;                     // rows of A (and of the accumulator) per CTA
-constexpr int kPHalfN = 128;                     // rows of B per CTA
 constexpr int kPTileM = 256;
-constexpr int kPTileN = 256;
-constexpr int kPBlockK = 512;                    // elements per stage: two 128-byte swizzled boxes
-constexpr int kPStages = 3;
-constexpr int kPBoxBytes = 128 * 128;            // 128 rows x 128 bytes of codes = 16 KB
-constexpr int kPSfaBytes = 4 * 512;              // own 128 rows x 4 K-tiles of 128 elements
-constexpr int kPSfbBytes = 2 * 4 * 512;          // both 128-row blocks of B x 4 K-tiles
+constexpr int kPTileN = 384;                     // two MMAs of N = 192 per K = 64
+constexpr int kPMmaN = 192;
+constexpr int kPSubN = 96;                       // rows of B per CTA per MMA
+constexpr int kPBlockK = 256;                    // elements per stage = 128 bytes of codes per row
+constexpr int kPStages = 4;
+constexpr int kPABytes = kPHalfM * 128;          // 16 KB
+constexpr int kPBSubBytes = kPSubN * 128;        // 12 KB
+constexpr int kPSfaBytes = 2 * 512;              // own 128 rows x 2 K-tiles of 128 elements
+constexpr int kPSfbBytes = 3 * 2 * 512;          // three 128-row blocks of B x 2 K-tiles
 constexpr int kPEpiWarps = 8;
 constexpr int kPProducerWarp = 12;
 constexpr int kPMmaWarp = 13;
 constexpr int kPThreads = 512;
 constexpr uint32_t kPTmemCols = 512;
-constexpr uint32_t kPTmemSfBase = 256;           // accumulator occupies columns 0..255
-constexpr uint32_t kPTmemSfPerBuf = 48;          // per stage: 16 columns SFA + 32 columns SFB
+constexpr uint32_t kPTmemSfBase = 384;           // accumulator occupies columns 0..383
+constexpr uint32_t kPTmemSfPerBuf = 32;          // per stage: 8 columns SFA + 24 columns SFB
 
 struct GemmPairSmem {
-    alignas(1024) uint8_t a[kPStages][2][kPBoxBytes];     // [stage][K half][128 rows x 128 B]
-    alignas(1024) uint8_t b[kPStages][2][kPBoxBytes];
-    alignas(128) uint8_t sfa[kPStages][kPSfaBytes];
+    alignas(1024) uint8_t a[kPStages][kPABytes];          // 128 rows x 128 B
+    alignas(1024) uint8_t b[kPStages][2][kPBSubBytes];    // [MMA half][96 rows x 128 B]
+    alignas(128) uint8_t sfa[kPStages][kPSfaBytes];       // [K-tile][512]
     alignas(128) uint8_t sfb[kPStages][kPSfbBytes];       // [row block][K-tile][512]
     alignas(128) uint8_t out_stage[kPEpiWarps][32 * 32];  // 32 rows x 16 bf16 per warp
     alignas(8) uint64_t full[kPStages];      // leader's copy is the live one
@@ -81,8 +86,8 @@ struct GemmPairParams {
     void* out;
     int64_t ld_out;
     int32_t M, N, K;
-    int32_t tiles_m, tiles_n;   // 256 x 256 pair tiles
-    int32_t k_stages;           // ceil(K / 512)
+    int32_t tiles_m, tiles_n;   // 256 x 384 pair tiles
+    int32_t k_stages;           // ceil(K / 256)
     int32_t sf_tiles_k;         // ceil(K / 128)
     int32_t sf_rows_a;          // ceil(M / 128)
     int32_t sf_rows_b;          // ceil(N / 128)
@@ -91,7 +96,7 @@ struct GemmPairParams {
 };
 
 // Instruction descriptor of the pair MMA: E2M1 x E2M1, E8M0 scales, both operands K-major,
-// M = 256 (128 per CTA), N = 256.  Scale-factor ids select which byte pair of the 32-bit TMEM
+// M = 256 (128 per CTA), N = 192.  Scale-factor ids select which byte pair of the 32-bit TMEM
 // scale column an instruction uses.
 __device__ __forceinline__ uint32_t make_idesc_mxf4_pair(uint32_t a_sf_id, uint32_t b_sf_id)
 {
@@ -99,7 +104,7 @@ __device__ __forceinline__ uint32_t make_idesc_mxf4_pair(uint32_t a_sf_id, uint3
     d |= b_sf_id << 4;                 // bits 4..5   B scale-factor id
     d |= 1u << 7;                      // bits 7..9   A format: E2M1
     d |= 1u << 10;                     // bits 10..12 B format: E2M1
-    d |= (kPTileN >> 3) << 17;         // bits 17..22 N / 8
+    d |= (kPMmaN >> 3) << 17;          // bits 17..22 N / 8
     d |= 1u << 23;                     // bit 23      scale format: E8M0
     d |= (kPTileM >> 4) << 24;         // bits 24..28 M / 16
     d |= a_sf_id << 29;                // bits 29..30 A scale-factor id
@@ -169,27 +174,27 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                 if (elect_one_sync()) {
                     // codes: counted on the leader's full barrier
                     const uint32_t full_leader = map_to_cta(smem_u32(&sm.full[s]), 0);
-                    mbar_arrive_expect_tx_cluster(full_leader, 4 * kPBoxBytes);
-                    const int32_t xa = ks * (kPBlockK / 2);
-                    const int32_t ya = tm * kPTileM + rank * kPHalfM, yb = tn * kPTileN + rank * kPHalfN;
-                    tma_load_2d_pair(sm.a[s][0], &tm_a, full_leader, xa, ya);
-                    tma_load_2d_pair(sm.b[s][0], &tm_b, full_leader, xa, yb);
-                    tma_load_2d_pair(sm.a[s][1], &tm_a, full_leader, xa + 128, ya);
-                    tma_load_2d_pair(sm.b[s][1], &tm_b, full_leader, xa + 128, yb);
+                    mbar_arrive_expect_tx_cluster(full_leader, kPABytes + 2 * kPBSubBytes);
+                    const int32_t x = ks * (kPBlockK / 2);
+                    const int32_t ya = tm * kPTileM + rank * kPHalfM;
+                    const int32_t yb = tn * kPTileN + rank * kPSubN;
+                    tma_load_2d_pair(sm.a[s], &tm_a, full_leader, x, ya);
+                    tma_load_2d_pair(sm.b[s][0], &tm_b, full_leader, x, yb);
+                    tma_load_2d_pair(sm.b[s][1], &tm_b, full_leader, x, yb + kPMmaN);
                     // scales: local barrier
-                    const int kt0 = ks * 4;
-                    const int nkt = min(4, p.sf_tiles_k - kt0);
+                    const int kt0 = ks * 2;
+                    const int nkt = min(2, p.sf_tiles_k - kt0);
                     const uint32_t sf_bytes = nkt * 512;
                     const int has_a = a_row_tile < p.sf_rows_a ? 1 : 0;
-                    const int nb0 = tn * 2;
-                    const int nnb = max(0, min(2, p.sf_rows_b - nb0));
+                    const int nb0 = tn * 3;
+                    const int nnb = max(0, min(3, p.sf_rows_b - nb0));
                     mbar_arrive_expect_tx(&sm.sf_full[s], sf_bytes * (has_a + nnb));
                     if (has_a)
                         bulk_load_1d(sm.sfa[s],
                                      p.a_scales + (static_cast<int64_t>(a_row_tile) * p.sf_tiles_k + kt0) * 512,
                                      sf_bytes, &sm.sf_full[s]);
                     for (int nb = 0; nb < nnb; ++nb)
-                        bulk_load_1d(&sm.sfb[s][nb * 2048],
+                        bulk_load_1d(&sm.sfb[s][nb * 1024],
                                      p.b_scales + (static_cast<int64_t>(nb0 + nb) * p.sf_tiles_k + kt0) * 512,
                                      sf_bytes, &sm.sf_full[s]);
                 }
@@ -227,17 +232,22 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                     const int nmma = (valid_k + 63) / 64;
                     if (elect_one_sync()) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
+                        for (int j = 0; j < 4; ++j) {
                             if (j < nmma) {
-                                // K half j>>2 (its own 128-byte swizzled box), 32 bytes per K = 64
-                                const uint64_t a_desc =
-                                    make_smem_desc(smem_u32(sm.a[s][j >> 2]) + (j & 3) * 32, 16, 1024, 2);
-                                const uint64_t b_desc =
-                                    make_smem_desc(smem_u32(sm.b[s][j >> 2]) + (j & 3) * 32, 16, 1024, 2);
+                                // K = 64 step j: 32 bytes along the 128-byte swizzled row; two
+                                // MMAs, one per 192-column half of the tile
+                                const uint64_t a_desc = make_smem_desc(smem_u32(sm.a[s]) + j * 32, 16, 1024, 2);
                                 const uint32_t sf_id = (j & 1) * 2;
-                                tcgen05_mma_mxf4_pair(tmem, a_desc, b_desc, make_idesc_mxf4_pair(sf_id, sf_id),
-                                                      sf_tmem + (j >> 1) * 4, sf_tmem + 16 + (j >> 1) * 8,
-                                                      (ks > 0 || j > 0) ? 1u : 0u);
+                                const uint32_t idesc = make_idesc_mxf4_pair(sf_id, sf_id);
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    const uint64_t b_desc =
+                                        make_smem_desc(smem_u32(sm.b[s][h]) + j * 32, 16, 1024, 2);
+                                    tcgen05_mma_mxf4_pair(tmem + h * kPMmaN, a_desc, b_desc, idesc,
+                                                          sf_tmem + (j >> 1) * 4,
+                                                          sf_tmem + 8 + (j >> 1) * 12 + h * 6,
+                                                          (ks > 0 || j > 0) ? 1u : 0u);
+                                }
                             }
                         }
                         // frees the shared-memory stage and its TMEM scale columns in both CTAs
@@ -253,9 +263,9 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
         // ------------------------------------------------------------ scale warps
         // Lane r of every quadrant must hold, per 128-row x 4-block scale tile, the 16 bytes at
         // offset 16*r of that tile: four 32-bit columns = rows r, r+32, r+64, r+96.  Stage s
-        // owns TMEM columns [s*48, s*48+48): SFA K-tiles 0..3 (4 columns each) | SFB K-tiles
-        // 0..3 (8 columns each: row blocks 0, 1).  The columns are free again once the producer
-        // has seen empty[s], which happens before sf_full[s] can complete.
+        // owns TMEM columns [s*32, s*32+32): SFA K-tiles 0,1 (4 columns each) | SFB K-tile 0
+        // (12 columns: row blocks 0,1,2) | SFB K-tile 1.  The columns are free again once the
+        // producer has seen empty[s], which happens before sf_full[s] can complete.
         setmaxnreg_dec<56>();
         const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
         const uint32_t sf_ready_leader_base = map_to_cta(smem_u32(&sm.sf_ready[0]), 0);
@@ -264,14 +274,12 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
             if (!mbar_wait(&sm.sf_full[s], (it / kPStages) & 1, &sm.abort_flag)) break;
             const uint32_t t = tmem + lane_base + kPTmemSfBase + s * kPTmemSfPerBuf;
             const uint8_t* sa = &sm.sfa[s][lane * 16];
-            const uint8_t* sb = &sm.sfb[s][lane * 16];
-            tmem_st_32x32b_x8(t, *reinterpret_cast<const uint4*>(sa), *reinterpret_cast<const uint4*>(sa + 512));
-            tmem_st_32x32b_x8(t + 8, *reinterpret_cast<const uint4*>(sa + 1024),
-                              *reinterpret_cast<const uint4*>(sa + 1536));
-#pragma unroll
-            for (int kt = 0; kt < 4; ++kt)
-                tmem_st_32x32b_x8(t + 16 + kt * 8, *reinterpret_cast<const uint4*>(sb + kt * 512),
-                                  *reinterpret_cast<const uint4*>(sb + 2048 + kt * 512));
+            const uint8_t* sb = &sm.sfb[s][lane * 16];           // [row block nb][K-tile kt] at nb*1024 + kt*512
+            auto ld = [](const uint8_t* q) { return *reinterpret_cast<const uint4*>(q); };
+            tmem_st_32x32b_x8(t, ld(sa), ld(sa + 512));                       // SFA kt0 | kt1
+            tmem_st_32x32b_x8(t + 8, ld(sb), ld(sb + 1024));                  // SFB kt0: nb0 | nb1
+            tmem_st_32x32b_x8(t + 16, ld(sb + 2048), ld(sb + 512));           // SFB kt0: nb2 | kt1: nb0
+            tmem_st_32x32b_x8(t + 24, ld(sb + 1024 + 512), ld(sb + 2048 + 512));  // SFB kt1: nb1 | nb2
             tmem_st_wait();
             tcgen05_fence_before();
             __syncwarp();
@@ -282,7 +290,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
         setmaxnreg_inc<192>();
         const int ew = warp - 4;
         const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
-        const int half = ew >> 2;                  // which 128 accumulator columns
+        const int half = ew >> 2;                  // which 192 accumulator columns
         uint8_t* stg = sm.out_stage[ew];
         const uint32_t tmem_empty_leader = map_to_cta(smem_u32(&sm.tmem_empty), 0);
         for (int tile_it = 0; tile_it < my_tiles; ++tile_it) {
@@ -290,58 +298,78 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
             const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
             if (!mbar_wait(&sm.tmem_full, tile_it & 1, &sm.abort_flag)) break;
             tcgen05_fence_after();
-            uint32_t r[4][32];
-            const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + half * 128;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(taddr + c * 32, r[c]);
-            tmem_ld_wait();
-            // the accumulator is in registers: release TMEM before converting and storing
-            tcgen05_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
-
+            const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + half * kPMmaN;
             const int64_t row0 = static_cast<int64_t>(tm) * kPTileM + rank * kPHalfM + quad * 32;
-            const int64_t colbase = static_cast<int64_t>(tn) * kPTileN + half * 128;
+            const int64_t colbase = static_cast<int64_t>(tn) * kPTileN + half * kPMmaN;
             if (p.out_fp32) {
+                // fp32 output: two rounds of 96 columns; TMEM is released after the second load
                 const int64_t row = row0 + lane;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int64_t col0 = colbase + c * 32;
-                    if (row >= p.M || col0 >= p.N) continue;
-                    float* dst = static_cast<float*>(p.out) + row * p.ld_out + col0;
-                    if (col0 + 32 <= p.N) {
+                for (int round = 0; round < 2; ++round) {
+                    uint32_t r[3][32];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            reinterpret_cast<float4*>(dst)[i] =
-                                make_float4(__uint_as_float(r[c][4 * i]) * p.alpha,
-                                            __uint_as_float(r[c][4 * i + 1]) * p.alpha,
-                                            __uint_as_float(r[c][4 * i + 2]) * p.alpha,
-                                            __uint_as_float(r[c][4 * i + 3]) * p.alpha);
-                    } else {
+                    for (int c = 0; c < 3; ++c) tmem_ld_32x32b_x32(taddr + round * 96 + c * 32, r[c]);
+                    tmem_ld_wait();
+                    if (round == 1) {
+                        tcgen05_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
+                    }
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (col0 + i < p.N) dst[i] = __uint_as_float(r[c][i]) * p.alpha;
+                    for (int c = 0; c < 3; ++c) {
+                        const int64_t col0 = colbase + round * 96 + c * 32;
+                        if (row >= p.M || col0 >= p.N) continue;
+                        float* dst = static_cast<float*>(p.out) + row * p.ld_out + col0;
+                        if (col0 + 32 <= p.N) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                reinterpret_cast<float4*>(dst)[i] =
+                                    make_float4(__uint_as_float(r[c][4 * i]) * p.alpha,
+                                                __uint_as_float(r[c][4 * i + 1]) * p.alpha,
+                                                __uint_as_float(r[c][4 * i + 2]) * p.alpha,
+                                                __uint_as_float(r[c][4 * i + 3]) * p.alpha);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (col0 + i < p.N) dst[i] = __uint_as_float(r[c][i]) * p.alpha;
+                        }
                     }
                 }
             } else {
+                // bf16 output: 192 columns of this thread's row as 96 packed words; the first 96
+                // columns are converted while the second 96 are still in flight, and TMEM is
+                // released before any store
+                uint32_t w[96];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
+                for (int round = 0; round < 2; ++round) {
+                    uint32_t r[3][32];
+#pragma unroll
+                    for (int c = 0; c < 3; ++c) tmem_ld_32x32b_x32(taddr + round * 96 + c * 32, r[c]);
+                    tmem_ld_wait();
+                    if (round == 1) {
+                        tcgen05_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 3; ++c)
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[c][2 * i]) * p.alpha,
+                                                                           __uint_as_float(r[c][2 * i + 1]) * p.alpha);
+                            w[round * 48 + c * 16 + i] = *reinterpret_cast<const uint32_t*>(&v);
+                        }
+                }
+#pragma unroll
+                for (int c = 0; c < 12; ++c) {
                     // own row (= lane), 16 columns -> 32 bytes; the two 16-byte chunks of a row
                     // are swapped on alternate groups of four rows so that row-wise writes and
                     // the 16-rows-per-instruction reads below stay bank-conflict free
 #pragma unroll
-                    for (int q = 0; q < 2; ++q) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            const __nv_bfloat162 v = __floats2bfloat162_rn(
-                                __uint_as_float(r[c >> 1][(c & 1) * 16 + 8 * q + 2 * h]) * p.alpha,
-                                __uint_as_float(r[c >> 1][(c & 1) * 16 + 8 * q + 2 * h + 1]) * p.alpha);
-                            w[h] = *reinterpret_cast<const uint32_t*>(&v);
-                        }
+                    for (int q = 0; q < 2; ++q)
                         *reinterpret_cast<uint4*>(stg + lane * 32 + ((q ^ ((lane >> 2) & 1)) * 16)) =
-                            make_uint4(w[0], w[1], w[2], w[3]);
-                    }
+                            make_uint4(w[c * 8 + q * 4], w[c * 8 + q * 4 + 1], w[c * 8 + q * 4 + 2],
+                                       w[c * 8 + q * 4 + 3]);
                     __syncwarp();
                     const int64_t col0 = colbase + c * 16 + (lane & 1) * 8;
 #pragma unroll
@@ -384,10 +412,10 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
                             int out_dtype, int64_t ld_out, int sm_count, cudaStream_t stream)
 {
     CUtensorMap tm_a, tm_b;
-    // codes as bytes: [rows x K/2], box = 128 bytes x 128 rows, 128-byte swizzle
+    // codes as bytes: [rows x K/2], boxes of 128 bytes x 128 rows (A) / 96 rows (B), 128-byte swizzle
     if (!make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a_codes, M, K / 2, K / 2, kPHalfM, 128,
                       CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b_codes, N, K / 2, K / 2, kPHalfN, 128,
+        !make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b_codes, N, K / 2, K / 2, kPSubN, 128,
                       CU_TENSOR_MAP_SWIZZLE_128B))
         return MXFP4_ERR_CUDA;
     GemmPairParams p;
