@@ -38,6 +38,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "../../include/mxfp4.h"
 #include "ptx_sm100.cuh"
@@ -69,7 +70,7 @@ struct GemmPairSmem {
     alignas(1024) uint8_t b[kPStages][2][kPBSubBytes];    // [MMA half][96 rows x 128 B]
     alignas(128) uint8_t sfa[kPStages][kPSfaBytes];       // [K-tile][512]
     alignas(128) uint8_t sfb[kPStages][kPSfbBytes];       // [row block][K-tile][512]
-    alignas(128) uint8_t out_stage[kPEpiWarps][32 * 32];  // 32 rows x 16 bf16 per warp
+    alignas(1024) uint8_t out_stage[kPEpiWarps][32 * 128]; // 32 rows x 64 bf16 per warp, 128-byte swizzle
     alignas(8) uint64_t full[kPStages];      // leader's copy is the live one
     uint64_t sf_full[kPStages];              // local
     uint64_t sf_ready[kPStages];             // leader's copy is the live one
@@ -113,7 +114,7 @@ __device__ __forceinline__ uint32_t make_idesc_mxf4_pair(uint32_t a_sf_id, uint3
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
 gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                      const GemmPairParams p)
+                      const __grid_constant__ CUtensorMap tm_out, const GemmPairParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     GemmPairSmem& sm = *reinterpret_cast<GemmPairSmem*>(
@@ -360,39 +361,28 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                             w[round * 48 + c * 16 + i] = *reinterpret_cast<const uint32_t*>(&v);
                         }
                 }
+                // three passes of 64 columns: the warp lays its 32 rows x 128 bytes out in the
+                // 128-byte swizzle and one lane hands the box to a TMA store (which clips at the
+                // matrix edges); the buffer is reused once the previous store has read it
 #pragma unroll
-                for (int c = 0; c < 12; ++c) {
-                    // own row (= lane), 16 columns -> 32 bytes; the two 16-byte chunks of a row
-                    // are swapped on alternate groups of four rows so that row-wise writes and
-                    // the 16-rows-per-instruction reads below stay bank-conflict free
-#pragma unroll
-                    for (int q = 0; q < 2; ++q)
-                        *reinterpret_cast<uint4*>(stg + lane * 32 + ((q ^ ((lane >> 2) & 1)) * 16)) =
-                            make_uint4(w[c * 8 + q * 4], w[c * 8 + q * 4 + 1], w[c * 8 + q * 4 + 2],
-                                       w[c * 8 + q * 4 + 3]);
+                for (int c = 0; c < 3; ++c) {
+                    if (lane == 0) bulk_wait_group_read<0>();
                     __syncwarp();
-                    const int64_t col0 = colbase + c * 16 + (lane & 1) * 8;
 #pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        const int rr = i * 16 + (lane >> 1);
-                        const uint4 v = *reinterpret_cast<const uint4*>(
-                            stg + rr * 32 + (((lane & 1) ^ ((rr >> 2) & 1)) * 16));
-                        const int64_t row = row0 + rr;
-                        if (row < p.M && col0 < p.N) {
-                            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.out) + row * p.ld_out + col0;
-                            if (col0 + 8 <= p.N) {
-                                *reinterpret_cast<uint4*>(dst) = v;
-                            } else {
-                                const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
-                                for (int k = 0; k < 8; ++k)
-                                    if (col0 + k < p.N) dst[k] = e[k];
-                            }
-                        }
+                    for (int q = 0; q < 8; ++q)
+                        *reinterpret_cast<uint4*>(stg + lane * 128 + ((q ^ (lane & 7)) * 16)) =
+                            make_uint4(w[c * 32 + q * 4], w[c * 32 + q * 4 + 1], w[c * 32 + q * 4 + 2],
+                                       w[c * 32 + q * 4 + 3]);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && row0 < p.M && colbase + c * 64 < p.N) {
+                        tma_store_2d(&tm_out, stg, static_cast<int32_t>(colbase + c * 64), static_cast<int32_t>(row0));
+                        bulk_commit_group();
                     }
-                    __syncwarp();
                 }
             }
         }
+        if (lane == 0) bulk_wait_group<0>();
     } else {
         setmaxnreg_dec<56>();   // idle warps of the producer/MMA warpgroup
     }
@@ -411,7 +401,15 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
                             const void* b_scales, int64_t M, int64_t N, int64_t K, float alpha, void* out,
                             int out_dtype, int64_t ld_out, int sm_count, cudaStream_t stream)
 {
-    CUtensorMap tm_a, tm_b;
+    CUtensorMap tm_a, tm_b, tm_out;
+    // bf16 output through TMA stores of 64 columns x 32 rows (fp32 output is stored directly)
+    if (out_dtype == MXFP4_OUT_BF16) {
+        if (!make_tmap_2d(&tm_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, out, M, N, ld_out * 2, 32, 64,
+                          CU_TENSOR_MAP_SWIZZLE_128B))
+            return MXFP4_ERR_CUDA;
+    } else {
+        memset(&tm_out, 0, sizeof(tm_out));
+    }
     // codes as bytes: [rows x K/2], boxes of 128 bytes x 128 rows (A) / 96 rows (B), 128-byte swizzle
     if (!make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a_codes, M, K / 2, K / 2, kPHalfM, 128,
                       CU_TENSOR_MAP_SWIZZLE_128B) ||
@@ -446,7 +444,7 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     }
     const int max_clusters = sm_count / 2;
     const int clusters = static_cast<int>(total < max_clusters ? total : max_clusters);
-    gemm_mxf4_pair_kernel<<<2 * clusters, kPThreads, smem, stream>>>(tm_a, tm_b, p);
+    gemm_mxf4_pair_kernel<<<2 * clusters, kPThreads, smem, stream>>>(tm_a, tm_b, tm_out, p);
     return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
