@@ -210,11 +210,15 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
             bool alive = true;
             // readiness of the current stage as seen by the test issued one stage earlier
             bool rdy_full = false, rdy_sf = false;
+            // descriptors of stage 0; a stage adds a constant, a K = 64 step adds 32 bytes
+            const uint64_t a_desc0 = make_smem_desc(smem_u32(sm.a[0]), 16, 1024, 2);
+            const uint64_t b_desc0 = make_smem_desc(smem_u32(sm.b[0][0]), 16, 1024, 2);
+            const uint32_t idesc0 = make_idesc_mxf4_pair(0, 0), idesc2 = make_idesc_mxf4_pair(2, 2);
+            int s = 0;
+            uint32_t parity = 0;
             for (int tile_it = 0; alive && tile_it < my_tiles; ++tile_it) {
                 if (tile_it > 0 && !mbar_wait(&sm.tmem_empty, (tile_it - 1) & 1, &sm.abort_flag)) break;
                 for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
-                    const int s = it % kPStages;
-                    const uint32_t parity = (it / kPStages) & 1;
                     // codes landed in both CTAs' shared memory; scales landed in both CTAs' TMEM
                     if ((!rdy_full && !mbar_wait(&sm.full[s], parity, &sm.abort_flag)) ||
                         (!rdy_sf && !mbar_wait(&sm.sf_ready[s], parity, &sm.abort_flag))) {
@@ -222,9 +226,9 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                         break;
                     }
                     tcgen05_fence_after();
+                    const int s1 = (s + 1 == kPStages) ? 0 : s + 1;
+                    const uint32_t parity1 = (s + 1 == kPStages) ? parity ^ 1u : parity;
                     if (it + 1 < total_it) {
-                        const int s1 = (it + 1) % kPStages;
-                        const uint32_t parity1 = ((it + 1) / kPStages) & 1;
                         rdy_full = mbar_test_wait(&sm.full[s1], parity1);
                         rdy_sf = mbar_test_wait(&sm.sf_ready[s1], parity1);
                     }
@@ -232,29 +236,28 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                     const int valid_k = min(kPBlockK, p.K - ks * kPBlockK);
                     const int nmma = (valid_k + 63) / 64;
                     if (elect_one_sync()) {
+                        const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(s * (kPABytes >> 4));
+                        const uint64_t b_desc = b_desc0 + static_cast<uint64_t>(s * ((2 * kPBSubBytes) >> 4));
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             if (j < nmma) {
                                 // K = 64 step j: 32 bytes along the 128-byte swizzled row; two
                                 // MMAs, one per 192-column half of the tile
-                                const uint64_t a_desc = make_smem_desc(smem_u32(sm.a[s]) + j * 32, 16, 1024, 2);
-                                const uint32_t sf_id = (j & 1) * 2;
-                                const uint32_t idesc = make_idesc_mxf4_pair(sf_id, sf_id);
 #pragma unroll
-                                for (int h = 0; h < 2; ++h) {
-                                    const uint64_t b_desc =
-                                        make_smem_desc(smem_u32(sm.b[s][h]) + j * 32, 16, 1024, 2);
-                                    tcgen05_mma_mxf4_pair(tmem + h * kPMmaN, a_desc, b_desc, idesc,
-                                                          sf_tmem + (j >> 1) * 4,
+                                for (int h = 0; h < 2; ++h)
+                                    tcgen05_mma_mxf4_pair(tmem + h * kPMmaN, a_desc + 2 * j,
+                                                          b_desc + 2 * j + h * (kPBSubBytes >> 4),
+                                                          (j & 1) ? idesc2 : idesc0, sf_tmem + (j >> 1) * 4,
                                                           sf_tmem + 8 + (j >> 1) * 12 + h * 6,
                                                           (ks > 0 || j > 0) ? 1u : 0u);
-                                }
                             }
                         }
                         // frees the shared-memory stage and its TMEM scale columns in both CTAs
                         tcgen05_commit_pair(&sm.empty[s], 3);
                     }
                     __syncwarp();
+                    s = s1;
+                    parity = parity1;
                 }
                 if (alive && elect_one_sync()) tcgen05_commit_pair(&sm.tmem_full, 3);
                 __syncwarp();
