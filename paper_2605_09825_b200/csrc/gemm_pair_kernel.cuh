@@ -296,6 +296,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
         const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
         const int half = ew >> 2;                  // which 192 accumulator columns
         uint8_t* stg = sm.out_stage[ew];
+        const uint64_t store_policy = l2_policy_evict_first();   // the output streams out once
         const uint32_t tmem_empty_leader = map_to_cta(smem_u32(&sm.tmem_empty), 0);
         for (int tile_it = 0; tile_it < my_tiles; ++tile_it) {
             const int tile = cluster_id + tile_it * n_clusters;
@@ -379,7 +380,8 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0 && row0 < p.M && colbase + c * 64 < p.N) {
-                        tma_store_2d(&tm_out, stg, static_cast<int32_t>(colbase + c * 64), static_cast<int32_t>(row0));
+                        tma_store_2d_hint(&tm_out, stg, static_cast<int32_t>(colbase + c * 64),
+                                          static_cast<int32_t>(row0), store_policy);
                         bulk_commit_group();
                     }
                 }

@@ -133,6 +133,24 @@ __device__ __forceinline__ void tma_store_2d(const void* tmap, const void* smem_
         : "memory");
 }
 
+// L2 eviction-priority policies for cache-hinted TMA traffic.
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+// 2-D tiled store with an L2 cache hint (streaming outputs should not displace operands).
+__device__ __forceinline__ void tma_store_2d_hint(const void* tmap, const void* smem_src, int32_t x,
+                                                  int32_t y, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+        ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(smem_src)), "r"(x), "r"(y), "l"(policy)
+        : "memory");
+}
+
 // 1-D bulk copies (addresses 16-byte aligned, size a multiple of 16).
 __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, uint32_t bytes,
                                              uint64_t* bar)
