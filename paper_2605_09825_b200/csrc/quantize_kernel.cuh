@@ -2,10 +2,13 @@
 // Appendix D), one persistent CTA per SM.
 //
 // Work unit: a tile of 128 operand rows x 128 elements along K (4 MX blocks).  A producer warp
-// streams source tiles into a ring of shared-memory stages with TMA; 512 consumer threads each
-// own one 32-element block per tile: the whole block sits in the thread's registers, so the
-// five butterfly stages (as packed fp32x2 operations), the block maximum and the rounding
-// need no cross-lane traffic.
+// streams source tiles into a ring of shared-memory stages with TMA.  The 512 consumer threads
+// form two groups of 256 that take alternate tiles; a thread handles two 32-element blocks of
+// its group's tile, one after the other, each entirely in registers, so the five butterfly
+// stages (as packed fp32x2 operations), the block maximum and the rounding need no cross-lane
+// traffic.  The two groups synchronise only among themselves, so they sit in different phases
+// (one in its integer/convert instructions while the other is in its floating-point ones)
+// instead of all sixteen warps queueing on the same pipe at the same time.
 // Results leave through shared memory: packed codes as a 128 x 64-byte tile written by a TMA
 // store (which also clips ragged edges), scales as one contiguous 512-byte tile.
 //
@@ -35,8 +38,8 @@ constexpr int kQScaleTileBytes = 512;
 
 struct QuantSmem {
     alignas(1024) uint8_t stage[kQStages][kQStageBytes];
-    alignas(1024) uint8_t code_tile[2][kQCodeTileBytes];
-    alignas(128) uint8_t scale_tile[2][kQScaleTileBytes];
+    alignas(1024) uint8_t code_tile[2][2][kQCodeTileBytes];    // [consumer group][double buffer]
+    alignas(128) uint8_t scale_tile[2][2][kQScaleTileBytes];
     alignas(8) uint64_t full[kQStages];
     uint64_t empty[kQStages];
     int abort_flag;
@@ -51,40 +54,13 @@ struct QuantParams {
     int32_t scale_layout;    // 0 canonical, 1 tiled
 };
 
-// Packed fp32 pairs: sm_100 adds, subtracts and multiplies two independent fp32 values held in
-// one 64-bit register with a single instruction (each lane is an ordinary IEEE fp32
-// round-to-nearest operation, so results are bit-identical to the scalar form).
-__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+// Packed fp32 pairs: sm_100 adds, multiplies and fuses two independent fp32 values held in a
+// float2 (an aligned register pair) with a single instruction; each lane is an ordinary IEEE
+// fp32 round-to-nearest operation, so results are bit-identical to the scalar form.  a - b is
+// formed as fma(b, -1, a): the product is exact, so there is still exactly one rounding.
+__device__ __forceinline__ float2 sub2(float2 a, float2 b)
 {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-
-__device__ __forceinline__ void unpack2(uint64_t p, float& lo, float& hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
-}
-
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-
-__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
+    return __ffma2_rn(b, make_float2(-1.0f, -1.0f), a);
 }
 
 // max(|a|, |b|, |c|) in one instruction.
@@ -96,23 +72,34 @@ __device__ __forceinline__ float max3_abs(float a, float b, float c)
 }
 
 // In-register 32-point Walsh-Hadamard transform of v[0..31] held as 16 pairs
-// P[i] = (v[2i], v[2i+1]).  Stage h = 1 was applied by the caller while forming the pairs
-// (its partners share a pair); stages h = 2, 4, 8, 16 pair whole registers, so each packed
-// add/sub does two butterflies.  Same five stages, same order, one fp32 rounding per output.
-__device__ __forceinline__ void fwht32_stages_2_to_16(uint64_t (&P)[16])
+// P[i] = (v[2i], v[2i+1]).  Stage h = 1 is applied while the pairs are formed (its partners
+// share a pair); stages h = 2, 4, 8, 16 pair whole registers, so each packed add/sub does two
+// butterflies.  Same five stages, same order, one fp32 rounding per output.
+template <int HP>
+__device__ __forceinline__ void fwht32_pair_stage(float2 (&P)[16])
 {
 #pragma unroll
-    for (int hp = 1; hp < 16; hp <<= 1) {
+    for (int i = 0; i < 16; i += 2 * HP) {
 #pragma unroll
-        for (int i = 0; i < 16; i += 2 * hp) {
-#pragma unroll
-            for (int j = i; j < i + hp; ++j) {
-                const uint64_t a = P[j], b = P[j + hp];
-                P[j] = add2(a, b);
-                P[j + hp] = sub2(a, b);
-            }
+        for (int j = i; j < i + HP; ++j) {
+            const float2 a = P[j], b = P[j + HP];
+            P[j] = __fadd2_rn(a, b);
+            P[j + HP] = sub2(a, b);
         }
     }
+}
+
+// Pair (element 2i, element 2i+1) of a block from the two fp32 bit patterns: optional sign
+// diagonal, then the h = 1 butterfly (the pair's halves are each other's partners).
+template <int HMODE>
+__device__ __forceinline__ float2 first_stage_pair(int i, uint32_t lo_bits, uint32_t hi_bits, uint32_t sign_mask)
+{
+    if (HMODE == 2) {
+        lo_bits ^= (sign_mask << (31 - 2 * i)) & 0x80000000u;
+        hi_bits ^= (sign_mask << (30 - 2 * i)) & 0x80000000u;
+    }
+    const float a = __uint_as_float(lo_bits), b = __uint_as_float(hi_bits);
+    return HMODE != 0 ? make_float2(__fadd_rn(a, b), __fsub_rn(a, b)) : make_float2(a, b);
 }
 
 // Eight E2M1 codes (one 32-bit word of packed output) from eight floats, round-to-nearest-even,
@@ -144,6 +131,87 @@ __device__ __forceinline__ uint32_t sr_e2m1(float s, uint32_t u8)
     return (r >> 22) | ((__float_as_uint(s) >> 28) & 8u);
 }
 
+// One 32-element block out of a shared-memory stage into registers as 16 pairs (sign diagonal
+// and first butterfly stage applied on the way in).
+template <int AXIS, int HMODE>
+__device__ __forceinline__ void load_block(const uint8_t* stage, int kb, int o, uint32_t sign_mask,
+                                           float2 (&P)[16])
+{
+    if (AXIS == 1) {
+        const uint8_t* base = stage + (kb >> 1) * (kQStageBytes / 2) + o * 128;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int chunk = (((kb & 1) * 4 + j) ^ (o & 7)) * 16;
+            const uint4 q = *reinterpret_cast<const uint4*>(base + chunk);
+            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                P[4 * j + i] = first_stage_pair<HMODE>(4 * j + i, w[i] * 65536u, w[i] & 0xFFFF0000u, sign_mask);
+        }
+    } else {
+        const uint16_t* base = reinterpret_cast<const uint16_t*>(stage) + (kb * 32) * 128 + o;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            P[i] = first_stage_pair<HMODE>(i, static_cast<uint32_t>(base[(2 * i) * 128]) * 65536u,
+                                           static_cast<uint32_t>(base[(2 * i + 1) * 128]) * 65536u, sign_mask);
+    }
+}
+
+// Remaining butterfly stages, block maximum, scale byte, rounding: block in, 16 bytes of packed
+// codes and the E8M0 byte out.  e0 = index of the block's first element in the operand view.
+template <int HMODE, int SR>
+__device__ __forceinline__ void quantize_block(float2 (&P)[16], uint64_t e0, const QuantParams& p,
+                                               uint32_t (&packed)[4], uint32_t& byte)
+{
+    if (HMODE != 0) {
+        fwht32_pair_stage<1>(P);
+        fwht32_pair_stage<2>(P);
+        fwht32_pair_stage<4>(P);
+        fwht32_pair_stage<8>(P);
+    }
+    float amax = max3_abs(P[0].x, P[0].y, P[1].x);
+#pragma unroll
+    for (int i = 1; i < 15; ++i) amax = max3_abs(amax, P[i].y, P[i + 1].x);
+    amax = fmaxf(amax, fabsf(P[15].y));
+    const uint32_t E = __float_as_uint(amax) >> 23;
+    byte = E > 2u ? E - 2u : 0u;                  // E <= 255 keeps byte <= 253 < 255
+    const float mult = __uint_as_float((254u - byte) << 23);
+    const float2 mult2 = make_float2(mult, mult);
+    float v[32];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float2 sp = __fmul2_rn(P[i], mult2);
+        v[2 * i] = sp.x;
+        v[2 * i + 1] = sp.y;
+    }
+    if (SR == 0) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            packed[q] = cvt_e2m1x8(v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4],
+                                   v[8 * q + 5], v[8 * q + 6], v[8 * q + 7]);
+    } else {
+        const uint64_t g = e0 >> 4;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            uint32_t r[4];
+            const uint64_t gg = g + half;
+            philox4x32_10(static_cast<uint32_t>(gg), static_cast<uint32_t>(gg >> 32), p.tag, 0u, p.seed_lo,
+                          p.seed_hi, r);
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                uint32_t w = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int e = q * 8 + i;                   // element in the 16-group
+                    const uint32_t u8 = (r[e >> 2] >> (8 * (e & 3))) & 0xFFu;
+                    w |= sr_e2m1(v[half * 16 + e], u8) << (4 * i);
+                }
+                packed[half * 2 + q] = w;
+            }
+        }
+    }
+}
+
 template <int AXIS, int HMODE, int SR>
 __global__ void __launch_bounds__(kQThreads, 1)
 quantize_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constant__ CUtensorMap tm_codes,
@@ -154,12 +222,13 @@ quantize_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constan
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int tid = threadIdx.x;
     const int total_tiles = p.tiles_o * p.tiles_k;
+    const int my_tiles = blockIdx.x < total_tiles ? (total_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
 
     if (tid == 0) {
         sm.abort_flag = 0;
         for (int s = 0; s < kQStages; ++s) {
             mbar_init(&sm.full[s], 1);
-            mbar_init(&sm.empty[s], kQConsumers / 32);
+            mbar_init(&sm.empty[s], kQConsumers / 64);      // the 8 warps of one consumer group
         }
         fence_barrier_init();
     }
@@ -169,8 +238,8 @@ quantize_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constan
         // ------------------------------------------------------------ producer warp
         if (tid == kQConsumers) {
             tma_prefetch_desc(&tm_src);
-            int it = 0;
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+            for (int it = 0; it < my_tiles; ++it) {
+                const int tile = blockIdx.x + it * gridDim.x;
                 const int s = it % kQStages;
                 const uint32_t round = it / kQStages;
                 if (round > 0 && !mbar_wait(&sm.empty[s], (round - 1) & 1, &sm.abort_flag)) break;
@@ -192,142 +261,81 @@ quantize_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constan
     }
 
     // ---------------------------------------------------------------- consumers
-    const int kb = tid >> 7;   // which of the tile's 4 blocks along K
-    const int o = tid & 127;   // operand row inside the tile
-    if (tid == 0) tma_prefetch_desc(&tm_codes);
+    const int grp = tid >> 8;          // consumer group: takes tiles grp, grp + 2, ...
+    const int t = tid & 255;
+    const int kbh = t >> 7;            // this thread's blocks along K: kbh and kbh + 2
+    const int o = t & 127;             // operand row inside the tile
+    if (t == 0) tma_prefetch_desc(&tm_codes);
 
-    int it = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+    int trip = 0;
+    for (int it = grp; it < my_tiles; it += 2, ++trip) {
+        const int tile = blockIdx.x + it * gridDim.x;
         const int s = it % kQStages;
         const uint32_t round = it / kQStages;
-        const int buf = it & 1;
+        const int buf = trip & 1;
         int to, tk;
         if (AXIS == 1) { to = tile / p.tiles_k; tk = tile % p.tiles_k; }
         else           { tk = tile / p.tiles_o; to = tile % p.tiles_o; }
 
         const bool ok = mbar_wait(&sm.full[s], round & 1, &sm.abort_flag);
 
-        // the block as 16 packed pairs P[i] = (v[2i], v[2i+1]); the sign diagonal and the first
-        // butterfly stage (whose partners are the two halves of a pair) are applied on the way in
-        uint64_t P[16];
-        auto make_pair = [&](int i, uint32_t lo_bits, uint32_t hi_bits) {
-            if (HMODE == 2) {
-                lo_bits ^= (p.sign_mask << (31 - 2 * i)) & 0x80000000u;
-                hi_bits ^= (p.sign_mask << (30 - 2 * i)) & 0x80000000u;
-            }
-            const float a = __uint_as_float(lo_bits), b = __uint_as_float(hi_bits);
-            P[i] = HMODE != 0 ? pack2(__fadd_rn(a, b), __fsub_rn(a, b)) : pack2(a, b);
-        };
+        float2 P0[16], P1[16];
         if (ok) {
-            if (AXIS == 1) {
-                const uint8_t* base = &sm.stage[s][(kb >> 1) * (kQStageBytes / 2) + o * 128];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int chunk = (((kb & 1) * 4 + j) ^ (o & 7)) * 16;
-                    const uint4 q = *reinterpret_cast<const uint4*>(base + chunk);
-                    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) make_pair(4 * j + i, w[i] * 65536u, w[i] & 0xFFFF0000u);
-                }
-            } else {
-                const uint16_t* base =
-                    reinterpret_cast<const uint16_t*>(&sm.stage[s][0]) + (kb * 32) * 128 + o;
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    make_pair(i, static_cast<uint32_t>(base[(2 * i) * 128]) * 65536u,
-                              static_cast<uint32_t>(base[(2 * i + 1) * 128]) * 65536u);
-            }
+            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.sign_mask, P0);
+            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.sign_mask, P1);
         } else {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) P[i] = 0ull;
+            for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
         }
         // the stage is in registers now: hand it back to the producer
         __syncwarp();
         if ((tid & 31) == 0) mbar_arrive(&sm.empty[s]);
 
-        if (HMODE != 0) fwht32_stages_2_to_16(P);
-
-        float v[32];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) unpack2(P[i], v[2 * i], v[2 * i + 1]);
-        float amax = max3_abs(v[0], v[1], v[2]);
-#pragma unroll
-        for (int j = 3; j < 31; j += 2) amax = max3_abs(amax, v[j], v[j + 1]);
-        amax = fmaxf(amax, fabsf(v[31]));
-        const uint32_t E = __float_as_uint(amax) >> 23;
-        const uint32_t byte = E > 2u ? E - 2u : 0u;   // E <= 255 keeps byte <= 253 < 255
-        const float mult = __uint_as_float((254u - byte) << 23);
-        const uint64_t mult2 = pack2(mult, mult);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const uint64_t sp = mul2(P[i], mult2);
-            unpack2(sp, v[2 * i], v[2 * i + 1]);       // v now holds the scaled values
-        }
-
-        uint32_t packed[4];
-        if (SR == 0) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                packed[q] = cvt_e2m1x8(v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4],
-                                       v[8 * q + 5], v[8 * q + 6], v[8 * q + 7]);
-        } else {
-            const uint64_t e0 = static_cast<uint64_t>(to * kQTileO + o) * static_cast<uint64_t>(p.K) +
-                                static_cast<uint64_t>((tk * 4 + kb) * 32);
-            const uint64_t g = e0 >> 4;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t r[4];
-                const uint64_t gg = g + half;
-                philox4x32_10(static_cast<uint32_t>(gg), static_cast<uint32_t>(gg >> 32), p.tag, 0u,
-                              p.seed_lo, p.seed_hi, r);
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    uint32_t w = 0;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int j = half * 16 + q * 8 + i;       // element in the block
-                        const int e = q * 8 + i;                   // element in the 16-group
-                        const uint32_t u8 = (r[e >> 2] >> (8 * (e & 3))) & 0xFFu;
-                        w |= sr_e2m1(v[j], u8) << (4 * i);
-                    }
-                    packed[half * 2 + q] = w;
-                }
-            }
-        }
+        const uint64_t e_row = static_cast<uint64_t>(to * kQTileO + o) * static_cast<uint64_t>(p.K);
+        uint32_t packed0[4], packed1[4], byte0, byte1;
+        quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tk * 4 + kbh) * 32), p, packed0, byte0);
+        quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tk * 4 + kbh + 2) * 32), p, packed1, byte1);
 
         // stage the results: codes in the 64-byte swizzle the TMA store expects
-        *reinterpret_cast<uint4*>(&sm.code_tile[buf][o * 64 + ((kb ^ ((o >> 1) & 3)) * 16)]) =
-            make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        uint8_t* ct = &sm.code_tile[grp][buf][o * 64];
+        *reinterpret_cast<uint4*>(ct + ((kbh ^ ((o >> 1) & 3)) * 16)) =
+            make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]);
+        *reinterpret_cast<uint4*>(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16)) =
+            make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]);
         if (p.scale_layout == 1) {
-            sm.scale_tile[buf][(o & 31) * 16 + (o >> 5) * 4 + kb] = static_cast<uint8_t>(byte);
-        } else {
+            uint8_t* st = &sm.scale_tile[grp][buf][(o & 31) * 16 + (o >> 5) * 4];
+            st[kbh] = static_cast<uint8_t>(byte0);
+            st[kbh + 2] = static_cast<uint8_t>(byte1);
+        } else if (ok) {
             const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
-            const int64_t tg = static_cast<int64_t>(tk) * 4 + kb;
-            if (ok && og < p.outer && tg < p.nt) p.scales[og * p.nt + tg] = static_cast<uint8_t>(byte);
+            const int64_t tg = static_cast<int64_t>(tk) * 4 + kbh;
+            if (og < p.outer && tg < p.nt) p.scales[og * p.nt + tg] = static_cast<uint8_t>(byte0);
+            if (og < p.outer && tg + 2 < p.nt) p.scales[og * p.nt + tg + 2] = static_cast<uint8_t>(byte1);
         }
         fence_proxy_async_smem();
-        // the store issued one tile ago must have drained its buffer before the next tile
-        // (which every thread reaches only through the barrier below) overwrites it
-        if (tid == 0) bulk_wait_group_read<0>();
+        // the store this group issued one trip ago must have drained its buffer before the next
+        // trip (which every thread of the group reaches only through the barrier below)
+        // overwrites it
+        if (t == 0) bulk_wait_group_read<0>();
         uint32_t any_fail;
         asm volatile(
             "{\n\t.reg .pred P, Q;\n\t"
             "setp.ne.u32 Q, %1, 0;\n\t"
-            "barrier.cta.red.or.pred P, 1, %2, Q;\n\t"
+            "barrier.cta.red.or.pred P, %2, %3, Q;\n\t"
             "selp.u32 %0, 1, 0, P;\n\t}"
             : "=r"(any_fail)
-            : "r"(ok ? 0u : 1u), "n"(kQConsumers)
+            : "r"(ok ? 0u : 1u), "r"(grp + 1), "n"(kQConsumers / 2)
             : "memory");
         if (any_fail) break;
-        if (tid == 0) {
-            tma_store_2d(&tm_codes, &sm.code_tile[buf][0], tk * (kQTileK / 2), to * kQTileO);
+        if (t == 0) {
+            tma_store_2d(&tm_codes, &sm.code_tile[grp][buf][0], tk * (kQTileK / 2), to * kQTileO);
             if (p.scale_layout == 1)
                 bulk_store_1d(p.scales + (static_cast<int64_t>(to) * p.tiles_k + tk) * kQScaleTileBytes,
-                              &sm.scale_tile[buf][0], kQScaleTileBytes);
+                              &sm.scale_tile[grp][buf][0], kQScaleTileBytes);
             bulk_commit_group();
         }
     }
-    if (tid == 0) bulk_wait_group<0>();
+    if (t == 0) bulk_wait_group<0>();
 }
 
 }  // namespace mxfp4
