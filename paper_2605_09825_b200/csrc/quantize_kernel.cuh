@@ -131,6 +131,18 @@ __device__ __forceinline__ uint32_t sr_e2m1(float s, uint32_t u8)
     return (r >> 22) | ((__float_as_uint(s) >> 28) & 8u);
 }
 
+// h = 1 butterfly of the deterministic rotation straight from bf16: (a + b, a - b) with a the
+// bf16 value in the low 16 bits of `a_bits` and b already widened to fp32.  The mixed-precision
+// add/sub widen a exactly, so the result equals the fp32 operation on the widened value.
+__device__ __forceinline__ float2 first_stage_pair_bf16(uint32_t a_bits, float b)
+{
+    float s, d;
+    const unsigned short a16 = static_cast<unsigned short>(a_bits);
+    asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(s) : "h"(a16), "f"(b));
+    asm("sub.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(a16), "f"(b));
+    return make_float2(s, d);
+}
+
 // One 32-element block out of a shared-memory stage into registers as 16 pairs (sign diagonal
 // and first butterfly stage applied on the way in).
 template <int AXIS, int HMODE>
@@ -146,14 +158,19 @@ __device__ __forceinline__ void load_block(const uint8_t* stage, int kb, int o, 
             const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                P[4 * j + i] = first_stage_pair<HMODE>(4 * j + i, w[i] * 65536u, w[i] & 0xFFFF0000u, sign_mask);
+                P[4 * j + i] = HMODE == 1
+                                   ? first_stage_pair_bf16(w[i], __uint_as_float(w[i] & 0xFFFF0000u))
+                                   : first_stage_pair<HMODE>(4 * j + i, w[i] * 65536u, w[i] & 0xFFFF0000u, sign_mask);
         }
     } else {
         const uint16_t* base = reinterpret_cast<const uint16_t*>(stage) + (kb * 32) * 128 + o;
 #pragma unroll
         for (int i = 0; i < 16; ++i)
-            P[i] = first_stage_pair<HMODE>(i, static_cast<uint32_t>(base[(2 * i) * 128]) * 65536u,
-                                           static_cast<uint32_t>(base[(2 * i + 1) * 128]) * 65536u, sign_mask);
+            P[i] = HMODE == 1
+                       ? first_stage_pair_bf16(base[(2 * i) * 128],
+                                               __uint_as_float(static_cast<uint32_t>(base[(2 * i + 1) * 128]) * 65536u))
+                       : first_stage_pair<HMODE>(i, static_cast<uint32_t>(base[(2 * i) * 128]) * 65536u,
+                                                 static_cast<uint32_t>(base[(2 * i + 1) * 128]) * 65536u, sign_mask);
     }
 }
 
