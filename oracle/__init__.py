@@ -24,7 +24,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "mxfp4_oracle.c")
 _LIB = os.path.join(_HERE, "libmxfp4_oracle.so")
 
-HADAMARD_NONE, HADAMARD_DET, HADAMARD_RAND = 0, 1, 2
+HADAMARD_NONE, HADAMARD_DET, HADAMARD_RAND, HADAMARD_DET16, HADAMARD_RAND16 = 0, 1, 2, 3, 4
 ROUND_RNE, ROUND_SR = 0, 1
 
 
@@ -55,6 +55,8 @@ def _load():
     lib.oracle_sign_mask.restype = ctypes.c_uint32
     lib.oracle_fwht32.argtypes = [ctypes.POINTER(ctypes.c_float)]
     lib.oracle_fwht32.restype = None
+    lib.oracle_fwht16x2.argtypes = [ctypes.POINTER(ctypes.c_float)]
+    lib.oracle_fwht16x2.restype = None
     lib.oracle_quantize.argtypes = [ctypes.POINTER(ctypes.c_uint16), i64, i64, i64, ctypes.c_int,
                                     ctypes.c_int, ctypes.c_int, ctypes.c_uint64, ctypes.c_uint32,
                                     u8p, u8p]
@@ -102,6 +104,14 @@ def fwht32(v) -> np.ndarray:
     a = np.ascontiguousarray(v, dtype=np.float32).copy()
     assert a.shape == (32,)
     _load().oracle_fwht32(_ptr(a, ctypes.c_float))
+    return a
+
+
+def fwht16x2(v) -> np.ndarray:
+    """Two unnormalised 16-point Walsh-Hadamard transforms, one per half of a 32-vector."""
+    a = np.ascontiguousarray(v, dtype=np.float32).copy()
+    assert a.shape == (32,)
+    _load().oracle_fwht16x2(_ptr(a, ctypes.c_float))
     return a
 
 
@@ -208,8 +218,8 @@ def gemm(a_codes, a_scales, b_codes, b_scales, alpha: float = 1.0, rows=None):
 
 
 def _alpha(hadamard_mode: int) -> float:
-    # H H^T = 32 I for the +-1 matrix: the product of two rotated operands carries a factor 32
-    return 1.0 / 32.0 if hadamard_mode != 0 else 1.0
+    # H H^T = n I for the +-1 matrix of order n: the product of two rotated operands carries n
+    return {0: 1.0, 1: 1.0 / 32.0, 2: 1.0 / 32.0, 3: 1.0 / 16.0, 4: 1.0 / 16.0}[hadamard_mode]
 
 
 def linear_fprop(X, W, hadamard_mode=1, rounding=0, seed=0, rows=None):

@@ -25,6 +25,9 @@
  *     fp32 butterfly (h = 1,2,4,8,16); the 1/32 is an exact factor on the GEMM.
  *   - random sign flips: one 32-bit mask per seed, shared by every tile and by
  *     both operands (so D*D = I cancels in the product).
+ *   - the 16-point variant (the paper's final choice, Appendix A.2) rotates each half of an
+ *     MX block with its own 16-point transform (stages h = 1,2,4,8); its randomized form
+ *     uses the low 16 bits of the same mask for both halves; the exact factor is 1/16.
  *   - stochastic rounding: 8 random bits per element from Philox4x32-10 keyed by
  *     the seed and counted by the element index in the operand view.
  *     PARITY UNPINNED against the paper for the stochastic-rounding bit pattern:
@@ -86,6 +89,22 @@ uint32_t oracle_sign_mask(uint64_t seed)
 void oracle_fwht32(float v[MX_BLOCK])
 {
     for (int h = 1; h < MX_BLOCK; h *= 2) {
+        for (int i = 0; i < MX_BLOCK; i += 2 * h) {
+            for (int j = i; j < i + h; ++j) {
+                float a = v[j];
+                float b = v[j + h];
+                v[j] = a + b;
+                v[j + h] = a - b;
+            }
+        }
+    }
+}
+
+/* Two independent 16-point transforms, one per half of the 32-tile (Appendix A.2: H16 in a
+ * tiled layout): the first four stages of the 32-point butterfly. */
+void oracle_fwht16x2(float v[MX_BLOCK])
+{
+    for (int h = 1; h < 16; h *= 2) {
         for (int i = 0; i < MX_BLOCK; i += 2 * h) {
             for (int j = i; j < i + h; ++j) {
                 float a = v[j];
@@ -189,7 +208,8 @@ static uint8_t quantize_tile(const float v[MX_BLOCK], int rounding, uint64_t e0,
  *             the output is the transposed operand, Appendix C Dgrad/Wgrad)
  * codes  : [outer x K/2] bytes, element k even in bits 3:0, odd in bits 7:4
  * scales : [outer x K/32] bytes, canonical row-major
- * hadamard_mode: 0 none, 1 deterministic H32, 2 randomized H32 (sign mask from seed)
+ * hadamard_mode: 0 none, 1 deterministic H32, 2 randomized H32 (sign mask from seed),
+ *                3 deterministic H16 (per half-block), 4 randomized H16
  * rounding     : 0 round-to-nearest-even, 1 stochastic
  * Returns 0, or -1 on a bad argument.
  */
@@ -199,11 +219,16 @@ int oracle_quantize(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld,
 {
     if (!src || !codes || !scales) return -1;
     if (axis != 0 && axis != 1) return -1;
-    if (hadamard_mode < 0 || hadamard_mode > 2 || rounding < 0 || rounding > 1) return -1;
+    if (hadamard_mode < 0 || hadamard_mode > 4 || rounding < 0 || rounding > 1) return -1;
     int64_t outer = axis ? rows : cols;
     int64_t K = axis ? cols : rows;
     if (outer <= 0 || K <= 0 || K % MX_BLOCK != 0 || ld < cols) return -1;
-    const uint32_t mask = (hadamard_mode == 2) ? oracle_sign_mask(seed) : 0u;
+    uint32_t mask = 0u;
+    if (hadamard_mode == 2) mask = oracle_sign_mask(seed);
+    if (hadamard_mode == 4) {
+        uint32_t m16 = oracle_sign_mask(seed) & 0xFFFFu;   /* same 16 signs for both halves */
+        mask = m16 | (m16 << 16);
+    }
     const int64_t nt = K / MX_BLOCK;
 
 #pragma omp parallel for schedule(static)
@@ -216,11 +241,12 @@ int oracle_quantize(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld,
                 uint16_t b = axis ? src[o * ld + k] : src[k * ld + o];
                 v[j] = bf16_bits_to_float(b);
             }
-            if (hadamard_mode == 2) {
+            if (hadamard_mode == 2 || hadamard_mode == 4) {
                 for (int j = 0; j < MX_BLOCK; ++j)
                     if ((mask >> j) & 1u) v[j] = -v[j];
             }
-            if (hadamard_mode != 0) oracle_fwht32(v);
+            if (hadamard_mode == 1 || hadamard_mode == 2) oracle_fwht32(v);
+            if (hadamard_mode == 3 || hadamard_mode == 4) oracle_fwht16x2(v);
             uint64_t e0 = (uint64_t)o * (uint64_t)K + (uint64_t)(t * MX_BLOCK);
             uint8_t byte = quantize_tile(v, rounding, e0, seed, tag, code);
             scales[o * nt + t] = byte;

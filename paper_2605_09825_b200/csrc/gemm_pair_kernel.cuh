@@ -440,12 +440,14 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     const int64_t total = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
     if (total > 0x3FFFFFFF) return MXFP4_ERR_SHAPE;
     const size_t smem = sizeof(GemmPairSmem) + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};          // the attribute is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
+    if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(gemm_mxf4_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess)
             return MXFP4_ERR_CUDA;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     const int max_clusters = sm_count / 2;
     const int clusters = static_cast<int>(total < max_clusters ? total : max_clusters);

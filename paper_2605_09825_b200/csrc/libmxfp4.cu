@@ -62,13 +62,15 @@ static int launch_quantize(const CUtensorMap& tm_src, const CUtensorMap& tm_code
                            const QuantParams& p, int grid, cudaStream_t stream)
 {
     const size_t smem = sizeof(QuantSmem) + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};          // the attribute is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
+    if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(quantize_kernel<AXIS, HMODE, SR>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess)
             return MXFP4_ERR_CUDA;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     quantize_kernel<AXIS, HMODE, SR><<<grid, kQThreads, smem, stream>>>(tm_src, tm_codes, p);
     return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;

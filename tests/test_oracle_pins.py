@@ -266,6 +266,48 @@ def test_worked_tiles():
     assert quant_tile(outlier, hadamard_mode=1) == (w["outlier_h32"][1], w["outlier_h32"][0])
 
 
+def test_worked_tiles_16_point_variant():
+    w = _worked()
+    ramp = [j - 15.5 for j in range(32)]
+    outlier = [1.0] * 32
+    outlier[5] = 50.0
+    assert quant_tile(ramp, hadamard_mode=3) == (w["ramp_h16"][1], w["ramp_h16"][0])
+    assert quant_tile(outlier, hadamard_mode=3) == (w["outlier_h16"][1], w["outlier_h16"][0])
+
+
+def test_fwht16_matches_the_sylvester_matrix_per_half():
+    H = scipy.linalg.hadamard(16).astype(np.float64)
+    rng = np.random.default_rng(15)
+    for _ in range(20):
+        v = rng.integers(-64, 64, 32).astype(np.float32)
+        hv = oracle.fwht16x2(v)
+        assert (hv[:16] == H @ v[:16]).all() and (hv[16:] == H @ v[16:]).all()
+        assert (oracle.fwht16x2(hv) == 16 * v).all()
+    a = rng.integers(-32, 32, 32).astype(np.float32)
+    b = rng.integers(-32, 32, 32).astype(np.float32)
+    assert float(oracle.fwht16x2(a) @ oracle.fwht16x2(b)) == 16 * float(a @ b)
+    # the 16-point butterfly is the first four stages of the 32-point one: bits must agree
+    # with a numpy strided-stage formulation on values that do not add exactly
+    for _ in range(20):
+        v = (rng.standard_normal(32) * np.exp2(rng.integers(-20, 20, 32))).astype(np.float32)
+        w = v.copy()
+        for h in (1, 2, 4, 8):
+            w = w.reshape(-1, 2, h)
+            w = np.stack([w[:, 0, :] + w[:, 1, :], w[:, 0, :] - w[:, 1, :]], axis=1).reshape(32)
+        assert (oracle.fwht16x2(v).view(np.uint32) == w.view(np.uint32)).all()
+
+
+def test_randomized_16_point_is_sign_flip_then_rotation():
+    rng = np.random.default_rng(18)
+    src = _random_bits(rng, 16, 128)
+    for seed in (0, 7):
+        m = oracle.sign_mask(seed) & 0xFFFF
+        flip = np.array([0x8000 if (m >> (j % 16)) & 1 else 0 for j in range(128)], dtype=np.uint16)
+        a = oracle.quantize(src, 1, hadamard_mode=4, seed=seed)
+        b = oracle.quantize(src ^ flip[None, :], 1, hadamard_mode=3)
+        assert (a[0] == b[0]).all() and (a[1] == b[1]).all()
+
+
 def test_rotation_disperses_the_outlier():
     outlier = np.ones(32)
     outlier[5] = 50.0
@@ -434,7 +476,7 @@ def test_linear_passes_follow_the_cancellation_identities():
     tob = lambda x: ((x.view(np.uint32) + 0x7FFF + ((x.view(np.uint32) >> 16) & 1)) >> 16).astype(np.uint16)
     tof = lambda b: (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
     Xb, Wb, dYb = tob(X), tob(W), tob(dY)
-    for mode in (0, 1, 2):
+    for mode in (0, 1, 2, 3, 4):
         y, _ = oracle.linear_fprop(Xb, Wb, hadamard_mode=mode, seed=7)
         dx, _ = oracle.linear_dgrad(dYb, Wb, hadamard_mode=mode, seed=7)
         dw, _ = oracle.linear_wgrad(dYb, Xb, hadamard_mode=mode, seed=7)
@@ -449,7 +491,7 @@ def test_linear_passes_follow_the_cancellation_identities():
 def test_axis0_equals_axis1_on_the_transposed_source():
     rng = np.random.default_rng(31)
     src = _random_bits(rng, 96, 80)        # K = rows = 96 for axis 0
-    for mode, rnd in ((0, 0), (1, 0), (2, 0), (0, 1), (1, 1)):
+    for mode, rnd in ((0, 0), (1, 0), (2, 0), (0, 1), (1, 1), (3, 0), (4, 1)):
         a = oracle.quantize(src, 0, mode, rnd, seed=7, tag=1)
         b = oracle.quantize(np.ascontiguousarray(src.T), 1, mode, rnd, seed=7, tag=1)
         assert a[0].shape == (80, 48) and a[1].shape == (80, 3)
@@ -482,4 +524,4 @@ def test_bad_arguments_are_rejected():
     with pytest.raises(ValueError):
         oracle.quantize(src, 1)
     with pytest.raises(ValueError):
-        oracle.quantize(np.zeros((4, 64), dtype=np.uint16), 1, hadamard_mode=3)
+        oracle.quantize(np.zeros((4, 64), dtype=np.uint16), 1, hadamard_mode=5)
