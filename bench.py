@@ -46,11 +46,16 @@ WORKLOADS = {
 }
 
 
-def workload_label(name: str, tokens: int) -> str:
+HADAMARD = {"none": (0, "no rotation"), "h32": (1, "deterministic H32"), "rh32": (2, "randomized H32"),
+            "h16": (3, "deterministic H16"), "rh16": (4, "randomized H16")}
+
+
+def workload_label(name: str, tokens: int, hadamard: str = "h32") -> str:
+    rot = HADAMARD[hadamard][1]
     if name == "layer_stack":
         return ("Llama-3.1-8B layer linear stack (QKV, O, gate+up, down) x (Fprop, Dgrad, Wgrad), "
-                f"{tokens} tokens, deterministic H32, RNE")
-    return f"Llama-3.1-8B {name} linear x (Fprop, Dgrad, Wgrad), {tokens} tokens, deterministic H32, RNE"
+                f"{tokens} tokens, {rot}, RNE")
+    return f"Llama-3.1-8B {name} linear x (Fprop, Dgrad, Wgrad), {tokens} tokens, {rot}, RNE"
 
 
 def pass_dims(pass_: int, T: int, in_f: int, out_f: int):
@@ -182,7 +187,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT,
         "n_gpus": args.gpus, "steps": steps, "warmup": warm, "ms_per_step": mean * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "e2m1 x e2m1 -> f64",
-        "data": "synthetic", "config": {"workload": workload_label(args.workload, tokens),
+        "data": "synthetic", "config": {"workload": workload_label(args.workload, tokens, args.hadamard),
                                         "note": "CPU oracle on a bounded sample of this workload"},
         "cpu_baseline": base,
         "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -208,7 +213,8 @@ def run_ours(args):
     api.load_library()
     peaks = load_peaks()
     tokens, names = WORKLOADS[args.workload]
-    hmode, rnd, seed = api.HADAMARD_DET, api.ROUND_RNE, 0
+    hmode, rnd, seed = HADAMARD[args.hadamard][0], api.ROUND_RNE, 0
+    alpha = {0: 1.0, 1: 1.0 / 32, 2: 1.0 / 32, 3: 1.0 / 16, 4: 1.0 / 16}[hmode]
 
     # ---- inputs: seeded synthetic, generated on the host, then resident in HBM
     host, dev_in = {}, {}
@@ -291,7 +297,7 @@ def run_ours(args):
             ev[1].record(stream)
             api.quantize(b, ax_b, hmode, rnd, seed, 1, codes=bc, scales=b_s)
             ev[2].record(stream)
-            api.gemm(ac, a_s, bc, b_s, 1.0 / 32, api.OUT_BF16, out=out_buf[: M * N].view(M, N))
+            api.gemm(ac, a_s, bc, b_s, alpha, api.OUT_BF16, out=out_buf[: M * N].view(M, N))
             ev[3].record(stream)
             evs.append((ev, M, N, K))
         torch.cuda.synchronize()
@@ -403,7 +409,7 @@ def run_ours(args):
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "e2m1 (mxfp4) x e2m1, f32 accumulate",
         "data": "synthetic",
-        "config": {"workload": workload_label(args.workload, tokens), "passes_per_step": len(passes),
+        "config": {"workload": workload_label(args.workload, tokens, args.hadamard), "passes_per_step": len(passes),
                    "flops_per_step": flops_per_step, "out_dtype": "bf16",
                    "l2": "inputs larger than L2 (several GB per step), no flush needed",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
@@ -422,6 +428,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="layer_stack", choices=sorted(WORKLOADS))
+    ap.add_argument("--hadamard", default="h32", choices=sorted(HADAMARD))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-context", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -50,6 +50,8 @@ extern "C" {
 #define MXFP4_HADAMARD_NONE 0
 #define MXFP4_HADAMARD_DET 1  /* deterministic 32-point rotation                              */
 #define MXFP4_HADAMARD_RAND 2 /* sign diagonal from `seed`, then the rotation                 */
+#define MXFP4_HADAMARD_DET16 3  /* two 16-point rotations per 32-block (the paper's H16)      */
+#define MXFP4_HADAMARD_RAND16 4 /* 16 signs from `seed` (same for both halves), then H16      */
 
 #define MXFP4_ROUND_RNE 0 /* round to nearest, ties to even                                   */
 #define MXFP4_ROUND_SR 1  /* stochastic rounding, Philox4x32-10 keyed by (seed, element)      */
@@ -94,7 +96,8 @@ size_t mxfp4_scales_bytes(int64_t outer, int64_t K, int scale_layout);
  *   K must be a multiple of 32.  For MXFP4_AXIS_ROWS, cols must be a multiple of 8.
  *   hadamard_mode, rounding, seed: each 32-block v becomes H*v (mode 1) or H*(D*v) (mode 2,
  *                D the +-1 diagonal drawn from `seed`) in fp32 with a fixed five-stage
- *                butterfly; the block scale is 2^(floor(log2 amax) - 2); elements are rounded
+ *                butterfly; modes 3 / 4 rotate each half of the block with its own 16-point
+ *                transform instead (the same butterfly without its last stage); the block scale is 2^(floor(log2 amax) - 2); elements are rounded
  *                to E2M1 with saturation at 6.  With MXFP4_ROUND_SR each element uses 8 bits
  *                of Philox4x32-10(key = seed, counter = (e>>4, 0, operand_tag, 0)), e the
  *                element's index o*K + k in the operand view.
@@ -133,7 +136,7 @@ size_t mxfp4_linear_workspace_bytes(int64_t T, int64_t in_features, int64_t out_
  * Fused linear passes (Appendix C).  Each quantizes its two operands along the reduction
  * axis (same hadamard_mode / rounding / seed for both so that the rotation cancels;
  * operand_tag 0 for the first operand, 1 for the second) and runs the GEMM with
- * alpha = 2^-5 when rotated, 1 otherwise.  All matrices row-major and dense (ld = width).
+ * alpha = 2^-5 when rotated with H32, 2^-4 with H16, 1 otherwise.  All matrices row-major and dense (ld = width).
  *   fprop: Y[T x out]   = X[T x in]    * W[out x in]^T   (both row-wise along `in`)
  *   dgrad: dX[T x in]   = dY[T x out]  * W[out x in]     (dY row-wise along `out`; W column-wise)
  *   wgrad: dW[out x in] = dY[T x out]^T * X[T x in]      (both column-wise along tokens)

@@ -13,7 +13,7 @@ import torch
 
 from . import build as _build
 
-HADAMARD_NONE, HADAMARD_DET, HADAMARD_RAND = 0, 1, 2
+HADAMARD_NONE, HADAMARD_DET, HADAMARD_RAND, HADAMARD_DET16, HADAMARD_RAND16 = 0, 1, 2, 3, 4
 ROUND_RNE, ROUND_SR = 0, 1
 SCALES_CANONICAL, SCALES_TILED = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1

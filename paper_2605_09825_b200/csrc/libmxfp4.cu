@@ -86,7 +86,11 @@ static int dispatch_quantize(int hmode, int sr, const CUtensorMap& a, const CUte
         case 2: return launch_quantize<AXIS, 1, 0>(a, b, p, grid, st);
         case 3: return launch_quantize<AXIS, 1, 1>(a, b, p, grid, st);
         case 4: return launch_quantize<AXIS, 2, 0>(a, b, p, grid, st);
-        default: return launch_quantize<AXIS, 2, 1>(a, b, p, grid, st);
+        case 5: return launch_quantize<AXIS, 2, 1>(a, b, p, grid, st);
+        case 6: return launch_quantize<AXIS, 3, 0>(a, b, p, grid, st);
+        case 7: return launch_quantize<AXIS, 3, 1>(a, b, p, grid, st);
+        case 8: return launch_quantize<AXIS, 4, 0>(a, b, p, grid, st);
+        default: return launch_quantize<AXIS, 4, 1>(a, b, p, grid, st);
     }
 }
 
@@ -139,7 +143,7 @@ int mxfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_
 {
     if (!src_bf16 || !codes || !scales) return MXFP4_ERR_NULL;
     if (axis != 0 && axis != 1) return MXFP4_ERR_ENUM;
-    if (hadamard_mode < 0 || hadamard_mode > 2 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
+    if (hadamard_mode < 0 || hadamard_mode > 4 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
     if (scale_layout != 0 && scale_layout != 1) return MXFP4_ERR_ENUM;
     if (rows <= 0 || cols <= 0 || ld_src < cols) return MXFP4_ERR_SHAPE;
     const int64_t outer = axis ? rows : cols;
@@ -172,7 +176,12 @@ int mxfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_
     p.seed_lo = static_cast<uint32_t>(seed);
     p.seed_hi = static_cast<uint32_t>(seed >> 32);
     p.tag = operand_tag;
-    p.sign_mask = hadamard_mode == MXFP4_HADAMARD_RAND ? host_sign_mask(seed) : 0u;
+    p.sign_mask = 0u;
+    if (hadamard_mode == MXFP4_HADAMARD_RAND) p.sign_mask = host_sign_mask(seed);
+    if (hadamard_mode == MXFP4_HADAMARD_RAND16) {
+        const uint32_t m16 = host_sign_mask(seed) & 0xFFFFu;   // same 16 signs for both halves
+        p.sign_mask = m16 | (m16 << 16);
+    }
     p.scale_layout = scale_layout;
     const int64_t total = static_cast<int64_t>(p.tiles_o) * p.tiles_k;
     if (total > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
@@ -231,7 +240,7 @@ static int linear_pass(int pass, const void* a_src, const void* b_src, void* out
 {
     if (!a_src || !b_src || !out) return MXFP4_ERR_NULL;
     if (T <= 0 || in_f <= 0 || out_f <= 0) return MXFP4_ERR_SHAPE;
-    if (hmode < 0 || hmode > 2 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
+    if (hmode < 0 || hmode > 4 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
     int64_t M, N, K;
     linear_dims(pass, T, in_f, out_f, &M, &N, &K);
     if (K % 32 != 0 || in_f % 8 != 0 || out_f % 8 != 0) return MXFP4_ERR_SHAPE;
@@ -260,7 +269,8 @@ static int linear_pass(int pass, const void* a_src, const void* b_src, void* out
     rc = mxfp4_quantize(b_src, br, bc, bc, b_axis, hmode, rounding, seed, 1u, b_codes, b_scales,
                         MXFP4_SCALES_TILED, stream);
     if (rc != MXFP4_OK) return rc;
-    const float alpha = hmode != MXFP4_HADAMARD_NONE ? 0.03125f : 1.0f;
+    // H * H^T = n * I for the +-1 matrix of order n: undo it exactly in the epilogue
+    const float alpha = hmode == MXFP4_HADAMARD_NONE ? 1.0f : (hmode <= MXFP4_HADAMARD_RAND ? 0.03125f : 0.0625f);
     return mxfp4_gemm(a_codes, a_scales, b_codes, b_scales, M, N, K, alpha, out, out_dtype, N,
                       nullptr, 0, stream);
 }

@@ -71,6 +71,10 @@ __device__ __forceinline__ float max3_abs(float a, float b, float c)
     return r;
 }
 
+// HMODE: 0 none | 1 deterministic H32 | 2 randomized H32 | 3 deterministic H16 | 4 randomized
+// H16 (two independent 16-point transforms per MX block = the 32-point butterfly without its
+// last stage; the randomized form repeats the low 16 sign bits for the second half).
+//
 // In-register 32-point Walsh-Hadamard transform of v[0..31] held as 16 pairs
 // P[i] = (v[2i], v[2i+1]).  Stage h = 1 is applied while the pairs are formed (its partners
 // share a pair); stages h = 2, 4, 8, 16 pair whole registers, so each packed add/sub does two
@@ -94,7 +98,7 @@ __device__ __forceinline__ void fwht32_pair_stage(float2 (&P)[16])
 template <int HMODE>
 __device__ __forceinline__ float2 first_stage_pair(int i, uint32_t lo_bits, uint32_t hi_bits, uint32_t sign_mask)
 {
-    if (HMODE == 2) {
+    if (HMODE == 2 || HMODE == 4) {
         lo_bits ^= (sign_mask << (31 - 2 * i)) & 0x80000000u;
         hi_bits ^= (sign_mask << (30 - 2 * i)) & 0x80000000u;
     }
@@ -158,7 +162,7 @@ __device__ __forceinline__ void load_block(const uint8_t* stage, int kb, int o, 
             const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                P[4 * j + i] = HMODE == 1
+                P[4 * j + i] = (HMODE == 1 || HMODE == 3)
                                    ? first_stage_pair_bf16(w[i], __uint_as_float(w[i] & 0xFFFF0000u))
                                    : first_stage_pair<HMODE>(4 * j + i, w[i] * 65536u, w[i] & 0xFFFF0000u, sign_mask);
         }
@@ -166,7 +170,7 @@ __device__ __forceinline__ void load_block(const uint8_t* stage, int kb, int o, 
         const uint16_t* base = reinterpret_cast<const uint16_t*>(stage) + (kb * 32) * 128 + o;
 #pragma unroll
         for (int i = 0; i < 16; ++i)
-            P[i] = HMODE == 1
+            P[i] = (HMODE == 1 || HMODE == 3)
                        ? first_stage_pair_bf16(base[(2 * i) * 128],
                                                __uint_as_float(static_cast<uint32_t>(base[(2 * i + 1) * 128]) * 65536u))
                        : first_stage_pair<HMODE>(i, static_cast<uint32_t>(base[(2 * i) * 128]) * 65536u,
@@ -184,7 +188,7 @@ __device__ __forceinline__ void quantize_block(float2 (&P)[16], uint64_t e0, con
         fwht32_pair_stage<1>(P);
         fwht32_pair_stage<2>(P);
         fwht32_pair_stage<4>(P);
-        fwht32_pair_stage<8>(P);
+        if (HMODE <= 2) fwht32_pair_stage<8>(P);   // the 16-point variant stops after h = 8
     }
     float amax = max3_abs(P[0].x, P[0].y, P[1].x);
 #pragma unroll

@@ -57,7 +57,7 @@ def test_argument_errors_come_back_as_status_codes(lib):
     q = lib.mxfp4_quantize
     assert q(None, 32, 32, 32, 1, 0, 0, 0, 0, p, p, 0, None) == -1            # NULL
     assert q(p, 32, 32, 32, 2, 0, 0, 0, 0, p, p, 0, None) == -4               # axis
-    assert q(p, 32, 32, 32, 1, 3, 0, 0, 0, p, p, 0, None) == -4               # hadamard mode
+    assert q(p, 32, 32, 32, 1, 5, 0, 0, 0, p, p, 0, None) == -4               # hadamard mode
     assert q(p, 32, 32, 32, 1, 0, 2, 0, 0, p, p, 0, None) == -4               # rounding
     assert q(p, 32, 32, 32, 1, 0, 0, 0, 0, p, p, 9, None) == -4               # layout
     assert q(p, 32, 48, 48, 1, 0, 0, 0, 0, p, p, 0, None) == -2               # K % 32

@@ -55,7 +55,7 @@ def test_config3_gate_up_fprop_and_dgrad():
     _check_quant(t["W"], 0, 1, 0, 0, 1)         # W^T for Dgrad, column-wise
 
 
-@pytest.mark.parametrize("hmode,rnd", [(1, 0), (2, 0), (0, 1)])
+@pytest.mark.parametrize("hmode,rnd", [(1, 0), (2, 0), (0, 1), (3, 0)])
 def test_config4_down_wgrad_variants(hmode, rnd):
     t = synth.config4()
     _check_pass(2, t["dY"], t["X"], hmode, rnd, 7, f"config 4 wgrad mode {hmode} rounding {rnd}")

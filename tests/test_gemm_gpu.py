@@ -109,14 +109,14 @@ def test_gemm_is_deterministic_and_respects_ld_out():
 def test_config1_fprop_full_output():
     t = synth.config1()
     X, W = to_dev(t["X"]), to_dev(t["W"])
-    for hmode in (0, 1, 2):
+    for hmode in (0, 1, 2, 3, 4):
         y = api.linear_fprop(X, W, hmode, 0, 7, api.OUT_FP32)
         api.check()
         ref, S = oracle.linear_fprop(t["X"], t["W"], hmode, 0, 7)
         assert_gemm_close(y.cpu().numpy(), ref, S, False, f"config 1 fprop mode {hmode}")
 
 
-@pytest.mark.parametrize("hmode,rnd", [(0, 0), (1, 0), (2, 0), (0, 1)])
+@pytest.mark.parametrize("hmode,rnd", [(0, 0), (1, 0), (2, 0), (0, 1), (3, 0), (4, 1)])
 def test_three_passes_small_layer(hmode, rnd):
     rng = np.random.default_rng(40 + hmode)
     T, IN, OUT = 384, 512, 320

@@ -9,7 +9,7 @@ from paper_2605_09825_b200 import api, synth
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [(0, 0), (1, 0), (2, 0), (0, 1), (1, 1), (2, 1)]   # (hadamard_mode, rounding)
+VARIANTS = [(0, 0), (1, 0), (2, 0), (0, 1), (1, 1), (2, 1), (3, 0), (4, 0), (3, 1), (4, 1)]   # (hadamard_mode, rounding)
 
 
 def _check(bits, axis, hmode, rnd, seed=7, tag=1, layout=api.SCALES_TILED):
@@ -86,7 +86,7 @@ def test_every_bf16_pattern_and_special_blocks():
     bits = np.zeros((len(pats) + 2, 32), dtype=np.uint16)
     bits[np.arange(len(pats)), pats % 32] = pats
     bits[-1, :] = 0x8000
-    for hmode in (0, 1):
+    for hmode in (0, 1, 3):
         _check(bits, 1, hmode, 0)
         _check(bits, 1, hmode, 1)
 
