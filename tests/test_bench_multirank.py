@@ -1,6 +1,7 @@
 """Host-side logic of the N > 1 benchmark path: ranks are independent replicas; the reported time
 is the max over ranks.  Runs two gloo ranks on CPU."""
 import os
+import socket
 import subprocess
 import sys
 import textwrap
@@ -28,9 +29,12 @@ def test_max_over_ranks_with_two_gloo_ranks(tmp_path):
     script = tmp_path / "worker.py"
     script.write_text(WORKER)
     env = dict(os.environ, MASTER_ADDR="127.0.0.1")
+    with socket.socket() as sock:                       # a port nobody is using right now
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
     res = subprocess.run(
         [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
-         "--master-addr", "127.0.0.1", "--master-port", "29541", str(script)],
+         "--master-addr", "127.0.0.1", "--master-port", str(port), str(script)],
         capture_output=True, text=True, timeout=240, env=env)
     assert res.returncode == 0, res.stdout + res.stderr
     assert "rank 0 ok" in res.stdout and "rank 1 ok" in res.stdout
