@@ -205,6 +205,14 @@ int mxfp4_linear_static(int pass, const void* a, const void* b, void* out, int64
  */
 int mxfp4_check(void* stream);
 
+/*
+ * Self-test of the error path (no counterpart in the paper): enqueues a one-warp kernel whose
+ * only wait can never be satisfied and is limited to a few hundred attempts.  The kernel gives
+ * up within microseconds, records the time-out and returns normally -- nothing traps, faults
+ * or hangs -- so the next mxfp4_check(stream) returns MXFP4_ERR_TIMEOUT (and clears it).
+ */
+int mxfp4_selftest_wait_timeout(void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,7 @@ EXPORTS = (
     "mxfp4_version", "mxfp4_status_string", "mxfp4_codes_bytes", "mxfp4_scales_bytes",
     "mxfp4_quantize", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
     "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_host", "mxfp4_linear_static",
-    "mxfp4_check",
+    "mxfp4_check", "mxfp4_selftest_wait_timeout",
 )
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
@@ -76,6 +76,7 @@ def load_library() -> ctypes.CDLL:
     lib.mxfp4_linear_static.argtypes = [ci, vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp]
     lib.mxfp4_linear_static.restype = ci
     lib.mxfp4_check.argtypes, lib.mxfp4_check.restype = [vp], ci
+    lib.mxfp4_selftest_wait_timeout.argtypes, lib.mxfp4_selftest_wait_timeout.restype = [vp], ci
     _lib = lib
     return lib
 
@@ -244,6 +245,11 @@ def linear_static(pass_: int, a: torch.Tensor, b: torch.Tensor, T: int, in_f: in
                                             _stream())
     _raise(rc, "mxfp4_linear_static")
     return out
+
+
+def selftest_wait_timeout() -> None:
+    """Enqueue the bounded-wait self-test; the next :func:`check` raises with status -7."""
+    _raise(load_library().mxfp4_selftest_wait_timeout(_stream()), "mxfp4_selftest_wait_timeout")
 
 
 def check() -> None:

@@ -96,6 +96,22 @@ static int dispatch_quantize(int hmode, int sr, const CUtensorMap& a, const CUte
 
 static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Self-test of the bounded-wait discipline: one warp waits on a barrier that nothing will ever
+// complete, with a spin limit of a few hundred attempts.  The wait gives up, records the
+// timeout status and the kernel returns normally.
+__global__ void selftest_wait_timeout_kernel()
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(&bar, 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    mbar_wait(&bar, 0, &abort_flag, 256u);
+}
+
 }  // namespace mxfp4
 
 using namespace mxfp4;
@@ -369,6 +385,15 @@ int mxfp4_linear_static(int pass, const void* a, const void* b, void* out, int64
     // rewrite every code byte and every scale tile (padding included) the GEMM will read.
     return linear_pass(pass, a, b, out, T, in_features, out_features, hadamard_mode, rounding, seed,
                        out_dtype, scratch, MXFP4_STATIC_SCRATCH_BYTES, stream);
+}
+
+int mxfp4_selftest_wait_timeout(void* stream)
+{
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return MXFP4_ERR_CUDA;
+    if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
+    selftest_wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>();
+    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
 int mxfp4_check(void* stream)

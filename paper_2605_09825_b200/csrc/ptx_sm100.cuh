@@ -87,9 +87,10 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity)
 
 // Bounded wait.  `abort_flag` is a CTA-shared word: once set, waits return immediately so the
 // CTA drains and exits.  Returns false if the wait was abandoned.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t spin_limit = kSpinLimit)
 {
-    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+    for (uint32_t spin = 0; spin < spin_limit; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }

@@ -147,3 +147,14 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     want = api.linear_fprop(to_dev(Xb), to_dev(Wb))
     api.check()
     assert (Yh.cuda() == want).all()
+
+
+def test_an_expired_bounded_wait_is_reported_and_the_context_stays_usable():
+    api.check()                                       # clean slate
+    api.selftest_wait_timeout()
+    with pytest.raises(api.Mxfp4Error) as err:
+        api.check()
+    assert err.value.status == -7
+    api.check()                                       # the status was cleared by the read
+    # and the device still computes correctly afterwards
+    test_all_ones_counts_k()
