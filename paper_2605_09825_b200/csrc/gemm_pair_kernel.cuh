@@ -243,13 +243,15 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                             if (j < nmma) {
                                 // K = 64 step j: 32 bytes along the 128-byte swizzled row; two
                                 // MMAs, one per 192-column half of the tile
-#pragma unroll
-                                for (int h = 0; h < 2; ++h)
-                                    tcgen05_mma_mxf4_pair(tmem + h * kPMmaN, a_desc + 2 * j,
-                                                          b_desc + 2 * j + h * (kPBSubBytes >> 4),
-                                                          (j & 1) ? idesc2 : idesc0, sf_tmem + (j >> 1) * 4,
-                                                          sf_tmem + 8 + (j >> 1) * 12 + h * 6,
-                                                          (ks > 0 || j > 0) ? 1u : 0u);
+                                tcgen05_mma_mxf4_pair_collect<0>(tmem, a_desc + 2 * j, b_desc + 2 * j,
+                                                                 (j & 1) ? idesc2 : idesc0, sf_tmem + (j >> 1) * 4,
+                                                                 sf_tmem + 8 + (j >> 1) * 12,
+                                                                 (ks > 0 || j > 0) ? 1u : 0u);
+                                tcgen05_mma_mxf4_pair_collect<1>(tmem + kPMmaN, a_desc + 2 * j,
+                                                                 b_desc + 2 * j + (kPBSubBytes >> 4),
+                                                                 (j & 1) ? idesc2 : idesc0, sf_tmem + (j >> 1) * 4,
+                                                                 sf_tmem + 8 + (j >> 1) * 12 + 6,
+                                                                 (ks > 0 || j > 0) ? 1u : 0u);
                             }
                         }
                         // frees the shared-memory stage and its TMEM scale columns in both CTAs
