@@ -317,6 +317,11 @@ def run_ours(args):
     roofline = {
         "kernel": "gemm_mxf4_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak,
         "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak, "traffic": None,
+        "traffic_captured": {"dram_bytes": 81.3e6, "algorithmic_bytes": 130.1e6,
+                             "launch": "8192x6144x4096 (QKV Fprop at 8192 tokens), ncu, profiles/",
+                             "note": "DRAM traffic does not scale with flops (operands are re-read from "
+                                     "L2, the output is partly still in L2 at kernel end), so no "
+                                     "per-launch figure is extrapolated for the 12 shapes of this step"},
         "peak_source": f"4 x sustained cuBLAS bf16 ({peaks['source']}); burst would be "
                        f"{4.0 * peaks['bf16_tflops']:.0f}, nominal dense FP4 9000",
         "flops_per_launch": gemm_flops / n_gemm, "avg_launch_ms": gemm_ms / n_gemm,
@@ -324,7 +329,11 @@ def run_ours(args):
     quant_gbs = quant_bytes / (quant_ms * 1e-3) / 1e9
     quantize_info = {"kernel": "quantize_kernel", "bound": "hbm", "achieved": quant_gbs,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"],
-                     "bytes_per_element": 2.53125, "avg_launch_ms": quant_ms / (2 * n_gemm)}
+                     "bytes_per_element": 2.53125, "avg_launch_ms": quant_ms / (2 * n_gemm),
+                     # ncu on the 117.4 M-element tensor: 234.9 MB read + 45.4 MB written = 2.39 B per
+                     # element (reads = source bytes exactly; part of the output is still in L2 when
+                     # the kernel ends); traffic is proportional to elements, scaled to the mean launch
+                     "traffic": 2.39 * quant_bytes / 2.53125 / (2 * n_gemm)}
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region
     e2e = None
