@@ -94,6 +94,7 @@ struct GemmPairParams {
     int32_t sf_rows_b;          // ceil(N / 128)
     float alpha;
     int32_t out_fp32;
+    int32_t n_tma;              // bf16 output: columns written by TMA stores (N rounded down to 8)
 };
 
 // Instruction descriptor of the pair MMA: E2M1 x E2M1, E8M0 scales, both operands K-major,
@@ -381,7 +382,22 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                                        w[c * 32 + q * 4 + 3]);
                     fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0 && row0 < p.M && colbase + c * 64 < p.N) {
+                    if (p.n_tma < p.N) {
+                        // N is not a multiple of 8: a TMA store writes whole 16-byte granules, so
+                        // the tensor map ends at the last full granule and the few columns after
+                        // it are stored one by one from this thread's staged row
+                        const int64_t rc = p.n_tma - (colbase + c * 64);
+                        const int64_t row = row0 + lane;
+                        if (rc >= 0 && rc < 64 && row < p.M) {
+                            const int q = static_cast<int>(rc >> 3);
+                            const uint4 v = *reinterpret_cast<const uint4*>(stg + lane * 128 + ((q ^ (lane & 7)) * 16));
+                            const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+                            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.out) + row * p.ld_out + p.n_tma;
+                            for (int k = 0; k < 8; ++k)
+                                if (p.n_tma + k < p.N) dst[k] = e[k];
+                        }
+                    }
+                    if (lane == 0 && row0 < p.M && colbase + c * 64 < p.n_tma) {
                         tma_store_2d_hint(&tm_out, stg, static_cast<int32_t>(colbase + c * 64),
                                           static_cast<int32_t>(row0), store_policy);
                         bulk_commit_group();
@@ -410,8 +426,9 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
 {
     CUtensorMap tm_a, tm_b, tm_out;
     // bf16 output through TMA stores of 64 columns x 32 rows (fp32 output is stored directly)
-    if (out_dtype == MXFP4_OUT_BF16) {
-        if (!make_tmap_2d(&tm_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, out, M, N, ld_out * 2, 32, 64,
+    const int64_t n_tma = out_dtype == MXFP4_OUT_BF16 ? (N & ~static_cast<int64_t>(7)) : 0;
+    if (n_tma > 0) {
+        if (!make_tmap_2d(&tm_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, out, M, n_tma, ld_out * 2, 32, 64,
                           CU_TENSOR_MAP_SWIZZLE_128B))
             return MXFP4_ERR_CUDA;
     } else {
@@ -439,6 +456,7 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     p.sf_rows_b = static_cast<int32_t>((N + 127) / 128);
     p.alpha = alpha;
     p.out_fp32 = out_dtype == MXFP4_OUT_FP32;
+    p.n_tma = static_cast<int32_t>(n_tma);
     const int64_t total = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
     if (total > 0x3FFFFFFF) return MXFP4_ERR_SHAPE;
     const size_t smem = sizeof(GemmPairSmem) + 1024;

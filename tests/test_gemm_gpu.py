@@ -158,3 +158,19 @@ def test_an_expired_bounded_wait_is_reported_and_the_context_stays_usable():
     api.check()                                       # the status was cleared by the read
     # and the device still computes correctly afterwards
     test_all_ones_counts_k()
+
+
+@pytest.mark.parametrize("M,N,K,ld,out_dtype", [(130, 100, 32, 104, api.OUT_BF16), (257, 50, 160, 52, api.OUT_FP32),
+                                                (64, 385, 64, 392, api.OUT_BF16), (300, 769, 288, 776, api.OUT_FP32)])
+def test_ragged_n_with_padded_leading_dimension(M, N, K, ld, out_dtype):
+    # N is not a multiple of the 8-element store granule; the columns between N and ld must stay untouched
+    rng = np.random.default_rng(M + N + K)
+    ac, asc, bc, bsc = _random_operands(rng, M, N, K)
+    dt = torch.bfloat16 if out_dtype == api.OUT_BF16 else torch.float32
+    big = torch.full((M, ld), 7.0, dtype=dt, device="cuda")
+    api.gemm(_dev(ac), _dev(oracle.scales_to_tiled(asc)), _dev(bc), _dev(oracle.scales_to_tiled(bsc)), 0.5,
+             out_dtype, out=big[:, :N])
+    api.check()
+    ref, S = oracle.gemm(ac, asc, bc, bsc, alpha=0.5)
+    assert_gemm_close(big[:, :N].float().cpu().numpy(), ref, S, out_dtype == api.OUT_BF16, "ragged N")
+    assert (big[:, N:] == 7.0).all()

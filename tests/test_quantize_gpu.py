@@ -53,6 +53,13 @@ def test_ragged_shapes_span_tiles_and_tails(rows, cols, axis, hmode, rnd):
     assert (raw[~used] == 0).all()
 
 
+def test_narrow_column_wise_sources():
+    rng = np.random.default_rng(6)
+    _check(random_bits(rng, 64, 8), 0, 1, 0)        # outer = 8 operand rows, K = 64
+    _check(random_bits(rng, 32, 136), 0, 3, 1)      # outer = 136: one full tile + 8 rows
+    _check(random_bits(rng, 4128, 8), 0, 2, 0)      # K = 4128 = 32 tiles + one block
+
+
 def test_one_row_axis1():
     rng = np.random.default_rng(5)
     _check(random_bits(rng, 1, 64), 1, 1, 0)
