@@ -78,12 +78,15 @@ def test_strided_source_rows():
     full = random_bits(rng, 200, 512)
     dev = to_dev(full)
     view = dev[:, 64:64 + 256]                       # ld = 512, cols = 256, base 128-byte aligned
-    for axis in (1,):
-        codes, scales = api.quantize(view, axis, 1, 0)
+    for axis in (1, 0):
+        v = view if axis == 1 else view[:192]                  # column-wise blocks need rows % 32 == 0
+        sub = np.ascontiguousarray(full[:v.shape[0], 64:320])
+        codes, scales = api.quantize(v, axis, 1, 0)
         api.check()
-        want = oracle.quantize(np.ascontiguousarray(full[:, 64:320]), axis, 1, 0)
+        want = oracle.quantize(sub, axis, 1, 0)
+        outer, nt = want[1].shape
         assert (codes.cpu().numpy() == want[0]).all()
-        assert (oracle.scales_from_tiled(scales.cpu().numpy(), 200, 8) == want[1]).all()
+        assert (oracle.scales_from_tiled(scales.cpu().numpy(), outer, nt) == want[1]).all()
 
 
 def test_every_bf16_pattern_and_special_blocks():
@@ -136,3 +139,14 @@ def test_canary_bytes_around_outputs_stay_untouched():
 def test_config2_full_size(name, axis):
     t = synth.config2()
     _check(t[name], axis, 1, 0, seed=0, tag=0)
+
+
+def test_binding_raises_on_bad_shapes_and_missing_cuda_tensor():
+    x = torch.zeros((4, 48), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(api.Mxfp4Error) as e:
+        api.quantize(x, 1)
+    assert e.value.status == -2
+    with pytest.raises(ValueError):
+        api.quantize(torch.zeros((4, 64), dtype=torch.float32, device="cuda"), 1)
+    with pytest.raises(ValueError):
+        api.quantize(torch.zeros((4, 64), dtype=torch.bfloat16), 1)      # host tensor: no CPU path
