@@ -311,6 +311,39 @@ def run_ours(args):
     clocks = sampler.stop(t_begin, t_end)
     api.check()
 
+    # ---- the single-pass configurations (8192 tokens), fused call, L2 flushed between repetitions
+    per_config = {}
+    if args.workload == "layer_stack" and not args.no_configs:
+        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+        T8 = 8192
+        cases = [("config 2: QKV Fprop", "qkv", 0), ("config 3: gate+up Fprop", "gate_up", 0),
+                 ("config 3: gate+up Dgrad", "gate_up", 1), ("config 4: down Wgrad", "down", 2)]
+        for label, n, pss in cases:
+            o, i = dims[n]
+            d = dev_in[n]
+            a_t = (d["X"] if pss == 0 else d["dY"])[:T8]
+            b_t = d["X"][:T8] if pss == 2 else d["W"]
+            M, N, K = pass_dims(pss, T8, i, o)
+            times = []
+            for rep in range(8):
+                flush.zero_()
+                c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                c0.record(stream)
+                rc = fused[pss](a_t.data_ptr(), b_t.data_ptr(), out_buf.data_ptr(), T8, i, o, hmode, rnd, seed,
+                                api.OUT_BF16, ws.data_ptr(), ws_bytes, sptr)
+                c1.record(stream)
+                if rc != 0:
+                    raise api.Mxfp4Error(rc, "fused linear pass")
+                torch.cuda.synchronize()
+                if rep >= 3:
+                    times.append(c0.elapsed_time(c1))
+            ms = statistics.median(times)
+            tf = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+            per_config[label] = {"M": M, "N": N, "K": K, "ms": ms, "tflops_incl_quantize": tf,
+                                 "frac_of_nominal_fp4_peak": tf / 9000.0}
+        del flush
+        api.check()
+
     n_gemm = len(passes)
     fp4_peak = 4.0 * peaks["bf16_tflops_sustained"]
     gemm_tflops = gemm_flops / (gemm_ms * 1e-3) / 1e12
@@ -425,7 +458,7 @@ def run_ours(args):
         "roofline": roofline, "quantize": quantize_info,
         "frac_of_nominal_fp4_peak": world and (flops_per_step / (ms_per_step * 1e-3) / 1e12) / 9000.0,
         "cpu_baseline": cpu_base, "e2e": e2e, "gpu_launches": 3 * len(passes) * args.steps,
-        "clocks": clocks, "context": context,
+        "clocks": clocks, "context": context, "per_config": per_config,
     }
     print(json.dumps(line))
 
@@ -441,6 +474,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-context", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
