@@ -111,6 +111,27 @@ int mxfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_
                    void* codes, void* scales, int scale_layout, void* stream);
 
 /*
+ * mxfp4_quantize_pair -- mxfp4_quantize for two tensors in ONE kernel launch (the two operands
+ * of a linear pass, Appendix D: both are quantized along the GEMM's reduction axis).  The result
+ * for each tensor is bit-identical to its own mxfp4_quantize call; rotation, rounding and seed are
+ * shared, the operand tags are per tensor.  `a` and `b` point to HOST structs; every pointer
+ * inside them is a DEVICE pointer with the alignment and shape rules of mxfp4_quantize.
+ * Supported axis pairs (a, b): (COLS, COLS), (COLS, ROWS), (ROWS, ROWS) -- the three a linear
+ * layer's passes need; any other returns MXFP4_ERR_ENUM.  Nothing is launched on error.
+ */
+typedef struct mxfp4_quant_desc {
+    const void* src_bf16;   /* device, [rows x cols] bf16 row-major                 */
+    int64_t rows, cols, ld_src;
+    int32_t axis;           /* MXFP4_AXIS_COLS / MXFP4_AXIS_ROWS                     */
+    uint32_t operand_tag;
+    void* codes;            /* device out, [outer x K/2] bytes                      */
+    void* scales;           /* device out, mxfp4_scales_bytes(outer, K, layout)     */
+} mxfp4_quant_desc;
+
+int mxfp4_quantize_pair(const mxfp4_quant_desc* a, const mxfp4_quant_desc* b, int hadamard_mode,
+                        int rounding, uint64_t seed, int scale_layout, void* stream);
+
+/*
  * mxfp4_gemm -- the block-scaled product the linear layers run in place of their FP8 GEMM
  * (Appendix A.2 last paragraph; operand orientation per Appendix C):
  *   out[m][n] = alpha * sum_t 2^(sa[m][t]-127) * 2^(sb[n][t]-127) * sum_{k in block t} A[m][k]*B[n][k]

@@ -22,11 +22,18 @@ AXIS_ROWS, AXIS_COLS = 0, 1
 
 EXPORTS = (
     "mxfp4_version", "mxfp4_status_string", "mxfp4_codes_bytes", "mxfp4_scales_bytes",
-    "mxfp4_quantize", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
+    "mxfp4_quantize", "mxfp4_quantize_pair", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
     "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_host", "mxfp4_linear_static",
     "mxfp4_check", "mxfp4_selftest_wait_timeout",
 )
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+
+class QuantDesc(ctypes.Structure):
+    """``mxfp4_quant_desc``: one tensor of an ``mxfp4_quantize_pair`` call."""
+    _fields_ = [("src_bf16", ctypes.c_void_p), ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
+                ("ld_src", ctypes.c_int64), ("axis", ctypes.c_int32), ("operand_tag", ctypes.c_uint32),
+                ("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p)]
 
 
 class Mxfp4Error(RuntimeError):
@@ -62,6 +69,8 @@ def load_library() -> ctypes.CDLL:
     lib.mxfp4_scales_bytes.argtypes, lib.mxfp4_scales_bytes.restype = [i64, i64, ci], sz
     lib.mxfp4_quantize.argtypes = [vp, i64, i64, i64, ci, ci, ci, u64, u32, vp, vp, ci, vp]
     lib.mxfp4_quantize.restype = ci
+    lib.mxfp4_quantize_pair.argtypes = [ctypes.POINTER(QuantDesc), ctypes.POINTER(QuantDesc), ci, ci, u64, ci, vp]
+    lib.mxfp4_quantize_pair.restype = ci
     lib.mxfp4_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, ctypes.c_float, vp, ci, i64, vp, sz, vp]
     lib.mxfp4_gemm.restype = ci
     lib.mxfp4_linear_workspace_bytes.argtypes = [i64, i64, i64, ci]
@@ -142,6 +151,40 @@ def quantize(src: torch.Tensor, axis: int = AXIS_COLS, hadamard_mode: int = HADA
                             _dev_ptr(scales), scale_layout, _stream())
     _raise(rc, "mxfp4_quantize")
     return codes, scales
+
+
+def _quant_desc(src, axis, tag, scale_layout, codes, scales):
+    if src.dtype != torch.bfloat16 or src.dim() != 2 or src.stride(1) != 1:
+        raise ValueError("src must be a 2-D bf16 tensor with contiguous rows")
+    rows, cols = src.shape
+    outer, K = (rows, cols) if axis == AXIS_COLS else (cols, rows)
+    if K % 32 != 0 or K <= 0 or outer <= 0:
+        _raise(-2, "mxfp4_quantize_pair")
+    if codes is None:
+        codes = torch.empty((outer, K // 2), dtype=torch.uint8, device=src.device)
+    if scales is None:
+        scales = torch.empty(scales_bytes(outer, K, scale_layout), dtype=torch.uint8, device=src.device)
+    ld = src.stride(0) if rows > 1 else cols
+    return QuantDesc(_dev_ptr(src), rows, cols, ld, axis, tag, _dev_ptr(codes), _dev_ptr(scales)), codes, scales
+
+
+def quantize_pair(src_a: torch.Tensor, axis_a: int, src_b: torch.Tensor, axis_b: int,
+                  hadamard_mode: int = HADAMARD_NONE, rounding: int = ROUND_RNE, seed: int = 0,
+                  tags=(0, 1), scale_layout: int = SCALES_TILED, out_a=None, out_b=None):
+    """``mxfp4_quantize_pair``: both tensors through one launch.
+
+    ``out_a`` / ``out_b`` are optional ``(codes, scales)`` tensors.  Returns
+    ``((codes_a, scales_a), (codes_b, scales_b))``.
+    """
+    lib = load_library()
+    ca, sa = out_a if out_a is not None else (None, None)
+    cb, sb = out_b if out_b is not None else (None, None)
+    da, ca, sa = _quant_desc(src_a, axis_a, tags[0], scale_layout, ca, sa)
+    db, cb, sb = _quant_desc(src_b, axis_b, tags[1], scale_layout, cb, sb)
+    rc = lib.mxfp4_quantize_pair(ctypes.byref(da), ctypes.byref(db), hadamard_mode, rounding,
+                                 ctypes.c_uint64(seed), scale_layout, _stream())
+    _raise(rc, "mxfp4_quantize_pair")
+    return (ca, sa), (cb, sb)
 
 
 def gemm(a_codes: torch.Tensor, a_scales: torch.Tensor, b_codes: torch.Tensor, b_scales: torch.Tensor,

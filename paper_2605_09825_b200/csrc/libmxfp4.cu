@@ -57,41 +57,109 @@ static uint32_t host_sign_mask(uint64_t seed)
     return c[0];
 }
 
-template <int AXIS, int HMODE, int SR>
-static int launch_quantize(const CUtensorMap& tm_src, const CUtensorMap& tm_codes,
-                           const QuantParams& p, int grid, cudaStream_t stream)
+template <int AXIS0, int AXIS1, int HMODE, int SR>
+static int launch_quantize(const QuantJob& j0, const QuantJob& j1, int grid, cudaStream_t stream)
 {
     const size_t smem = sizeof(QuantSmem) + 1024;
     static bool attr_set[64] = {};          // the attribute is per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(quantize_kernel<AXIS, HMODE, SR>,
+        if (cudaFuncSetAttribute(quantize_kernel<AXIS0, AXIS1, HMODE, SR>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess)
             return MXFP4_ERR_CUDA;
         attr_set[dev] = true;
     }
-    quantize_kernel<AXIS, HMODE, SR><<<grid, kQThreads, smem, stream>>>(tm_src, tm_codes, p);
+    QuantJobs jobs;
+    jobs.j[0] = j0;
+    jobs.j[1] = j1;
+    quantize_kernel<AXIS0, AXIS1, HMODE, SR><<<grid, kQThreads, smem, stream>>>(jobs);
     return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
-template <int AXIS>
-static int dispatch_quantize(int hmode, int sr, const CUtensorMap& a, const CUtensorMap& b,
-                             const QuantParams& p, int grid, cudaStream_t st)
+template <int AXIS0, int AXIS1>
+static int dispatch_quantize(int hmode, int sr, const QuantJob& j0, const QuantJob& j1, int grid,
+                             cudaStream_t st)
 {
     switch (hmode * 2 + sr) {
-        case 0: return launch_quantize<AXIS, 0, 0>(a, b, p, grid, st);
-        case 1: return launch_quantize<AXIS, 0, 1>(a, b, p, grid, st);
-        case 2: return launch_quantize<AXIS, 1, 0>(a, b, p, grid, st);
-        case 3: return launch_quantize<AXIS, 1, 1>(a, b, p, grid, st);
-        case 4: return launch_quantize<AXIS, 2, 0>(a, b, p, grid, st);
-        case 5: return launch_quantize<AXIS, 2, 1>(a, b, p, grid, st);
-        case 6: return launch_quantize<AXIS, 3, 0>(a, b, p, grid, st);
-        case 7: return launch_quantize<AXIS, 3, 1>(a, b, p, grid, st);
-        case 8: return launch_quantize<AXIS, 4, 0>(a, b, p, grid, st);
-        default: return launch_quantize<AXIS, 4, 1>(a, b, p, grid, st);
+        case 0: return launch_quantize<AXIS0, AXIS1, 0, 0>(j0, j1, grid, st);
+        case 1: return launch_quantize<AXIS0, AXIS1, 0, 1>(j0, j1, grid, st);
+        case 2: return launch_quantize<AXIS0, AXIS1, 1, 0>(j0, j1, grid, st);
+        case 3: return launch_quantize<AXIS0, AXIS1, 1, 1>(j0, j1, grid, st);
+        case 4: return launch_quantize<AXIS0, AXIS1, 2, 0>(j0, j1, grid, st);
+        case 5: return launch_quantize<AXIS0, AXIS1, 2, 1>(j0, j1, grid, st);
+        case 6: return launch_quantize<AXIS0, AXIS1, 3, 0>(j0, j1, grid, st);
+        case 7: return launch_quantize<AXIS0, AXIS1, 3, 1>(j0, j1, grid, st);
+        case 8: return launch_quantize<AXIS0, AXIS1, 4, 0>(j0, j1, grid, st);
+        default: return launch_quantize<AXIS0, AXIS1, 4, 1>(j0, j1, grid, st);
     }
+}
+
+// Validates one tensor's arguments and fills its job (tensor maps + parameters).
+static int build_quant_job(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis,
+                           int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
+                           void* codes, void* scales, int scale_layout, QuantJob* job)
+{
+    if (!src_bf16 || !codes || !scales) return MXFP4_ERR_NULL;
+    if (axis != 0 && axis != 1) return MXFP4_ERR_ENUM;
+    if (hadamard_mode < 0 || hadamard_mode > 4 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
+    if (scale_layout != 0 && scale_layout != 1) return MXFP4_ERR_ENUM;
+    if (rows <= 0 || cols <= 0 || ld_src < cols) return MXFP4_ERR_SHAPE;
+    const int64_t outer = axis ? rows : cols;
+    const int64_t K = axis ? cols : rows;
+    if (K % 32 != 0) return MXFP4_ERR_SHAPE;
+    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (!aligned16(src_bf16) || !aligned16(codes) || !aligned16(scales)) return MXFP4_ERR_ALIGN;
+    if (ld_src % 8 != 0) return MXFP4_ERR_ALIGN;
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return MXFP4_ERR_CUDA;
+    if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
+
+    const bool ok_src =
+        axis == 1 ? make_tmap_2d(&job->tm_src, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, src_bf16, rows, cols,
+                                 ld_src * 2, 128, 64, CU_TENSOR_MAP_SWIZZLE_128B)
+                  : make_tmap_2d(&job->tm_src, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, src_bf16, rows, cols,
+                                 ld_src * 2, 128, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+    const bool ok_codes = make_tmap_2d(&job->tm_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, outer,
+                                       K / 2, K / 2, 128, 64, CU_TENSOR_MAP_SWIZZLE_64B);
+    if (!ok_src || !ok_codes) return MXFP4_ERR_CUDA;
+
+    QuantParams& p = job->p;
+    p.scales = static_cast<uint8_t*>(scales);
+    p.outer = outer;
+    p.K = K;
+    p.nt = K / 32;
+    p.tiles_o = static_cast<int32_t>((outer + kQTileO - 1) / kQTileO);
+    p.tiles_k = static_cast<int32_t>((K + kQTileK - 1) / kQTileK);
+    p.seed_lo = static_cast<uint32_t>(seed);
+    p.seed_hi = static_cast<uint32_t>(seed >> 32);
+    p.tag = operand_tag;
+    p.sign_mask = 0u;
+    if (hadamard_mode == MXFP4_HADAMARD_RAND) p.sign_mask = host_sign_mask(seed);
+    if (hadamard_mode == MXFP4_HADAMARD_RAND16) {
+        const uint32_t m16 = host_sign_mask(seed) & 0xFFFFu;   // same 16 signs for both halves
+        p.sign_mask = m16 | (m16 << 16);
+    }
+    p.scale_layout = scale_layout;
+    const int64_t total = static_cast<int64_t>(p.tiles_o) * p.tiles_k;
+    if (total > 0x3FFFFFFF) return MXFP4_ERR_SHAPE;
+    job->tiles = static_cast<int32_t>(total);
+    return MXFP4_OK;
+}
+
+// One launch for one or two jobs (axis1 is ignored when j1 is empty).
+static int launch_quant_jobs(const QuantJob& j0, const QuantJob& j1, int axis0, int axis1, int hmode, int sr,
+                             cudaStream_t st)
+{
+    const DeviceInfo& dev = device_info();
+    const int64_t total = static_cast<int64_t>(j0.tiles) + j1.tiles;
+    const int grid = static_cast<int>(total < dev.sm_count ? total : dev.sm_count);
+    if (j1.tiles == 0) axis1 = axis0;
+    if (axis0 == 1 && axis1 == 1) return dispatch_quantize<1, 1>(hmode, sr, j0, j1, grid, st);
+    if (axis0 == 1 && axis1 == 0) return dispatch_quantize<1, 0>(hmode, sr, j0, j1, grid, st);
+    if (axis0 == 0 && axis1 == 0) return dispatch_quantize<0, 0>(hmode, sr, j0, j1, grid, st);
+    return MXFP4_ERR_ENUM;   // (0, 1) is never asked for: callers order row-wise first
 }
 
 static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -157,54 +225,27 @@ int mxfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_
                    int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
                    void* codes, void* scales, int scale_layout, void* stream)
 {
-    if (!src_bf16 || !codes || !scales) return MXFP4_ERR_NULL;
-    if (axis != 0 && axis != 1) return MXFP4_ERR_ENUM;
-    if (hadamard_mode < 0 || hadamard_mode > 4 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
-    if (scale_layout != 0 && scale_layout != 1) return MXFP4_ERR_ENUM;
-    if (rows <= 0 || cols <= 0 || ld_src < cols) return MXFP4_ERR_SHAPE;
-    const int64_t outer = axis ? rows : cols;
-    const int64_t K = axis ? cols : rows;
-    if (K % 32 != 0) return MXFP4_ERR_SHAPE;
-    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
-    if (!aligned16(src_bf16) || !aligned16(codes) || !aligned16(scales)) return MXFP4_ERR_ALIGN;
-    if (ld_src % 8 != 0) return MXFP4_ERR_ALIGN;
-    const DeviceInfo& dev = device_info();
-    if (!dev.ok) return MXFP4_ERR_CUDA;
-    if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
+    QuantJob j0, j1;
+    const int rc = build_quant_job(src_bf16, rows, cols, ld_src, axis, hadamard_mode, rounding, seed,
+                                   operand_tag, codes, scales, scale_layout, &j0);
+    if (rc != MXFP4_OK) return rc;
+    memset(&j1, 0, sizeof(j1));
+    return launch_quant_jobs(j0, j1, axis, axis, hadamard_mode, rounding, static_cast<cudaStream_t>(stream));
+}
 
-    CUtensorMap tm_src, tm_codes;
-    const bool ok_src =
-        axis == 1 ? make_tmap_2d(&tm_src, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, src_bf16, rows, cols,
-                                 ld_src * 2, 128, 64, CU_TENSOR_MAP_SWIZZLE_128B)
-                  : make_tmap_2d(&tm_src, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, src_bf16, rows, cols,
-                                 ld_src * 2, 128, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
-    const bool ok_codes = make_tmap_2d(&tm_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, outer,
-                                       K / 2, K / 2, 128, 64, CU_TENSOR_MAP_SWIZZLE_64B);
-    if (!ok_src || !ok_codes) return MXFP4_ERR_CUDA;
-
-    QuantParams p;
-    p.scales = static_cast<uint8_t*>(scales);
-    p.outer = outer;
-    p.K = K;
-    p.nt = K / 32;
-    p.tiles_o = static_cast<int32_t>((outer + kQTileO - 1) / kQTileO);
-    p.tiles_k = static_cast<int32_t>((K + kQTileK - 1) / kQTileK);
-    p.seed_lo = static_cast<uint32_t>(seed);
-    p.seed_hi = static_cast<uint32_t>(seed >> 32);
-    p.tag = operand_tag;
-    p.sign_mask = 0u;
-    if (hadamard_mode == MXFP4_HADAMARD_RAND) p.sign_mask = host_sign_mask(seed);
-    if (hadamard_mode == MXFP4_HADAMARD_RAND16) {
-        const uint32_t m16 = host_sign_mask(seed) & 0xFFFFu;   // same 16 signs for both halves
-        p.sign_mask = m16 | (m16 << 16);
-    }
-    p.scale_layout = scale_layout;
-    const int64_t total = static_cast<int64_t>(p.tiles_o) * p.tiles_k;
-    if (total > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
-    const int grid = static_cast<int>(total < dev.sm_count ? total : dev.sm_count);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return axis == 1 ? dispatch_quantize<1>(hadamard_mode, rounding, tm_src, tm_codes, p, grid, st)
-                     : dispatch_quantize<0>(hadamard_mode, rounding, tm_src, tm_codes, p, grid, st);
+int mxfp4_quantize_pair(const mxfp4_quant_desc* a, const mxfp4_quant_desc* b, int hadamard_mode,
+                        int rounding, uint64_t seed, int scale_layout, void* stream)
+{
+    if (!a || !b) return MXFP4_ERR_NULL;
+    if (a->axis == MXFP4_AXIS_ROWS && b->axis == MXFP4_AXIS_COLS) return MXFP4_ERR_ENUM;
+    QuantJob ja, jb;
+    int rc = build_quant_job(a->src_bf16, a->rows, a->cols, a->ld_src, a->axis, hadamard_mode, rounding, seed,
+                             a->operand_tag, a->codes, a->scales, scale_layout, &ja);
+    if (rc != MXFP4_OK) return rc;
+    rc = build_quant_job(b->src_bf16, b->rows, b->cols, b->ld_src, b->axis, hadamard_mode, rounding, seed,
+                         b->operand_tag, b->codes, b->scales, scale_layout, &jb);
+    if (rc != MXFP4_OK) return rc;
+    return launch_quant_jobs(ja, jb, a->axis, b->axis, hadamard_mode, rounding, static_cast<cudaStream_t>(stream));
 }
 
 int mxfp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes,
@@ -279,11 +320,15 @@ static int linear_pass(int pass, const void* a_src, const void* b_src, void* out
     } else {                                 // A = dY [T x out] column-wise, B = X [T x in] column-wise
         ar = T; ac = out_f; a_axis = 0; br = T; bc = in_f; b_axis = 0;
     }
-    int rc = mxfp4_quantize(a_src, ar, ac, ac, a_axis, hmode, rounding, seed, 0u, a_codes, a_scales,
-                            MXFP4_SCALES_TILED, stream);
+    // both operands through one quantize launch
+    QuantJob ja, jb;
+    int rc = build_quant_job(a_src, ar, ac, ac, a_axis, hmode, rounding, seed, 0u, a_codes, a_scales,
+                             MXFP4_SCALES_TILED, &ja);
     if (rc != MXFP4_OK) return rc;
-    rc = mxfp4_quantize(b_src, br, bc, bc, b_axis, hmode, rounding, seed, 1u, b_codes, b_scales,
-                        MXFP4_SCALES_TILED, stream);
+    rc = build_quant_job(b_src, br, bc, bc, b_axis, hmode, rounding, seed, 1u, b_codes, b_scales,
+                         MXFP4_SCALES_TILED, &jb);
+    if (rc != MXFP4_OK) return rc;
+    rc = launch_quant_jobs(ja, jb, a_axis, b_axis, hmode, rounding, static_cast<cudaStream_t>(stream));
     if (rc != MXFP4_OK) return rc;
     // H * H^T = n * I for the +-1 matrix of order n: undo it exactly in the epilogue
     const float alpha = hmode == MXFP4_HADAMARD_NONE ? 1.0f : (hmode <= MXFP4_HADAMARD_RAND ? 0.03125f : 0.0625f);

@@ -54,6 +54,21 @@ struct QuantParams {
     int32_t scale_layout;    // 0 canonical, 1 tiled
 };
 
+// One tensor to quantize: its source and code tensor maps plus parameters.  A launch takes two
+// jobs (the second may be empty) so that both operands of a linear pass go through one kernel:
+// the tail of the first tensor overlaps the start of the second and one launch gap disappears.
+struct QuantJob {
+    CUtensorMap tm_src;
+    CUtensorMap tm_codes;
+    QuantParams p;
+    int32_t tiles;           // tiles_o * tiles_k, 0 for an empty job
+};
+// Both jobs as one kernel parameter: indexing it with the (block-uniform) job number reads the
+// fields straight from parameter space instead of holding both sets in registers.
+struct QuantJobs {
+    QuantJob j[2];
+};
+
 // Packed fp32 pairs: sm_100 adds, multiplies and fuses two independent fp32 values held in a
 // float2 (an aligned register pair) with a single instruction; each lane is an ordinary IEEE
 // fp32 round-to-nearest operation, so results are bit-identical to the scalar form.  a - b is
@@ -233,16 +248,116 @@ __device__ __forceinline__ void quantize_block(float2 (&P)[16], uint64_t e0, con
     }
 }
 
+// tile index of a job -> (operand-row tile, K tile); the fastest-varying index walks the source's
+// contiguous axis
+template <int AXIS>
+__device__ __forceinline__ void tile_coords(const QuantParams& p, int tile, int& to, int& tk)
+{
+    if (AXIS == 1) { to = tile / p.tiles_k; tk = tile % p.tiles_k; }
+    else           { tk = tile / p.tiles_o; to = tile % p.tiles_o; }
+}
+
+template <int AXIS>
+__device__ __forceinline__ void issue_tile_load(const CUtensorMap* tm_src, const QuantParams& p, int tile,
+                                                uint8_t* stage, uint64_t* full)
+{
+    int to, tk;
+    tile_coords<AXIS>(p, tile, to, tk);
+    mbar_arrive_expect_tx(full, kQStageBytes);
+    if (AXIS == 1) {
+        tma_load_2d(stage, tm_src, full, tk * kQTileK, to * kQTileO);
+        tma_load_2d(stage + kQStageBytes / 2, tm_src, full, tk * kQTileK + 64, to * kQTileO);
+    } else {
+        tma_load_2d(stage, tm_src, full, to * kQTileO, tk * kQTileK);
+    }
+}
+
+// One tile of one job, as seen by a consumer thread: wait for the stage, rotate + quantize this
+// thread's two blocks, stage codes and scales, and (thread 0 of the group) store them.  `p` and
+// `tm_codes` refer to kernel parameters, so every field is a constant-bank operand.  Returns
+// false when a wait gave up (the group leaves the kernel).
 template <int AXIS, int HMODE, int SR>
+__device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
+                                             int tile, int it, int trip, int grp, int t)
+{
+    const int kbh = t >> 7;            // this thread's blocks along K: kbh and kbh + 2
+    const int o = t & 127;             // operand row inside the tile
+    const int s = it % kQStages;
+    const uint32_t round = it / kQStages;
+    const int buf = trip & 1;
+    int to, tk;
+    tile_coords<AXIS>(p, tile, to, tk);
+
+    const bool ok = mbar_wait(&sm.full[s], round & 1, &sm.abort_flag);
+
+    float2 P0[16], P1[16];
+    if (ok) {
+        load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.sign_mask, P0);
+        load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.sign_mask, P1);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
+    }
+    // the stage is in registers now: hand it back to the producer
+    __syncwarp();
+    if ((t & 31) == 0) mbar_arrive(&sm.empty[s]);
+
+    const uint64_t e_row = static_cast<uint64_t>(to * kQTileO + o) * static_cast<uint64_t>(p.K);
+    uint32_t packed0[4], packed1[4], byte0, byte1;
+    quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tk * 4 + kbh) * 32), p, packed0, byte0);
+    quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tk * 4 + kbh + 2) * 32), p, packed1, byte1);
+
+    // stage the results: codes in the 64-byte swizzle the TMA store expects
+    uint8_t* ct = &sm.code_tile[grp][buf][o * 64];
+    *reinterpret_cast<uint4*>(ct + ((kbh ^ ((o >> 1) & 3)) * 16)) =
+        make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]);
+    *reinterpret_cast<uint4*>(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16)) =
+        make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]);
+    if (p.scale_layout == 1) {
+        uint8_t* st = &sm.scale_tile[grp][buf][(o & 31) * 16 + (o >> 5) * 4];
+        st[kbh] = static_cast<uint8_t>(byte0);
+        st[kbh + 2] = static_cast<uint8_t>(byte1);
+    } else if (ok) {
+        const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
+        const int64_t tg = static_cast<int64_t>(tk) * 4 + kbh;
+        if (og < p.outer && tg < p.nt) p.scales[og * p.nt + tg] = static_cast<uint8_t>(byte0);
+        if (og < p.outer && tg + 2 < p.nt) p.scales[og * p.nt + tg + 2] = static_cast<uint8_t>(byte1);
+    }
+    fence_proxy_async_smem();
+    // the store this group issued one trip ago must have drained its buffer before the next
+    // trip (which every thread of the group reaches only through the barrier below)
+    // overwrites it
+    if (t == 0) bulk_wait_group_read<0>();
+    uint32_t any_fail;
+    asm volatile(
+        "{\n\t.reg .pred P, Q;\n\t"
+        "setp.ne.u32 Q, %1, 0;\n\t"
+        "barrier.cta.red.or.pred P, %2, %3, Q;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(any_fail)
+        : "r"(ok ? 0u : 1u), "r"(grp + 1), "n"(kQConsumers / 2)
+        : "memory");
+    if (any_fail) return false;
+    if (t == 0) {
+        tma_store_2d(tm_codes, &sm.code_tile[grp][buf][0], tk * (kQTileK / 2), to * kQTileO);
+        if (p.scale_layout == 1)
+            bulk_store_1d(p.scales + (static_cast<int64_t>(to) * p.tiles_k + tk) * kQScaleTileBytes,
+                          &sm.scale_tile[grp][buf][0], kQScaleTileBytes);
+        bulk_commit_group();
+    }
+    return true;
+}
+
+template <int AXIS0, int AXIS1, int HMODE, int SR>
 __global__ void __launch_bounds__(kQThreads, 1)
-quantize_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constant__ CUtensorMap tm_codes,
-                const QuantParams p)
+quantize_kernel(const __grid_constant__ QuantJobs jobs)
 {
     extern __shared__ uint8_t smem_raw[];
     QuantSmem& sm = *reinterpret_cast<QuantSmem*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int tid = threadIdx.x;
-    const int total_tiles = p.tiles_o * p.tiles_k;
+    const int tiles0 = jobs.j[0].tiles;
+    const int total_tiles = tiles0 + jobs.j[1].tiles;
     const int my_tiles = blockIdx.x < total_tiles ? (total_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
 
     if (tid == 0) {
@@ -258,24 +373,18 @@ quantize_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constan
     if (tid >= kQConsumers) {
         // ------------------------------------------------------------ producer warp
         if (tid == kQConsumers) {
-            tma_prefetch_desc(&tm_src);
+            tma_prefetch_desc(&jobs.j[0].tm_src);
+            if (jobs.j[1].tiles > 0) tma_prefetch_desc(&jobs.j[1].tm_src);
             for (int it = 0; it < my_tiles; ++it) {
                 const int tile = blockIdx.x + it * gridDim.x;
                 const int s = it % kQStages;
                 const uint32_t round = it / kQStages;
                 if (round > 0 && !mbar_wait(&sm.empty[s], (round - 1) & 1, &sm.abort_flag)) break;
-                // the fastest-varying tile index walks the source's contiguous axis
-                int to, tk;
-                if (AXIS == 1) { to = tile / p.tiles_k; tk = tile % p.tiles_k; }
-                else           { tk = tile / p.tiles_o; to = tile % p.tiles_o; }
-                mbar_arrive_expect_tx(&sm.full[s], kQStageBytes);
-                if (AXIS == 1) {
-                    tma_load_2d(&sm.stage[s][0], &tm_src, &sm.full[s], tk * kQTileK, to * kQTileO);
-                    tma_load_2d(&sm.stage[s][kQStageBytes / 2], &tm_src, &sm.full[s],
-                                tk * kQTileK + 64, to * kQTileO);
-                } else {
-                    tma_load_2d(&sm.stage[s][0], &tm_src, &sm.full[s], to * kQTileO, tk * kQTileK);
-                }
+                if (tile < tiles0)
+                    issue_tile_load<AXIS0>(&jobs.j[0].tm_src, jobs.j[0].p, tile, &sm.stage[s][0], &sm.full[s]);
+                else
+                    issue_tile_load<AXIS1>(&jobs.j[1].tm_src, jobs.j[1].p, tile - tiles0, &sm.stage[s][0],
+                                           &sm.full[s]);
             }
         }
         return;
@@ -284,76 +393,27 @@ quantize_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constan
     // ---------------------------------------------------------------- consumers
     const int grp = tid >> 8;          // consumer group: takes tiles grp, grp + 2, ...
     const int t = tid & 255;
-    const int kbh = t >> 7;            // this thread's blocks along K: kbh and kbh + 2
-    const int o = t & 127;             // operand row inside the tile
-    if (t == 0) tma_prefetch_desc(&tm_codes);
+    if (t == 0) {
+        tma_prefetch_desc(&jobs.j[0].tm_codes);
+        if (jobs.j[1].tiles > 0) tma_prefetch_desc(&jobs.j[1].tm_codes);
+    }
 
-    int trip = 0;
-    for (int it = grp; it < my_tiles; it += 2, ++trip) {
-        const int tile = blockIdx.x + it * gridDim.x;
-        const int s = it % kQStages;
-        const uint32_t round = it / kQStages;
-        const int buf = trip & 1;
-        int to, tk;
-        if (AXIS == 1) { to = tile / p.tiles_k; tk = tile % p.tiles_k; }
-        else           { tk = tile / p.tiles_o; to = tile % p.tiles_o; }
-
-        const bool ok = mbar_wait(&sm.full[s], round & 1, &sm.abort_flag);
-
-        float2 P0[16], P1[16];
-        if (ok) {
-            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.sign_mask, P0);
-            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.sign_mask, P1);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
-        }
-        // the stage is in registers now: hand it back to the producer
-        __syncwarp();
-        if ((tid & 31) == 0) mbar_arrive(&sm.empty[s]);
-
-        const uint64_t e_row = static_cast<uint64_t>(to * kQTileO + o) * static_cast<uint64_t>(p.K);
-        uint32_t packed0[4], packed1[4], byte0, byte1;
-        quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tk * 4 + kbh) * 32), p, packed0, byte0);
-        quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tk * 4 + kbh + 2) * 32), p, packed1, byte1);
-
-        // stage the results: codes in the 64-byte swizzle the TMA store expects
-        uint8_t* ct = &sm.code_tile[grp][buf][o * 64];
-        *reinterpret_cast<uint4*>(ct + ((kbh ^ ((o >> 1) & 3)) * 16)) =
-            make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]);
-        *reinterpret_cast<uint4*>(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16)) =
-            make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]);
-        if (p.scale_layout == 1) {
-            uint8_t* st = &sm.scale_tile[grp][buf][(o & 31) * 16 + (o >> 5) * 4];
-            st[kbh] = static_cast<uint8_t>(byte0);
-            st[kbh + 2] = static_cast<uint8_t>(byte1);
-        } else if (ok) {
-            const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
-            const int64_t tg = static_cast<int64_t>(tk) * 4 + kbh;
-            if (og < p.outer && tg < p.nt) p.scales[og * p.nt + tg] = static_cast<uint8_t>(byte0);
-            if (og < p.outer && tg + 2 < p.nt) p.scales[og * p.nt + tg + 2] = static_cast<uint8_t>(byte1);
-        }
-        fence_proxy_async_smem();
-        // the store this group issued one trip ago must have drained its buffer before the next
-        // trip (which every thread of the group reaches only through the barrier below)
-        // overwrites it
-        if (t == 0) bulk_wait_group_read<0>();
-        uint32_t any_fail;
-        asm volatile(
-            "{\n\t.reg .pred P, Q;\n\t"
-            "setp.ne.u32 Q, %1, 0;\n\t"
-            "barrier.cta.red.or.pred P, %2, %3, Q;\n\t"
-            "selp.u32 %0, 1, 0, P;\n\t}"
-            : "=r"(any_fail)
-            : "r"(ok ? 0u : 1u), "r"(grp + 1), "n"(kQConsumers / 2)
-            : "memory");
-        if (any_fail) break;
-        if (t == 0) {
-            tma_store_2d(&tm_codes, &sm.code_tile[grp][buf][0], tk * (kQTileK / 2), to * kQTileO);
-            if (p.scale_layout == 1)
-                bulk_store_1d(p.scales + (static_cast<int64_t>(to) * p.tiles_k + tk) * kQScaleTileBytes,
-                              &sm.scale_tile[grp][buf][0], kQScaleTileBytes);
-            bulk_commit_group();
+    // this CTA's tiles come in increasing order: first those of job 0, then those of job 1, each
+    // through a loop specialised for that job's axis and parameters
+    int it = grp, trip = 0;
+    bool alive = true;
+    for (; it < my_tiles; it += 2, ++trip) {
+        const int gtile = blockIdx.x + it * gridDim.x;
+        if (gtile >= tiles0) break;
+        alive = consume_tile<AXIS0, HMODE, SR>(sm, jobs.j[0].p, &jobs.j[0].tm_codes, gtile, it, trip, grp, t);
+        if (!alive) break;
+    }
+    if (alive) {
+        for (; it < my_tiles; it += 2, ++trip) {
+            const int gtile = blockIdx.x + it * gridDim.x;
+            if (!consume_tile<AXIS1, HMODE, SR>(sm, jobs.j[1].p, &jobs.j[1].tm_codes, gtile - tiles0, it, trip,
+                                                grp, t))
+                break;
         }
     }
     if (t == 0) bulk_wait_group<0>();

@@ -150,3 +150,36 @@ def test_binding_raises_on_bad_shapes_and_missing_cuda_tensor():
         api.quantize(torch.zeros((4, 64), dtype=torch.float32, device="cuda"), 1)
     with pytest.raises(ValueError):
         api.quantize(torch.zeros((4, 64), dtype=torch.bfloat16), 1)      # host tensor: no CPU path
+
+
+@pytest.mark.parametrize("hmode,rnd", [(0, 0), (1, 0), (2, 1), (3, 0), (4, 1)])
+@pytest.mark.parametrize("axes", [(1, 1), (1, 0), (0, 0)])
+def test_pair_launch_matches_oracle_for_both_tensors(axes, hmode, rnd):
+    """Two tensors of different shapes through one launch: each bit-exact against the oracle,
+    including the hand-over from the first tensor's tiles to the second's inside one CTA."""
+    rng = np.random.default_rng(101 + 10 * axes[0] + axes[1])
+    shapes = [(416, 1184), (1056, 288)] if axes == (1, 1) else [(608, 736), (352, 1000)]
+    bits = [random_bits(rng, r, c) for r, c in shapes]
+    (ca, sa), (cb, sb) = api.quantize_pair(to_dev(bits[0]), axes[0], to_dev(bits[1]), axes[1], hmode, rnd, 11,
+                                           tags=(0, 1))
+    api.check()
+    for b, ax, tag, c, s in ((bits[0], axes[0], 0, ca, sa), (bits[1], axes[1], 1, cb, sb)):
+        want_codes, want_scales = oracle.quantize(b, ax, hmode, rnd, 11, tag)
+        assert np.array_equal(c.cpu().numpy(), want_codes)
+        outer, K = want_codes.shape[0], want_codes.shape[1] * 2
+        assert np.array_equal(oracle.scales_from_tiled(s.cpu().numpy(), outer, K // 32), want_scales)
+
+
+def test_pair_launch_tiny_first_tensor_and_rejected_axis_order():
+    rng = np.random.default_rng(103)
+    small, big = random_bits(rng, 1, 64), random_bits(rng, 2000, 608)
+    (ca, sa), (cb, sb) = api.quantize_pair(to_dev(small), 1, to_dev(big), 1, 1, 0, 3)
+    api.check()
+    wc, _ = oracle.quantize(small, 1, 1, 0, 3, 0)
+    assert np.array_equal(ca.cpu().numpy(), wc)
+    wc, ws = oracle.quantize(big, 1, 1, 0, 3, 1)
+    assert np.array_equal(cb.cpu().numpy(), wc)
+    assert np.array_equal(oracle.scales_from_tiled(sb.cpu().numpy(), 2000, 608 // 32), ws)
+    with pytest.raises(api.Mxfp4Error) as exc:
+        api.quantize_pair(to_dev(random_bits(rng, 64, 64)), 0, to_dev(random_bits(rng, 64, 64)), 1)
+    assert exc.value.status == -4
