@@ -61,6 +61,8 @@ def _load():
                                     ctypes.c_int, ctypes.c_int, ctypes.c_uint64, ctypes.c_uint32,
                                     u8p, u8p]
     lib.oracle_quantize.restype = ctypes.c_int
+    lib.oracle_quantize_2d.argtypes = lib.oracle_quantize.argtypes
+    lib.oracle_quantize_2d.restype = ctypes.c_int
     lib.oracle_scale_offset_tiled.argtypes = [i64, i64, i64]
     lib.oracle_scale_offset_tiled.restype = i64
     lib.oracle_dequantize.argtypes = [u8p, u8p, i64, i64, ctypes.POINTER(ctypes.c_double)]
@@ -116,11 +118,13 @@ def fwht16x2(v) -> np.ndarray:
 
 
 def quantize(src_bits: np.ndarray, axis: int = 1, hadamard_mode: int = 0, rounding: int = 0,
-             seed: int = 0, tag: int = 0):
+             seed: int = 0, tag: int = 0, block2d: bool = False):
     """MXFP4-quantize a [rows x cols] bf16 matrix (uint16 bit patterns).
 
     Returns ``(codes [outer x K/2] uint8, scales [outer x K/32] uint8)`` for the operand view
     (axis=1: outer=rows, K=cols; axis=0: outer=cols, K=rows -- the transposed operand).
+    ``block2d`` selects the 32 x 32 block strategy of Appendix D (one scale per 32 operand rows
+    x 32 elements, replicated into every row's scale entry) instead of 1 x 32 blocks.
     """
     assert src_bits.dtype == np.uint16 and src_bits.ndim == 2
     src = np.ascontiguousarray(src_bits)
@@ -128,9 +132,10 @@ def quantize(src_bits: np.ndarray, axis: int = 1, hadamard_mode: int = 0, roundi
     outer, K = (rows, cols) if axis == 1 else (cols, rows)
     codes = np.empty((outer, K // 2), dtype=np.uint8)
     scales = np.empty((outer, K // 32), dtype=np.uint8)
-    rc = _load().oracle_quantize(_ptr(src, ctypes.c_uint16), rows, cols, cols, axis, hadamard_mode,
-                                 rounding, ctypes.c_uint64(seed), ctypes.c_uint32(tag),
-                                 _ptr(codes, ctypes.c_uint8), _ptr(scales, ctypes.c_uint8))
+    fn = _load().oracle_quantize_2d if block2d else _load().oracle_quantize
+    rc = fn(_ptr(src, ctypes.c_uint16), rows, cols, cols, axis, hadamard_mode,
+            rounding, ctypes.c_uint64(seed), ctypes.c_uint32(tag),
+            _ptr(codes, ctypes.c_uint8), _ptr(scales, ctypes.c_uint8))
     if rc != 0:
         raise ValueError(f"oracle_quantize rejected its arguments (rc={rc})")
     return codes, scales

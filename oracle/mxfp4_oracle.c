@@ -175,21 +175,33 @@ static uint32_t sr_bits(uint64_t e, uint64_t seed, uint32_t tag)
     return (word >> (8u * (uint32_t)(e & 3u))) & 0xFFu;
 }
 
-/* Quantize one 32-tile that is already in fp32 (after the optional rotation).
- * Writes 32 codes (one per byte, unpacked) and returns the E8M0 scale byte. */
-static uint8_t quantize_tile(const float v[MX_BLOCK], int rounding, uint64_t e0, uint64_t seed,
-                             uint32_t tag, uint8_t code[MX_BLOCK])
+/* Largest magnitude of one 32-tile that is already in fp32 (after the optional rotation). */
+static float tile_amax(const float v[MX_BLOCK])
 {
     float amax = 0.0f;
     for (int j = 0; j < MX_BLOCK; ++j) {
         float a = fabsf(v[j]);
         if (a > amax) amax = a;
     }
+    return amax;
+}
+
+/* E8M0 byte of Eq. (1) for a block whose largest magnitude is amax:
+ * 2^(floor(log2 amax) - 2), i.e. the fp32 biased exponent minus 2, clamped to [0, 254]. */
+static uint8_t scale_byte_from_amax(float amax)
+{
     int E = (int)((float_bits(amax) >> 23) & 0xFFu);
     int byte = E - 2;
     if (byte < 0) byte = 0;
     if (byte > 254) byte = 254;
-    float mult = ldexpf(1.0f, 127 - byte);
+    return (uint8_t)byte;
+}
+
+/* Round the 32 values of a tile to E2M1 codes (one per byte, unpacked) under a given scale. */
+static void round_tile(const float v[MX_BLOCK], uint8_t byte, int rounding, uint64_t e0, uint64_t seed,
+                       uint32_t tag, uint8_t code[MX_BLOCK])
+{
+    float mult = ldexpf(1.0f, 127 - (int)byte);
     for (int j = 0; j < MX_BLOCK; ++j) {
         float s = v[j] * mult;
         float a = fabsf(s);
@@ -197,7 +209,43 @@ static uint8_t quantize_tile(const float v[MX_BLOCK], int rounding, uint64_t e0,
         int sign = (int)(float_bits(v[j]) >> 31);
         code[j] = (uint8_t)((sign << 3) | mag);
     }
-    return (uint8_t)byte;
+}
+
+/* Quantize one 32-tile (1D block: the tile is its own scale group).
+ * Writes 32 codes and returns the E8M0 scale byte. */
+static uint8_t quantize_tile(const float v[MX_BLOCK], int rounding, uint64_t e0, uint64_t seed,
+                             uint32_t tag, uint8_t code[MX_BLOCK])
+{
+    uint8_t byte = scale_byte_from_amax(tile_amax(v));
+    round_tile(v, byte, rounding, e0, seed, tag, code);
+    return byte;
+}
+
+/* One 32-tile of the operand view, widened to fp32, sign-flipped and rotated as the mode asks. */
+static void load_rotated_tile(const uint16_t* src, int64_t ld, int axis, int64_t o, int64_t t,
+                              int hadamard_mode, uint32_t mask, float v[MX_BLOCK])
+{
+    for (int j = 0; j < MX_BLOCK; ++j) {
+        int64_t k = t * MX_BLOCK + j;
+        uint16_t b = axis ? src[o * ld + k] : src[k * ld + o];
+        v[j] = bf16_bits_to_float(b);
+    }
+    if (hadamard_mode == 2 || hadamard_mode == 4) {
+        for (int j = 0; j < MX_BLOCK; ++j)
+            if ((mask >> j) & 1u) v[j] = -v[j];
+    }
+    if (hadamard_mode == 1 || hadamard_mode == 2) oracle_fwht32(v);
+    if (hadamard_mode == 3 || hadamard_mode == 4) oracle_fwht16x2(v);
+}
+
+static uint32_t mode_sign_mask(int hadamard_mode, uint64_t seed)
+{
+    if (hadamard_mode == 2) return oracle_sign_mask(seed);
+    if (hadamard_mode == 4) {
+        uint32_t m16 = oracle_sign_mask(seed) & 0xFFFFu;   /* same 16 signs for both halves */
+        return m16 | (m16 << 16);
+    }
+    return 0u;
 }
 
 /*
@@ -223,12 +271,7 @@ int oracle_quantize(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld,
     int64_t outer = axis ? rows : cols;
     int64_t K = axis ? cols : rows;
     if (outer <= 0 || K <= 0 || K % MX_BLOCK != 0 || ld < cols) return -1;
-    uint32_t mask = 0u;
-    if (hadamard_mode == 2) mask = oracle_sign_mask(seed);
-    if (hadamard_mode == 4) {
-        uint32_t m16 = oracle_sign_mask(seed) & 0xFFFFu;   /* same 16 signs for both halves */
-        mask = m16 | (m16 << 16);
-    }
+    const uint32_t mask = mode_sign_mask(hadamard_mode, seed);
     const int64_t nt = K / MX_BLOCK;
 
 #pragma omp parallel for schedule(static)
@@ -236,22 +279,61 @@ int oracle_quantize(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld,
         for (int64_t t = 0; t < nt; ++t) {
             float v[MX_BLOCK];
             uint8_t code[MX_BLOCK];
-            for (int j = 0; j < MX_BLOCK; ++j) {
-                int64_t k = t * MX_BLOCK + j;
-                uint16_t b = axis ? src[o * ld + k] : src[k * ld + o];
-                v[j] = bf16_bits_to_float(b);
-            }
-            if (hadamard_mode == 2 || hadamard_mode == 4) {
-                for (int j = 0; j < MX_BLOCK; ++j)
-                    if ((mask >> j) & 1u) v[j] = -v[j];
-            }
-            if (hadamard_mode == 1 || hadamard_mode == 2) oracle_fwht32(v);
-            if (hadamard_mode == 3 || hadamard_mode == 4) oracle_fwht16x2(v);
+            load_rotated_tile(src, ld, axis, o, t, hadamard_mode, mask, v);
             uint64_t e0 = (uint64_t)o * (uint64_t)K + (uint64_t)(t * MX_BLOCK);
             uint8_t byte = quantize_tile(v, rounding, e0, seed, tag, code);
             scales[o * nt + t] = byte;
             uint8_t* dst = codes + o * (K / 2) + t * (MX_BLOCK / 2);
             for (int j = 0; j < MX_BLOCK; j += 2) dst[j / 2] = (uint8_t)(code[j] | (code[j + 1] << 4));
+        }
+    }
+    return 0;
+}
+
+/*
+ * oracle_quantize_2d: the 32 x 32 block strategy of Appendix D.  Same operand view, rotation,
+ * rounding, code packing and canonical scale array as oracle_quantize, but ONE E8M0 scale is
+ * shared by a region of 32 consecutive operand rows x one 32-element block along K (regions are
+ * aligned to multiples of 32 in both directions; when outer is not a multiple of 32 the last
+ * region has fewer rows).  The scale comes from the largest magnitude over the whole region --
+ * of the rotated values when a rotation is on -- and is written to scales[o][t] for every row o
+ * of the region, so a consumer of 1D scales reads it unchanged.
+ */
+int oracle_quantize_2d(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, int axis,
+                       int hadamard_mode, int rounding, uint64_t seed, uint32_t tag, uint8_t* codes,
+                       uint8_t* scales)
+{
+    if (!src || !codes || !scales) return -1;
+    if (axis != 0 && axis != 1) return -1;
+    if (hadamard_mode < 0 || hadamard_mode > 4 || rounding < 0 || rounding > 1) return -1;
+    int64_t outer = axis ? rows : cols;
+    int64_t K = axis ? cols : rows;
+    if (outer <= 0 || K <= 0 || K % MX_BLOCK != 0 || ld < cols) return -1;
+    const uint32_t mask = mode_sign_mask(hadamard_mode, seed);
+    const int64_t nt = K / MX_BLOCK;
+    const int64_t groups = (outer + MX_BLOCK - 1) / MX_BLOCK;
+
+#pragma omp parallel for schedule(static)
+    for (int64_t g = 0; g < groups; ++g) {
+        const int64_t o_begin = g * MX_BLOCK;
+        const int64_t o_end = o_begin + MX_BLOCK < outer ? o_begin + MX_BLOCK : outer;
+        for (int64_t t = 0; t < nt; ++t) {
+            float v[MX_BLOCK][MX_BLOCK];
+            float amax = 0.0f;
+            for (int64_t o = o_begin; o < o_end; ++o) {
+                load_rotated_tile(src, ld, axis, o, t, hadamard_mode, mask, v[o - o_begin]);
+                float a = tile_amax(v[o - o_begin]);
+                if (a > amax) amax = a;
+            }
+            const uint8_t byte = scale_byte_from_amax(amax);
+            for (int64_t o = o_begin; o < o_end; ++o) {
+                uint8_t code[MX_BLOCK];
+                uint64_t e0 = (uint64_t)o * (uint64_t)K + (uint64_t)(t * MX_BLOCK);
+                round_tile(v[o - o_begin], byte, rounding, e0, seed, tag, code);
+                scales[o * nt + t] = byte;
+                uint8_t* dst = codes + o * (K / 2) + t * (MX_BLOCK / 2);
+                for (int j = 0; j < MX_BLOCK; j += 2) dst[j / 2] = (uint8_t)(code[j] | (code[j + 1] << 4));
+            }
         }
     }
     return 0;
