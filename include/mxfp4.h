@@ -59,6 +59,9 @@ extern "C" {
 #define MXFP4_SCALES_CANONICAL 0 /* scales[o][t], row-major, outer x K/32 bytes               */
 #define MXFP4_SCALES_TILED 1     /* 128-row x 4-block tiles of 512 bytes (what the GEMM reads)*/
 
+#define MXFP4_BLOCK_1X32 0  /* one scale per 32 elements along K (Appendix D, 1D)               */
+#define MXFP4_BLOCK_32X32 1 /* one scale per 32 operand rows x 32 elements (Appendix D, 2D)      */
+
 #define MXFP4_OUT_BF16 0
 #define MXFP4_OUT_FP32 1
 
@@ -109,6 +112,41 @@ size_t mxfp4_scales_bytes(int64_t outer, int64_t K, int scale_layout);
 int mxfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis,
                    int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
                    void* codes, void* scales, int scale_layout, void* stream);
+
+/*
+ * mxfp4_quantize_2d -- mxfp4_quantize with the 32 x 32 block strategy of Appendix D: one E8M0
+ * scale is shared by 32 consecutive operand rows x one 32-element block along K (regions aligned
+ * to multiples of 32 both ways; a last region may have fewer rows).  The scale comes from the
+ * largest magnitude in the region -- of the rotated values when hadamard_mode != 0 -- and is
+ * written into the scale entry of every row of the region, so codes and scales have exactly the
+ * format of mxfp4_quantize and feed mxfp4_gemm unchanged.  With hadamard_mode 0 the result is
+ * transpose-invariant: axis ROWS gives the transposed codes and scales of axis COLS.
+ * Arguments, shapes, alignment and errors as mxfp4_quantize.
+ */
+int mxfp4_quantize_2d(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis,
+                      int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
+                      void* codes, void* scales, int scale_layout, void* stream);
+
+/*
+ * mxfp4_quantize_dual -- both orientations of one tensor from ONE read of it (Appendix D; a
+ * linear layer uses each of X, W, dY once blocked along its rows and once down its columns,
+ * Appendix C).  Writes
+ *   codes_rowwise / scales_rowwise : the operand of mxfp4_quantize(axis = MXFP4_AXIS_COLS),
+ *                                    [rows x cols/2] bytes, stochastic-rounding tag tag_rowwise;
+ *   codes_colwise / scales_colwise : the operand of mxfp4_quantize(axis = MXFP4_AXIS_ROWS),
+ *                                    the transposed operand [cols x rows/2] bytes, tag tag_colwise;
+ * each bit-identical to the single-axis call (block_shape MXFP4_BLOCK_1X32) or to
+ * mxfp4_quantize_2d (MXFP4_BLOCK_32X32) with the same rotation, rounding and seed.
+ * rows and cols must both be multiples of 32 (both are reduction axes), ld_src a multiple of 8;
+ * all five pointers are device pointers, 16-byte aligned; scale buffers are sized with
+ * mxfp4_scales_bytes(rows, cols, layout) and mxfp4_scales_bytes(cols, rows, layout).
+ * Algorithmic traffic: 2 + 2 * (1/2 + 1/32) = 3.0625 bytes per element instead of 5.0625 for
+ * two single-axis calls.  Nothing is launched on error.
+ */
+int mxfp4_quantize_dual(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int hadamard_mode,
+                        int rounding, uint64_t seed, uint32_t tag_rowwise, uint32_t tag_colwise,
+                        int block_shape, void* codes_rowwise, void* scales_rowwise, void* codes_colwise,
+                        void* scales_colwise, int scale_layout, void* stream);
 
 /*
  * mxfp4_quantize_pair -- mxfp4_quantize for two tensors in ONE kernel launch (the two operands

@@ -16,13 +16,14 @@ from . import build as _build
 HADAMARD_NONE, HADAMARD_DET, HADAMARD_RAND, HADAMARD_DET16, HADAMARD_RAND16 = 0, 1, 2, 3, 4
 ROUND_RNE, ROUND_SR = 0, 1
 SCALES_CANONICAL, SCALES_TILED = 0, 1
+BLOCK_1X32, BLOCK_32X32 = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
 PASS_FPROP, PASS_DGRAD, PASS_WGRAD = 0, 1, 2
 AXIS_ROWS, AXIS_COLS = 0, 1
 
 EXPORTS = (
     "mxfp4_version", "mxfp4_status_string", "mxfp4_codes_bytes", "mxfp4_scales_bytes",
-    "mxfp4_quantize", "mxfp4_quantize_pair", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
+    "mxfp4_quantize", "mxfp4_quantize_2d", "mxfp4_quantize_dual", "mxfp4_quantize_pair", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
     "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_host", "mxfp4_linear_static",
     "mxfp4_check", "mxfp4_selftest_wait_timeout",
 )
@@ -69,6 +70,10 @@ def load_library() -> ctypes.CDLL:
     lib.mxfp4_scales_bytes.argtypes, lib.mxfp4_scales_bytes.restype = [i64, i64, ci], sz
     lib.mxfp4_quantize.argtypes = [vp, i64, i64, i64, ci, ci, ci, u64, u32, vp, vp, ci, vp]
     lib.mxfp4_quantize.restype = ci
+    lib.mxfp4_quantize_2d.argtypes = lib.mxfp4_quantize.argtypes
+    lib.mxfp4_quantize_2d.restype = ci
+    lib.mxfp4_quantize_dual.argtypes = [vp, i64, i64, i64, ci, ci, u64, u32, u32, ci, vp, vp, vp, vp, ci, vp]
+    lib.mxfp4_quantize_dual.restype = ci
     lib.mxfp4_quantize_pair.argtypes = [ctypes.POINTER(QuantDesc), ctypes.POINTER(QuantDesc), ci, ci, u64, ci, vp]
     lib.mxfp4_quantize_pair.restype = ci
     lib.mxfp4_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, ctypes.c_float, vp, ci, i64, vp, sz, vp]
@@ -128,8 +133,9 @@ def _raise(rc: int, what: str):
 def quantize(src: torch.Tensor, axis: int = AXIS_COLS, hadamard_mode: int = HADAMARD_NONE,
              rounding: int = ROUND_RNE, seed: int = 0, operand_tag: int = 0,
              scale_layout: int = SCALES_TILED, codes: torch.Tensor | None = None,
-             scales: torch.Tensor | None = None):
-    """``mxfp4_quantize`` on a 2-D bf16 CUDA tensor (rows may be strided: ``ld = stride(0)``).
+             scales: torch.Tensor | None = None, block_shape: int = 0):
+    """``mxfp4_quantize`` (``block_shape`` BLOCK_1X32) or ``mxfp4_quantize_2d`` (BLOCK_32X32) on a
+    2-D bf16 CUDA tensor (rows may be strided: ``ld = stride(0)``).
 
     Returns ``(codes uint8 [outer, K/2], scales uint8 [scales_bytes])``; output tensors are
     allocated with torch unless passed in.
@@ -146,11 +152,40 @@ def quantize(src: torch.Tensor, axis: int = AXIS_COLS, hadamard_mode: int = HADA
     if scales is None:
         scales = torch.empty(scales_bytes(outer, K, scale_layout), dtype=torch.uint8, device=src.device)
     ld = src.stride(0) if rows > 1 else cols   # a single row's stride is arbitrary in torch
-    rc = lib.mxfp4_quantize(_dev_ptr(src), rows, cols, ld, axis, hadamard_mode, rounding,
-                            ctypes.c_uint64(seed), ctypes.c_uint32(operand_tag), _dev_ptr(codes),
-                            _dev_ptr(scales), scale_layout, _stream())
+    fn = lib.mxfp4_quantize_2d if block_shape == BLOCK_32X32 else lib.mxfp4_quantize
+    rc = fn(_dev_ptr(src), rows, cols, ld, axis, hadamard_mode, rounding,
+            ctypes.c_uint64(seed), ctypes.c_uint32(operand_tag), _dev_ptr(codes),
+            _dev_ptr(scales), scale_layout, _stream())
     _raise(rc, "mxfp4_quantize")
     return codes, scales
+
+
+def quantize_dual(src: torch.Tensor, hadamard_mode: int = HADAMARD_NONE, rounding: int = ROUND_RNE,
+                  seed: int = 0, tags=(0, 1), block_shape: int = 0, scale_layout: int = SCALES_TILED,
+                  out_row=None, out_col=None):
+    """``mxfp4_quantize_dual``: row-wise and column-wise operands of ``src`` from one read.
+
+    Returns ``((codes [rows, cols/2], scales), (codes [cols, rows/2], scales))``; ``out_row`` /
+    ``out_col`` are optional ``(codes, scales)`` tensors to write into.
+    """
+    if src.dtype != torch.bfloat16 or src.dim() != 2 or src.stride(1) != 1:
+        raise ValueError("src must be a 2-D bf16 tensor with contiguous rows")
+    rows, cols = src.shape
+    lib = load_library()
+    if rows % 32 != 0 or cols % 32 != 0 or rows <= 0 or cols <= 0:
+        _raise(-2, "mxfp4_quantize_dual")
+    cr, sr = out_row if out_row is not None else (
+        torch.empty((rows, cols // 2), dtype=torch.uint8, device=src.device),
+        torch.empty(scales_bytes(rows, cols, scale_layout), dtype=torch.uint8, device=src.device))
+    cc, sc = out_col if out_col is not None else (
+        torch.empty((cols, rows // 2), dtype=torch.uint8, device=src.device),
+        torch.empty(scales_bytes(cols, rows, scale_layout), dtype=torch.uint8, device=src.device))
+    rc = lib.mxfp4_quantize_dual(_dev_ptr(src), rows, cols, src.stride(0), hadamard_mode, rounding,
+                                 ctypes.c_uint64(seed), ctypes.c_uint32(tags[0]), ctypes.c_uint32(tags[1]),
+                                 block_shape, _dev_ptr(cr), _dev_ptr(sr), _dev_ptr(cc), _dev_ptr(sc),
+                                 scale_layout, _stream())
+    _raise(rc, "mxfp4_quantize_dual")
+    return (cr, sr), (cc, sc)
 
 
 def _quant_desc(src, axis, tag, scale_layout, codes, scales):

@@ -10,6 +10,7 @@
 #include "ptx_sm100.cuh"
 #include "tma_host.cuh"
 #include "quantize_kernel.cuh"
+#include "quantize_dual_kernel.cuh"
 #include "gemm_pair_kernel.cuh"
 
 namespace mxfp4 {
@@ -96,10 +97,33 @@ static int dispatch_quantize(int hmode, int sr, const QuantJob& j0, const QuantJ
     }
 }
 
+static void fill_quant_params(QuantParams* pp, int64_t outer, int64_t K, int hadamard_mode, uint64_t seed,
+                              uint32_t operand_tag, void* scales, int scale_layout, int block2d)
+{
+    QuantParams& p = *pp;
+    p.scales = static_cast<uint8_t*>(scales);
+    p.outer = outer;
+    p.K = K;
+    p.nt = K / 32;
+    p.tiles_o = static_cast<int32_t>((outer + kQTileO - 1) / kQTileO);
+    p.tiles_k = static_cast<int32_t>((K + kQTileK - 1) / kQTileK);
+    p.seed_lo = static_cast<uint32_t>(seed);
+    p.seed_hi = static_cast<uint32_t>(seed >> 32);
+    p.tag = operand_tag;
+    p.sign_mask = 0u;
+    if (hadamard_mode == MXFP4_HADAMARD_RAND) p.sign_mask = host_sign_mask(seed);
+    if (hadamard_mode == MXFP4_HADAMARD_RAND16) {
+        const uint32_t m16 = host_sign_mask(seed) & 0xFFFFu;   // same 16 signs for both halves
+        p.sign_mask = m16 | (m16 << 16);
+    }
+    p.scale_layout = scale_layout;
+    p.block2d = block2d;
+}
+
 // Validates one tensor's arguments and fills its job (tensor maps + parameters).
 static int build_quant_job(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis,
                            int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
-                           void* codes, void* scales, int scale_layout, QuantJob* job)
+                           void* codes, void* scales, int scale_layout, QuantJob* job, int block2d = 0)
 {
     if (!src_bf16 || !codes || !scales) return MXFP4_ERR_NULL;
     if (axis != 0 && axis != 1) return MXFP4_ERR_ENUM;
@@ -126,22 +150,7 @@ static int build_quant_job(const void* src_bf16, int64_t rows, int64_t cols, int
     if (!ok_src || !ok_codes) return MXFP4_ERR_CUDA;
 
     QuantParams& p = job->p;
-    p.scales = static_cast<uint8_t*>(scales);
-    p.outer = outer;
-    p.K = K;
-    p.nt = K / 32;
-    p.tiles_o = static_cast<int32_t>((outer + kQTileO - 1) / kQTileO);
-    p.tiles_k = static_cast<int32_t>((K + kQTileK - 1) / kQTileK);
-    p.seed_lo = static_cast<uint32_t>(seed);
-    p.seed_hi = static_cast<uint32_t>(seed >> 32);
-    p.tag = operand_tag;
-    p.sign_mask = 0u;
-    if (hadamard_mode == MXFP4_HADAMARD_RAND) p.sign_mask = host_sign_mask(seed);
-    if (hadamard_mode == MXFP4_HADAMARD_RAND16) {
-        const uint32_t m16 = host_sign_mask(seed) & 0xFFFFu;   // same 16 signs for both halves
-        p.sign_mask = m16 | (m16 << 16);
-    }
-    p.scale_layout = scale_layout;
+    fill_quant_params(&p, outer, K, hadamard_mode, seed, operand_tag, scales, scale_layout, block2d);
     const int64_t total = static_cast<int64_t>(p.tiles_o) * p.tiles_k;
     if (total > 0x3FFFFFFF) return MXFP4_ERR_SHAPE;
     job->tiles = static_cast<int32_t>(total);
@@ -160,6 +169,23 @@ static int launch_quant_jobs(const QuantJob& j0, const QuantJob& j1, int axis0, 
     if (axis0 == 1 && axis1 == 0) return dispatch_quantize<1, 0>(hmode, sr, j0, j1, grid, st);
     if (axis0 == 0 && axis1 == 0) return dispatch_quantize<0, 0>(hmode, sr, j0, j1, grid, st);
     return MXFP4_ERR_ENUM;   // (0, 1) is never asked for: callers order row-wise first
+}
+
+template <int HMODE, int SR>
+static int launch_quantize_dual(const QuantDualJob& job, int grid, cudaStream_t stream)
+{
+    const size_t smem = sizeof(QuantDualSmem) + 1024;
+    static bool attr_set[64] = {};          // the attribute is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(quantize_dual_kernel<HMODE, SR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess)
+            return MXFP4_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    quantize_dual_kernel<HMODE, SR><<<grid, kQThreads, smem, stream>>>(job);
+    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
 static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -231,6 +257,69 @@ int mxfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_
     if (rc != MXFP4_OK) return rc;
     memset(&j1, 0, sizeof(j1));
     return launch_quant_jobs(j0, j1, axis, axis, hadamard_mode, rounding, static_cast<cudaStream_t>(stream));
+}
+
+int mxfp4_quantize_2d(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis,
+                      int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
+                      void* codes, void* scales, int scale_layout, void* stream)
+{
+    QuantJob j0, j1;
+    const int rc = build_quant_job(src_bf16, rows, cols, ld_src, axis, hadamard_mode, rounding, seed,
+                                   operand_tag, codes, scales, scale_layout, &j0, 1);
+    if (rc != MXFP4_OK) return rc;
+    memset(&j1, 0, sizeof(j1));
+    return launch_quant_jobs(j0, j1, axis, axis, hadamard_mode, rounding, static_cast<cudaStream_t>(stream));
+}
+
+int mxfp4_quantize_dual(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int hadamard_mode,
+                        int rounding, uint64_t seed, uint32_t tag_rowwise, uint32_t tag_colwise,
+                        int block_shape, void* codes_rowwise, void* scales_rowwise, void* codes_colwise,
+                        void* scales_colwise, int scale_layout, void* stream)
+{
+    if (!src_bf16 || !codes_rowwise || !scales_rowwise || !codes_colwise || !scales_colwise) return MXFP4_ERR_NULL;
+    if (hadamard_mode < 0 || hadamard_mode > 4 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
+    if (scale_layout != 0 && scale_layout != 1) return MXFP4_ERR_ENUM;
+    if (block_shape != MXFP4_BLOCK_1X32 && block_shape != MXFP4_BLOCK_32X32) return MXFP4_ERR_ENUM;
+    if (rows <= 0 || cols <= 0 || ld_src < cols) return MXFP4_ERR_SHAPE;
+    if (rows % 32 != 0 || cols % 32 != 0) return MXFP4_ERR_SHAPE;      // both axes are reduction axes here
+    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (!aligned16(src_bf16) || !aligned16(codes_rowwise) || !aligned16(scales_rowwise) ||
+        !aligned16(codes_colwise) || !aligned16(scales_colwise))
+        return MXFP4_ERR_ALIGN;
+    if (ld_src % 8 != 0) return MXFP4_ERR_ALIGN;
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return MXFP4_ERR_CUDA;
+    if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
+
+    QuantDualJob job;
+    const bool ok = make_tmap_2d(&job.tm_src, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, src_bf16, rows, cols, ld_src * 2,
+                                 128, 64, CU_TENSOR_MAP_SWIZZLE_128B) &&
+                    make_tmap_2d(&job.tm_codes_row, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes_rowwise, rows, cols / 2,
+                                 cols / 2, 128, 64, CU_TENSOR_MAP_SWIZZLE_64B) &&
+                    make_tmap_2d(&job.tm_codes_col, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes_colwise, cols, rows / 2,
+                                 rows / 2, 128, 64, CU_TENSOR_MAP_SWIZZLE_64B);
+    if (!ok) return MXFP4_ERR_CUDA;
+    const int b2d = block_shape == MXFP4_BLOCK_32X32;
+    fill_quant_params(&job.pr, rows, cols, hadamard_mode, seed, tag_rowwise, scales_rowwise, scale_layout, b2d);
+    fill_quant_params(&job.pc, cols, rows, hadamard_mode, seed, tag_colwise, scales_colwise, scale_layout, b2d);
+    job.tiles_r = job.pr.tiles_o;
+    job.tiles_c = job.pr.tiles_k;
+    const int64_t total = static_cast<int64_t>(job.tiles_r) * job.tiles_c;
+    if (total > 0x3FFFFFFF) return MXFP4_ERR_SHAPE;
+    const int grid = static_cast<int>(total < dev.sm_count ? total : dev.sm_count);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (hadamard_mode * 2 + rounding) {
+        case 0: return launch_quantize_dual<0, 0>(job, grid, st);
+        case 1: return launch_quantize_dual<0, 1>(job, grid, st);
+        case 2: return launch_quantize_dual<1, 0>(job, grid, st);
+        case 3: return launch_quantize_dual<1, 1>(job, grid, st);
+        case 4: return launch_quantize_dual<2, 0>(job, grid, st);
+        case 5: return launch_quantize_dual<2, 1>(job, grid, st);
+        case 6: return launch_quantize_dual<3, 0>(job, grid, st);
+        case 7: return launch_quantize_dual<3, 1>(job, grid, st);
+        case 8: return launch_quantize_dual<4, 0>(job, grid, st);
+        default: return launch_quantize_dual<4, 1>(job, grid, st);
+    }
 }
 
 int mxfp4_quantize_pair(const mxfp4_quant_desc* a, const mxfp4_quant_desc* b, int hadamard_mode,

@@ -52,6 +52,7 @@ struct QuantParams {
     int32_t tiles_o, tiles_k;
     uint32_t seed_lo, seed_hi, tag, sign_mask;
     int32_t scale_layout;    // 0 canonical, 1 tiled
+    int32_t block2d;         // 0: 1 x 32 blocks, 1: 32 x 32 blocks (scale shared by 32 operand rows)
 };
 
 // One tensor to quantize: its source and code tensor maps plus parameters.  A launch takes two
@@ -193,11 +194,9 @@ __device__ __forceinline__ void load_block(const uint8_t* stage, int kb, int o, 
     }
 }
 
-// Remaining butterfly stages, block maximum, scale byte, rounding: block in, 16 bytes of packed
-// codes and the E8M0 byte out.  e0 = index of the block's first element in the operand view.
-template <int HMODE, int SR>
-__device__ __forceinline__ void quantize_block(float2 (&P)[16], uint64_t e0, const QuantParams& p,
-                                               uint32_t (&packed)[4], uint32_t& byte)
+// Remaining butterfly stages and the block maximum.
+template <int HMODE>
+__device__ __forceinline__ float rotate_and_amax(float2 (&P)[16])
 {
     if (HMODE != 0) {
         fwht32_pair_stage<1>(P);
@@ -208,7 +207,22 @@ __device__ __forceinline__ void quantize_block(float2 (&P)[16], uint64_t e0, con
     float amax = max3_abs(P[0].x, P[0].y, P[1].x);
 #pragma unroll
     for (int i = 1; i < 15; ++i) amax = max3_abs(amax, P[i].y, P[i + 1].x);
-    amax = fmaxf(amax, fabsf(P[15].y));
+    return fmaxf(amax, fabsf(P[15].y));
+}
+
+// Largest of a non-negative float over the lanes named by `mask` (bit patterns of non-negative
+// floats order like unsigned integers).
+__device__ __forceinline__ float lanes_max(uint32_t mask, float v)
+{
+    return __uint_as_float(__reduce_max_sync(mask, __float_as_uint(v)));
+}
+
+// Scale byte from the block maximum, scaling, rounding, packing: 16 bytes of packed codes and
+// the E8M0 byte out.  e0 = index of the block's first element in the operand view.
+template <int SR>
+__device__ __forceinline__ void scale_round_pack(const float2 (&P)[16], float amax, uint64_t e0,
+                                                 const QuantParams& p, uint32_t (&packed)[4], uint32_t& byte)
+{
     const uint32_t E = __float_as_uint(amax) >> 23;
     byte = E > 2u ? E - 2u : 0u;                  // E <= 255 keeps byte <= 253 < 255
     const float mult = __uint_as_float((254u - byte) << 23);
@@ -226,7 +240,7 @@ __device__ __forceinline__ void quantize_block(float2 (&P)[16], uint64_t e0, con
             packed[q] = cvt_e2m1x8(v[8 * q], v[8 * q + 1], v[8 * q + 2], v[8 * q + 3], v[8 * q + 4],
                                    v[8 * q + 5], v[8 * q + 6], v[8 * q + 7]);
     } else {
-        const uint64_t g = e0 >> 4;
+        const uint64_t g = e0 >> 4;                 // two 16-element Philox groups per block
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             uint32_t r[4];
@@ -246,6 +260,17 @@ __device__ __forceinline__ void quantize_block(float2 (&P)[16], uint64_t e0, con
             }
         }
     }
+}
+
+// One block owned by one thread, whose warp holds 32 consecutive operand rows of the same block
+// column: with 32 x 32 blocks (Appendix D) the maximum is taken over the warp.
+template <int HMODE, int SR>
+__device__ __forceinline__ void quantize_block(float2 (&P)[16], uint64_t e0, const QuantParams& p,
+                                               uint32_t (&packed)[4], uint32_t& byte)
+{
+    float amax = rotate_and_amax<HMODE>(P);
+    if (p.block2d) amax = lanes_max(0xFFFFFFFFu, amax);
+    scale_round_pack<SR>(P, amax, e0, p, packed, byte);
 }
 
 // tile index of a job -> (operand-row tile, K tile); the fastest-varying index walks the source's
