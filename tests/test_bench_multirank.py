@@ -21,7 +21,7 @@ WORKER = textwrap.dedent("""
     assert bench.aggregate_over_ranks(3.0, 1) == 3.0
     dist.barrier()
     dist.destroy_process_group()
-    print("rank", rank, "ok")
+    sys.stdout.write("rank%d-ok\n" % rank)     # one write per rank: the two ranks share a pipe
 """) % ROOT
 
 
@@ -37,7 +37,7 @@ def test_max_over_ranks_with_two_gloo_ranks(tmp_path):
          "--master-addr", "127.0.0.1", "--master-port", str(port), str(script)],
         capture_output=True, text=True, timeout=240, env=env)
     assert res.returncode == 0, res.stdout + res.stderr
-    assert "rank 0 ok" in res.stdout and "rank 1 ok" in res.stdout
+    assert "rank0-ok" in res.stdout and "rank1-ok" in res.stdout
 
 
 def test_reference_arm_exits_quietly_on_other_ranks():
