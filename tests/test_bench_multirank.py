@@ -21,7 +21,7 @@ WORKER = textwrap.dedent("""
     assert bench.aggregate_over_ranks(3.0, 1) == 3.0
     dist.barrier()
     dist.destroy_process_group()
-    sys.stdout.write("rank" + str(rank) + "-ok\n")     # one write per rank: the two ranks share a pipe
+    print("rank" + str(rank) + "-ok")              # one token per rank: the two ranks share a pipe
 """) % ROOT
 
 
