@@ -4,12 +4,15 @@
 One "step" is one pass of the whole hot path -- Hadamard + quantize of both operands and the
 block-scaled GEMM, for Fprop, Dgrad and Wgrad of every linear of the workload -- over one batch
 of seeded synthetic tensors shaped like Llama-3.1-8B layers.  The default workload is the full
-layer linear stack at 16384 tokens (12 fused passes, each one two-tensor quantize launch + one
-GEMM launch), the one
-configuration that exercises every step of the path; ``--workload qkv|gate_up|down`` selects
-the single-linear configurations.
+layer linear stack at 16384 tokens (4 linears x 3 passes = 12 GEMMs), the one configuration that
+exercises every step of the path; ``--workload qkv|gate_up|down`` selects the single-linear
+configurations.  ``--schedule layer`` (default) runs each linear as forward + backward with every
+tensor read once by the dual-axis quantize (3 quantize + 3 GEMM launches per linear);
+``--schedule per_pass`` runs the three per-pass entry points (one two-tensor quantize launch + one
+GEMM launch each).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload W] [--schedule S]
+                    [--impl ours|reference]
 
 Prints ONE JSON line.  ``value`` is whole-job TFLOP/s (2*M*N*K per GEMM, quantize time
 included) with inputs resident in HBM; ``e2e`` is the same metric through the host-buffer
@@ -241,14 +244,40 @@ def run_ours(args):
         passes.append((n, 2, d["dY"], d["X"]) + pass_dims(2, tokens, i, o))
     flops_per_step = sum(2.0 * M * N * K for (_, _, _, _, M, N, K) in passes)
     fused = [lib.mxfp4_linear_fprop, lib.mxfp4_linear_dgrad, lib.mxfp4_linear_wgrad]
+    layer = args.schedule == "layer"
+    if layer:
+        saved_bytes = max(api.linear_layer_bytes(tokens, i, o, api.LAYER_SAVED) for o, i in dims.values())
+        lws_bytes = max(api.linear_layer_bytes(tokens, i, o, w) for o, i in dims.values()
+                        for w in (api.LAYER_FORWARD, api.LAYER_BACKWARD))
+        saved = torch.empty(saved_bytes, dtype=torch.uint8, device="cuda")
+        lws = torch.empty(lws_bytes, dtype=torch.uint8, device="cuda")
+        out_buf2 = torch.empty(max_out, dtype=torch.bfloat16, device="cuda")
 
-    def step():
+    def step_per_pass():
         for (n, p, a, b, M, N, K) in passes:
             o, i = dims[n]
             rc = fused[p](a.data_ptr(), b.data_ptr(), out_buf.data_ptr(), tokens, i, o, hmode, rnd, seed,
                           api.OUT_BF16, ws.data_ptr(), ws_bytes, sptr)
             if rc != 0:
                 raise api.Mxfp4Error(rc, "fused linear pass")
+
+    def step_layer():
+        # forward then backward of each linear: X, W and dY are each read once
+        for n in names:
+            o, i = dims[n]
+            d = dev_in[n]
+            rc = lib.mxfp4_linear_forward(d["X"].data_ptr(), d["W"].data_ptr(), out_buf.data_ptr(), tokens, i, o,
+                                          hmode, rnd, seed, api.OUT_BF16, saved.data_ptr(), saved_bytes,
+                                          lws.data_ptr(), lws_bytes, sptr)
+            if rc != 0:
+                raise api.Mxfp4Error(rc, "mxfp4_linear_forward")
+            rc = lib.mxfp4_linear_backward(d["dY"].data_ptr(), out_buf.data_ptr(), out_buf2.data_ptr(), tokens, i, o,
+                                           hmode, rnd, seed, api.OUT_BF16, api.OUT_BF16, saved.data_ptr(),
+                                           saved_bytes, lws.data_ptr(), lws_bytes, sptr)
+            if rc != 0:
+                raise api.Mxfp4Error(rc, "mxfp4_linear_backward")
+
+    step = step_layer if layer else step_per_pass
 
     def sync_all():
         torch.cuda.synchronize()
@@ -276,37 +305,76 @@ def run_ours(args):
     api.check()
 
     # ---- the same step, decomposed, with CUDA events around every launch (roofline inputs)
+    q_bytes_per_element = 3.0625 if layer else 2.53125
+
     def a_b_axes(p):
         return ((1, 1), (1, 0), (0, 0))[p]
 
     gemm_ms = gemm_flops = quant_ms = quant_bytes = 0.0
+    n_quant = 0
+    r256 = lambda v: (v + 255) // 256 * 256
+
+    def operand_views(buf, off, outer, K):
+        """(codes, scales, next offset) inside a byte buffer, as the library lays operands out."""
+        c = buf[off: off + outer * K // 2].view(outer, K // 2)
+        off += r256(outer * K // 2)
+        sb = api.scales_bytes(outer, K)
+        return c, buf[off: off + sb], off + r256(sb)
+
     for rep in range(2):
         evs = []
-        for (n, p, a, b, M, N, K) in passes:
-            ax_a, ax_b = a_b_axes(p)
-            ac = ws[: M * K // 2].view(M, K // 2)
-            off = (M * K // 2 + 255) // 256 * 256
-            asz = api.scales_bytes(M, K)
-            a_s = ws[off: off + asz]
-            off = off + (asz + 255) // 256 * 256
-            bc = ws[off: off + N * K // 2].view(N, K // 2)
-            off = off + (N * K // 2 + 255) // 256 * 256
-            b_s = ws[off: off + api.scales_bytes(N, K)]
-            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-            ev[0].record(stream)
-            api.quantize_pair(a, ax_a, b, ax_b, hmode, rnd, seed, tags=(0, 1), out_a=(ac, a_s), out_b=(bc, b_s))
-            ev[1].record(stream)
-            api.gemm(ac, a_s, bc, b_s, alpha, api.OUT_BF16, out=out_buf[: M * N].view(M, N))
-            ev[2].record(stream)
-            evs.append((ev, M, N, K))
+        if layer:
+            for n in names:
+                o, i = dims[n]
+                d = dev_in[n]
+                T = tokens
+                xr_c, xr_s, off = operand_views(lws, 0, T, i)
+                wr_c, wr_s, _ = operand_views(lws, off, o, i)
+                xt_c, xt_s, off = operand_views(saved, 0, i, T)
+                wt_c, wt_s, _ = operand_views(saved, off, i, o)
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(8)]
+                ev[0].record(stream)
+                api.quantize_dual(d["X"], hmode, rnd, seed, tags=(0, 1), out_row=(xr_c, xr_s), out_col=(xt_c, xt_s))
+                ev[1].record(stream)
+                api.quantize_dual(d["W"], hmode, rnd, seed, tags=(1, 1), out_row=(wr_c, wr_s), out_col=(wt_c, wt_s))
+                ev[2].record(stream)
+                api.gemm(xr_c, xr_s, wr_c, wr_s, alpha, api.OUT_BF16, out=out_buf[: T * o].view(T, o))
+                ev[3].record(stream)
+                dy_c, dy_s, off = operand_views(lws, 0, T, o)
+                dyt_c, dyt_s, _ = operand_views(lws, off, o, T)
+                ev[4].record(stream)
+                api.quantize_dual(d["dY"], hmode, rnd, seed, tags=(0, 0), out_row=(dy_c, dy_s), out_col=(dyt_c, dyt_s))
+                ev[5].record(stream)
+                api.gemm(dy_c, dy_s, wt_c, wt_s, alpha, api.OUT_BF16, out=out_buf[: T * i].view(T, i))
+                ev[6].record(stream)
+                api.gemm(dyt_c, dyt_s, xt_c, xt_s, alpha, api.OUT_BF16, out=out_buf2[: o * i].view(o, i))
+                ev[7].record(stream)
+                evs.append(([(ev[0], ev[1], T * i), (ev[1], ev[2], o * i), (ev[4], ev[5], T * o)],
+                            [(ev[2], ev[3], 2.0 * T * o * i), (ev[5], ev[6], 2.0 * T * o * i),
+                             (ev[6], ev[7], 2.0 * T * o * i)]))
+        else:
+            for (n, p, a, b, M, N, K) in passes:
+                ax_a, ax_b = a_b_axes(p)
+                ac, a_s, off = operand_views(ws, 0, M, K)
+                bc, b_s, _ = operand_views(ws, off, N, K)
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+                ev[0].record(stream)
+                api.quantize_pair(a, ax_a, b, ax_b, hmode, rnd, seed, tags=(0, 1), out_a=(ac, a_s), out_b=(bc, b_s))
+                ev[1].record(stream)
+                api.gemm(ac, a_s, bc, b_s, alpha, api.OUT_BF16, out=out_buf[: M * N].view(M, N))
+                ev[2].record(stream)
+                evs.append(([(ev[0], ev[1], (M + N) * K)], [(ev[1], ev[2], 2.0 * M * N * K)]))
         torch.cuda.synchronize()
         if rep == 0:
             continue   # first decomposed pass is a warm-up
-        for ev, M, N, K in evs:
-            quant_ms += ev[0].elapsed_time(ev[1])
-            quant_bytes += (M + N) * K * 2.53125
-            gemm_ms += ev[1].elapsed_time(ev[2])
-            gemm_flops += 2.0 * M * N * K
+        for qs, gs in evs:
+            for a0, a1, elems in qs:
+                quant_ms += a0.elapsed_time(a1)
+                quant_bytes += elems * q_bytes_per_element
+                n_quant += 1
+            for a0, a1, fl in gs:
+                gemm_ms += a0.elapsed_time(a1)
+                gemm_flops += fl
     clocks = sampler.stop(t_begin, t_end)
     api.check()
 
@@ -359,14 +427,16 @@ def run_ours(args):
         "flops_per_launch": gemm_flops / n_gemm, "avg_launch_ms": gemm_ms / n_gemm,
     }
     quant_gbs = quant_bytes / (quant_ms * 1e-3) / 1e9
-    quantize_info = {"kernel": "quantize_kernel", "bound": "hbm", "achieved": quant_gbs,
-                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"],
-                     "bytes_per_element": 2.53125, "avg_launch_ms": quant_ms / n_gemm,
-                     "tensors_per_launch": 2,
-                     # ncu on the 117.4 M-element tensor: 234.9 MB read + 45.4 MB written = 2.39 B per
-                     # element (reads = source bytes exactly; part of the output is still in L2 when
-                     # the kernel ends); traffic is proportional to elements, scaled to the mean launch
-                     "traffic": 2.39 * quant_bytes / 2.53125 / n_gemm}
+    # ncu, single-axis kernel on a 117.4 M-element tensor: 234.9 MB read + 45.4 MB written = 2.39 B
+    # per element (reads = source bytes exactly; part of the output is still in L2 when the kernel
+    # ends); the dual-axis kernel reads the same 2 B and writes twice the codes.  Traffic is
+    # proportional to elements, so it is scaled to the mean launch.
+    traffic_per_element = 2.39 + (0.39 if layer else 0.0)
+    quantize_info = {"kernel": "quantize_dual_kernel" if layer else "quantize_kernel", "bound": "hbm",
+                     "achieved": quant_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": quant_gbs / peaks["hbm_gbs"], "bytes_per_element": q_bytes_per_element,
+                     "avg_launch_ms": quant_ms / n_quant, "launches_per_step": n_quant,
+                     "traffic": traffic_per_element * quant_bytes / q_bytes_per_element / n_quant}
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region
     e2e = None
@@ -452,12 +522,14 @@ def run_ours(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "e2m1 (mxfp4) x e2m1, f32 accumulate",
         "data": "synthetic",
         "config": {"workload": workload_label(args.workload, tokens, args.hadamard), "passes_per_step": len(passes),
+                   "schedule": ("layer: forward + backward per linear, each of X, W, dY read once by the dual-axis "
+                                "quantize" if layer else "per pass: both operands of each pass quantized from bf16"),
                    "flops_per_step": flops_per_step, "out_dtype": "bf16",
                    "l2": "inputs larger than L2 (several GB per step), no flush needed",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "roofline": roofline, "quantize": quantize_info,
         "frac_of_nominal_fp4_peak": world and (flops_per_step / (ms_per_step * 1e-3) / 1e12) / 9000.0,
-        "cpu_baseline": cpu_base, "e2e": e2e, "gpu_launches": 2 * len(passes) * args.steps,
+        "cpu_baseline": cpu_base, "e2e": e2e, "gpu_launches": 2 * len(passes) * args.steps,   # per linear: 3 quantize + 3 GEMM (layer) or 3 x (1 + 1)
         "clocks": clocks, "context": context, "per_config": per_config,
     }
     print(json.dumps(line))
@@ -466,6 +538,9 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--schedule", default="layer", choices=["layer", "per_pass"],
+                    help="layer: mxfp4_linear_forward/backward (each tensor read once); per_pass: the three "
+                         "per-pass entry points")
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -213,6 +213,36 @@ int mxfp4_linear_wgrad(const void* dY, const void* X, void* dW, int64_t T, int64
                        int out_dtype, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Layer-level form of the same three passes (Appendix C), each tensor read ONCE: a linear layer
+ * uses X, W and dY each in both block orientations (X: Fprop + Wgrad, W: Fprop + Dgrad,
+ * dY: Dgrad + Wgrad), so the forward call quantizes X and W with mxfp4_quantize_dual, runs the
+ * Fprop GEMM and keeps the column-wise operands (X^T, W^T as MXFP4 codes + scales: 0.53 bytes
+ * per element instead of the bf16 tensors) in `saved` for the backward call, which quantizes dY
+ * once for both of its GEMMs.  Y, dX and dW are bit-identical to mxfp4_linear_fprop / _dgrad /
+ * _wgrad with the same rotation, rounding and seed (same operand tags, same kernels).
+ *   T, in_features, out_features  all multiples of 32.
+ *   saved      device, mxfp4_linear_layer_bytes(.., MXFP4_LAYER_SAVED) bytes, 256-byte aligned;
+ *              written by forward, read by backward (the caller keeps it alive in between).
+ *   workspace  device scratch, mxfp4_linear_layer_bytes(.., MXFP4_LAYER_FORWARD / _BACKWARD)
+ *              bytes, 256-byte aligned; free again once the call's work has run on `stream`.
+ *   dx_dtype, dw_dtype  MXFP4_OUT_*.
+ * Launches: forward 2 quantize + 1 GEMM, backward 1 quantize + 2 GEMMs (5 for the layer's three
+ * passes instead of 6, and 3.06 instead of 5.06 bytes of quantize traffic per element).
+ * mxfp4_linear_layer_bytes returns 0 for a bad argument.
+ */
+#define MXFP4_LAYER_SAVED 0
+#define MXFP4_LAYER_FORWARD 1
+#define MXFP4_LAYER_BACKWARD 2
+size_t mxfp4_linear_layer_bytes(int64_t T, int64_t in_features, int64_t out_features, int which);
+int mxfp4_linear_forward(const void* X, const void* W, void* Y, int64_t T, int64_t in_features,
+                         int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int out_dtype,
+                         void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream);
+int mxfp4_linear_backward(const void* dY, void* dX, void* dW, int64_t T, int64_t in_features,
+                          int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int dx_dtype,
+                          int dw_dtype, const void* saved, size_t saved_bytes, void* workspace,
+                          size_t workspace_bytes, void* stream);
+
+/*
  * Host-buffer form of the three passes: a_host / b_host / out_host are HOST pointers (pinned
  * memory makes the copies asynchronous).  The call copies both inputs to the caller's device
  * staging buffers, runs the pass there, copies the result back and returns after the

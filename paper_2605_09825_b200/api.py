@@ -18,13 +18,15 @@ ROUND_RNE, ROUND_SR = 0, 1
 SCALES_CANONICAL, SCALES_TILED = 0, 1
 BLOCK_1X32, BLOCK_32X32 = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
+LAYER_SAVED, LAYER_FORWARD, LAYER_BACKWARD = 0, 1, 2
 PASS_FPROP, PASS_DGRAD, PASS_WGRAD = 0, 1, 2
 AXIS_ROWS, AXIS_COLS = 0, 1
 
 EXPORTS = (
     "mxfp4_version", "mxfp4_status_string", "mxfp4_codes_bytes", "mxfp4_scales_bytes",
     "mxfp4_quantize", "mxfp4_quantize_2d", "mxfp4_quantize_dual", "mxfp4_quantize_pair", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
-    "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_host", "mxfp4_linear_static",
+    "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_layer_bytes", "mxfp4_linear_forward",
+    "mxfp4_linear_backward", "mxfp4_linear_host", "mxfp4_linear_static",
     "mxfp4_check", "mxfp4_selftest_wait_timeout",
 )
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
@@ -84,6 +86,11 @@ def load_library() -> ctypes.CDLL:
         fn = getattr(lib, name)
         fn.argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, sz, vp]
         fn.restype = ci
+    lib.mxfp4_linear_layer_bytes.argtypes, lib.mxfp4_linear_layer_bytes.restype = [i64, i64, i64, ci], sz
+    lib.mxfp4_linear_forward.argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, sz, vp, sz, vp]
+    lib.mxfp4_linear_forward.restype = ci
+    lib.mxfp4_linear_backward.argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, ci, vp, sz, vp, sz, vp]
+    lib.mxfp4_linear_backward.restype = ci
     lib.mxfp4_linear_host.argtypes = [ci, vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, vp, vp, vp,
                                       sz, vp]
     lib.mxfp4_linear_host.restype = ci
@@ -283,6 +290,56 @@ def linear_wgrad(dY, X, hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0, 
     in_f = X.shape[1]
     return _linear("mxfp4_linear_wgrad", PASS_WGRAD, dY, X, T, in_f, out_f, (out_f, in_f),
                    hadamard_mode, rounding, seed, out_dtype, workspace, out)
+
+
+def linear_layer_bytes(T: int, in_f: int, out_f: int, which: int) -> int:
+    return int(load_library().mxfp4_linear_layer_bytes(T, in_f, out_f, which))
+
+
+def _out_tensor(shape, out_dtype, device, out):
+    if out is not None:
+        return out
+    return torch.empty(shape, dtype=torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32, device=device)
+
+
+def linear_forward(X, W, hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0, out_dtype=OUT_BF16,
+                   saved=None, workspace=None, out=None):
+    """``mxfp4_linear_forward``: Y = X W^T with X and W each read once.  Returns ``(Y, saved)``;
+    ``saved`` (uint8) holds the column-wise operands ``linear_backward`` needs."""
+    for t in (X, W):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise ValueError("inputs must be contiguous bf16 tensors")
+    T, in_f = X.shape
+    out_f = W.shape[0]
+    if saved is None:
+        saved = torch.empty(max(linear_layer_bytes(T, in_f, out_f, LAYER_SAVED), 1), dtype=torch.uint8, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(max(linear_layer_bytes(T, in_f, out_f, LAYER_FORWARD), 1), dtype=torch.uint8,
+                                device=X.device)
+    out = _out_tensor((T, out_f), out_dtype, X.device, out)
+    rc = load_library().mxfp4_linear_forward(_dev_ptr(X), _dev_ptr(W), _dev_ptr(out), T, in_f, out_f, hadamard_mode,
+                                             rounding, ctypes.c_uint64(seed), out_dtype, _dev_ptr(saved),
+                                             saved.numel(), _dev_ptr(workspace), workspace.numel(), _stream())
+    _raise(rc, "mxfp4_linear_forward")
+    return out, saved
+
+
+def linear_backward(dY, saved, in_f: int, hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0,
+                    dx_dtype=OUT_BF16, dw_dtype=OUT_BF16, workspace=None, dX=None, dW=None):
+    """``mxfp4_linear_backward``: ``(dX, dW)`` from dY and what ``linear_forward`` saved."""
+    if dY.dtype != torch.bfloat16 or not dY.is_contiguous():
+        raise ValueError("dY must be a contiguous bf16 tensor")
+    T, out_f = dY.shape
+    if workspace is None:
+        workspace = torch.empty(max(linear_layer_bytes(T, in_f, out_f, LAYER_BACKWARD), 1), dtype=torch.uint8,
+                                device=dY.device)
+    dX = _out_tensor((T, in_f), dx_dtype, dY.device, dX)
+    dW = _out_tensor((out_f, in_f), dw_dtype, dY.device, dW)
+    rc = load_library().mxfp4_linear_backward(_dev_ptr(dY), _dev_ptr(dX), _dev_ptr(dW), T, in_f, out_f, hadamard_mode,
+                                              rounding, ctypes.c_uint64(seed), dx_dtype, dw_dtype, _dev_ptr(saved),
+                                              saved.numel(), _dev_ptr(workspace), workspace.numel(), _stream())
+    _raise(rc, "mxfp4_linear_backward")
+    return dX, dW
 
 
 def linear_host(pass_: int, a_host: torch.Tensor, b_host: torch.Tensor, out_host: torch.Tensor, T: int,

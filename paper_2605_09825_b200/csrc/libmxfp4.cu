@@ -449,6 +449,107 @@ int mxfp4_linear_wgrad(const void* dY, const void* X, void* dW, int64_t T, int64
                        rounding, seed, out_dtype, workspace, workspace_bytes, stream);
 }
 
+// Operand buffer = [codes][scales], each rounded up to 256 bytes.
+static size_t operand_bytes(int64_t outer, int64_t K)
+{
+    return round_up(mxfp4_codes_bytes(outer, K), 256) + round_up(mxfp4_scales_bytes(outer, K, 1), 256);
+}
+
+size_t mxfp4_linear_layer_bytes(int64_t T, int64_t in_features, int64_t out_features, int which)
+{
+    if (T <= 0 || in_features <= 0 || out_features <= 0) return 0;
+    if (T % 32 != 0 || in_features % 32 != 0 || out_features % 32 != 0) return 0;
+    switch (which) {
+        case MXFP4_LAYER_SAVED:      // X^T [in x T] and W^T [in x out]
+            return operand_bytes(in_features, T) + operand_bytes(in_features, out_features);
+        case MXFP4_LAYER_FORWARD:    // X [T x in] and W [out x in]
+            return operand_bytes(T, in_features) + operand_bytes(out_features, in_features);
+        case MXFP4_LAYER_BACKWARD:   // dY [T x out] and dY^T [out x T]
+            return operand_bytes(T, out_features) + operand_bytes(out_features, T);
+        default: return 0;
+    }
+}
+
+static int layer_args_ok(int64_t T, int64_t in_f, int64_t out_f, int hmode, int rounding, const void* saved,
+                         size_t saved_bytes, const void* workspace, size_t workspace_bytes, int ws_kind)
+{
+    if (T <= 0 || in_f <= 0 || out_f <= 0) return MXFP4_ERR_SHAPE;
+    if (T % 32 != 0 || in_f % 32 != 0 || out_f % 32 != 0) return MXFP4_ERR_SHAPE;
+    if (hmode < 0 || hmode > 4 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
+    if (!saved || saved_bytes < mxfp4_linear_layer_bytes(T, in_f, out_f, MXFP4_LAYER_SAVED)) return MXFP4_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < mxfp4_linear_layer_bytes(T, in_f, out_f, ws_kind)) return MXFP4_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(saved) & 255u) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return MXFP4_ERR_ALIGN;
+    return MXFP4_OK;
+}
+
+static float rotation_alpha(int hmode)
+{
+    // H * H^T = n * I for the +-1 matrix of order n: undone exactly in the GEMM epilogue
+    return hmode == MXFP4_HADAMARD_NONE ? 1.0f : (hmode <= MXFP4_HADAMARD_RAND ? 0.03125f : 0.0625f);
+}
+
+int mxfp4_linear_forward(const void* X, const void* W, void* Y, int64_t T, int64_t in_features,
+                         int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int out_dtype,
+                         void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!X || !W || !Y) return MXFP4_ERR_NULL;
+    int rc = layer_args_ok(T, in_features, out_features, hadamard_mode, rounding, saved, saved_bytes, workspace,
+                           workspace_bytes, MXFP4_LAYER_FORWARD);
+    if (rc != MXFP4_OK) return rc;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    uint8_t* x_codes = ws;
+    uint8_t* x_scales = x_codes + round_up(mxfp4_codes_bytes(T, in_features), 256);
+    uint8_t* w_codes = ws + operand_bytes(T, in_features);
+    uint8_t* w_scales = w_codes + round_up(mxfp4_codes_bytes(out_features, in_features), 256);
+    uint8_t* sv = static_cast<uint8_t*>(saved);
+    uint8_t* xt_codes = sv;
+    uint8_t* xt_scales = xt_codes + round_up(mxfp4_codes_bytes(in_features, T), 256);
+    uint8_t* wt_codes = sv + operand_bytes(in_features, T);
+    uint8_t* wt_scales = wt_codes + round_up(mxfp4_codes_bytes(in_features, out_features), 256);
+    // tags as in the per-pass entry points: A operands 0, B operands 1 (X^T is Wgrad's B, W^T Dgrad's B)
+    rc = mxfp4_quantize_dual(X, T, in_features, in_features, hadamard_mode, rounding, seed, 0u, 1u,
+                             MXFP4_BLOCK_1X32, x_codes, x_scales, xt_codes, xt_scales, MXFP4_SCALES_TILED, stream);
+    if (rc != MXFP4_OK) return rc;
+    rc = mxfp4_quantize_dual(W, out_features, in_features, in_features, hadamard_mode, rounding, seed, 1u, 1u,
+                             MXFP4_BLOCK_1X32, w_codes, w_scales, wt_codes, wt_scales, MXFP4_SCALES_TILED, stream);
+    if (rc != MXFP4_OK) return rc;
+    return mxfp4_gemm(x_codes, x_scales, w_codes, w_scales, T, out_features, in_features,
+                      rotation_alpha(hadamard_mode), Y, out_dtype, out_features, nullptr, 0, stream);
+}
+
+int mxfp4_linear_backward(const void* dY, void* dX, void* dW, int64_t T, int64_t in_features,
+                          int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int dx_dtype,
+                          int dw_dtype, const void* saved, size_t saved_bytes, void* workspace,
+                          size_t workspace_bytes, void* stream)
+{
+    if (!dY || !dX || !dW) return MXFP4_ERR_NULL;
+    int rc = layer_args_ok(T, in_features, out_features, hadamard_mode, rounding, saved, saved_bytes, workspace,
+                           workspace_bytes, MXFP4_LAYER_BACKWARD);
+    if (rc != MXFP4_OK) return rc;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    uint8_t* dy_codes = ws;
+    uint8_t* dy_scales = dy_codes + round_up(mxfp4_codes_bytes(T, out_features), 256);
+    uint8_t* dyt_codes = ws + operand_bytes(T, out_features);
+    uint8_t* dyt_scales = dyt_codes + round_up(mxfp4_codes_bytes(out_features, T), 256);
+    const uint8_t* sv = static_cast<const uint8_t*>(saved);
+    const uint8_t* xt_codes = sv;
+    const uint8_t* xt_scales = xt_codes + round_up(mxfp4_codes_bytes(in_features, T), 256);
+    const uint8_t* wt_codes = sv + operand_bytes(in_features, T);
+    const uint8_t* wt_scales = wt_codes + round_up(mxfp4_codes_bytes(in_features, out_features), 256);
+    rc = mxfp4_quantize_dual(dY, T, out_features, out_features, hadamard_mode, rounding, seed, 0u, 0u,
+                             MXFP4_BLOCK_1X32, dy_codes, dy_scales, dyt_codes, dyt_scales, MXFP4_SCALES_TILED, stream);
+    if (rc != MXFP4_OK) return rc;
+    const float alpha = rotation_alpha(hadamard_mode);
+    // dX [T x in] = dY [T x out] . (W^T operand [in x out])^T
+    rc = mxfp4_gemm(dy_codes, dy_scales, wt_codes, wt_scales, T, in_features, out_features, alpha, dX, dx_dtype,
+                    in_features, nullptr, 0, stream);
+    if (rc != MXFP4_OK) return rc;
+    // dW [out x in] = dY^T [out x T] . (X^T operand [in x T])^T
+    return mxfp4_gemm(dyt_codes, dyt_scales, xt_codes, xt_scales, out_features, in_features, T, alpha, dW, dw_dtype,
+                      in_features, nullptr, 0, stream);
+}
+
 int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* out_host, int64_t T,
                       int64_t in_features, int64_t out_features, int hadamard_mode, int rounding,
                       uint64_t seed, int out_dtype, void* dev_a, void* dev_b, void* dev_out,
