@@ -256,6 +256,27 @@ int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* ou
                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Host-buffer form of mxfp4_linear_forward + mxfp4_linear_backward for one linear layer: the six
+ * *_host pointers are HOST buffers (pinned memory makes the copies asynchronous and lets them
+ * overlap), every other pointer is a DEVICE buffer the caller owns.  X, W and dY cross the bus
+ * once each (the per-pass form copies every tensor twice), on a copy stream of the library's
+ * own in the order they are needed; the kernels run on `stream`; Y, dX and dW return on a second
+ * copy stream, each as soon as its GEMM has finished, so results flow out while dY still flows
+ * in.  The call returns after everything has drained: the three host outputs are valid.
+ *   dev_x, dev_w, dev_dy    device staging for the bf16 inputs ([T x in], [out x in], [T x out]);
+ *   dev_y, dev_dx, dev_dw   device staging for the outputs; all six distinct;
+ *   saved, workspace        as for forward / backward; workspace must cover the larger of
+ *                           MXFP4_LAYER_FORWARD and MXFP4_LAYER_BACKWARD.
+ * The library creates its two copy streams and its events on first use per device and keeps them.
+ * Outputs are bit-identical to the device-buffer calls.
+ */
+int mxfp4_linear_layer_host(const void* X_host, const void* W_host, const void* dY_host, void* Y_host,
+                            void* dX_host, void* dW_host, int64_t T, int64_t in_features, int64_t out_features,
+                            int hadamard_mode, int rounding, uint64_t seed, int y_dtype, int dx_dtype, int dw_dtype,
+                            void* dev_x, void* dev_w, void* dev_dy, void* dev_y, void* dev_dx, void* dev_dw,
+                            void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * mxfp4_linear_static -- the fused passes for callers that cannot allocate device memory.
  * (The paper has no counterpart to this entry point; it exists for integration only.)
  *

@@ -26,7 +26,7 @@ EXPORTS = (
     "mxfp4_version", "mxfp4_status_string", "mxfp4_codes_bytes", "mxfp4_scales_bytes",
     "mxfp4_quantize", "mxfp4_quantize_2d", "mxfp4_quantize_dual", "mxfp4_quantize_pair", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
     "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_layer_bytes", "mxfp4_linear_forward",
-    "mxfp4_linear_backward", "mxfp4_linear_host", "mxfp4_linear_static",
+    "mxfp4_linear_backward", "mxfp4_linear_layer_host", "mxfp4_linear_host", "mxfp4_linear_static",
     "mxfp4_check", "mxfp4_selftest_wait_timeout",
 )
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
@@ -91,6 +91,9 @@ def load_library() -> ctypes.CDLL:
     lib.mxfp4_linear_forward.restype = ci
     lib.mxfp4_linear_backward.argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, ci, vp, sz, vp, sz, vp]
     lib.mxfp4_linear_backward.restype = ci
+    lib.mxfp4_linear_layer_host.argtypes = [vp] * 6 + [i64, i64, i64, ci, ci, u64, ci, ci, ci] + [vp] * 6 + \
+        [vp, sz, vp, sz, vp]
+    lib.mxfp4_linear_layer_host.restype = ci
     lib.mxfp4_linear_host.argtypes = [ci, vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, vp, vp, vp,
                                       sz, vp]
     lib.mxfp4_linear_host.restype = ci
@@ -340,6 +343,22 @@ def linear_backward(dY, saved, in_f: int, hadamard_mode=HADAMARD_DET, rounding=R
                                               saved.numel(), _dev_ptr(workspace), workspace.numel(), _stream())
     _raise(rc, "mxfp4_linear_backward")
     return dX, dW
+
+
+def linear_layer_host(X_host, W_host, dY_host, Y_host, dX_host, dW_host, dev: dict, saved, workspace,
+                      hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0, y_dtype=OUT_BF16,
+                      dx_dtype=OUT_BF16, dw_dtype=OUT_BF16):
+    """``mxfp4_linear_layer_host``: forward + backward of one linear from host (ideally pinned)
+    tensors into host tensors; ``dev`` maps "x", "w", "dy", "y", "dx", "dw" to device staging."""
+    T, in_f = X_host.shape
+    out_f = W_host.shape[0]
+    rc = load_library().mxfp4_linear_layer_host(
+        X_host.data_ptr(), W_host.data_ptr(), dY_host.data_ptr(), Y_host.data_ptr(), dX_host.data_ptr(),
+        dW_host.data_ptr(), T, in_f, out_f, hadamard_mode, rounding, ctypes.c_uint64(seed), y_dtype, dx_dtype,
+        dw_dtype, _dev_ptr(dev["x"]), _dev_ptr(dev["w"]), _dev_ptr(dev["dy"]), _dev_ptr(dev["y"]),
+        _dev_ptr(dev["dx"]), _dev_ptr(dev["dw"]), _dev_ptr(saved), saved.numel(), _dev_ptr(workspace),
+        workspace.numel(), _stream())
+    _raise(rc, "mxfp4_linear_layer_host")
 
 
 def linear_host(pass_: int, a_host: torch.Tensor, b_host: torch.Tensor, out_host: torch.Tensor, T: int,

@@ -518,10 +518,11 @@ int mxfp4_linear_forward(const void* X, const void* W, void* Y, int64_t T, int64
                       rotation_alpha(hadamard_mode), Y, out_dtype, out_features, nullptr, 0, stream);
 }
 
-int mxfp4_linear_backward(const void* dY, void* dX, void* dW, int64_t T, int64_t in_features,
-                          int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int dx_dtype,
-                          int dw_dtype, const void* saved, size_t saved_bytes, void* workspace,
-                          size_t workspace_bytes, void* stream)
+// mxfp4_linear_backward; `after_dx` (optional) is recorded between the two GEMMs.
+static int linear_backward_impl(const void* dY, void* dX, void* dW, int64_t T, int64_t in_features,
+                                int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int dx_dtype,
+                                int dw_dtype, const void* saved, size_t saved_bytes, void* workspace,
+                                size_t workspace_bytes, void* stream, cudaEvent_t after_dx)
 {
     if (!dY || !dX || !dW) return MXFP4_ERR_NULL;
     int rc = layer_args_ok(T, in_features, out_features, hadamard_mode, rounding, saved, saved_bytes, workspace,
@@ -545,9 +546,106 @@ int mxfp4_linear_backward(const void* dY, void* dX, void* dW, int64_t T, int64_t
     rc = mxfp4_gemm(dy_codes, dy_scales, wt_codes, wt_scales, T, in_features, out_features, alpha, dX, dx_dtype,
                     in_features, nullptr, 0, stream);
     if (rc != MXFP4_OK) return rc;
+    if (after_dx && cudaEventRecord(after_dx, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MXFP4_ERR_CUDA;
     // dW [out x in] = dY^T [out x T] . (X^T operand [in x T])^T
     return mxfp4_gemm(dyt_codes, dyt_scales, xt_codes, xt_scales, out_features, in_features, T, alpha, dW, dw_dtype,
                       in_features, nullptr, 0, stream);
+}
+
+int mxfp4_linear_backward(const void* dY, void* dX, void* dW, int64_t T, int64_t in_features,
+                          int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int dx_dtype,
+                          int dw_dtype, const void* saved, size_t saved_bytes, void* workspace,
+                          size_t workspace_bytes, void* stream)
+{
+    return linear_backward_impl(dY, dX, dW, T, in_features, out_features, hadamard_mode, rounding, seed, dx_dtype,
+                                dw_dtype, saved, saved_bytes, workspace, workspace_bytes, stream, nullptr);
+}
+
+// Copy streams and events of the host-buffer layer call, one set per device, created on first
+// use and kept for the life of the process.
+struct HostPipe {
+    cudaStream_t h2d, d2h;
+    cudaEvent_t start, xw, dy, y, dx, dw, done;
+    bool ready;
+};
+
+static int host_pipe(HostPipe** out)
+{
+    static HostPipe pipes[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
+    HostPipe& p = pipes[dev];
+    if (!p.ready) {
+        if (cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking) != cudaSuccess)
+            return MXFP4_ERR_CUDA;
+        cudaEvent_t* evs[7] = {&p.start, &p.xw, &p.dy, &p.y, &p.dx, &p.dw, &p.done};
+        for (cudaEvent_t* e : evs)
+            if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return MXFP4_ERR_CUDA;
+        p.ready = true;
+    }
+    *out = &p;
+    return MXFP4_OK;
+}
+
+int mxfp4_linear_layer_host(const void* X_host, const void* W_host, const void* dY_host, void* Y_host,
+                            void* dX_host, void* dW_host, int64_t T, int64_t in_features, int64_t out_features,
+                            int hadamard_mode, int rounding, uint64_t seed, int y_dtype, int dx_dtype, int dw_dtype,
+                            void* dev_x, void* dev_w, void* dev_dy, void* dev_y, void* dev_dx, void* dev_dw,
+                            void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!X_host || !W_host || !dY_host || !Y_host || !dX_host || !dW_host) return MXFP4_ERR_NULL;
+    if (!dev_x || !dev_w || !dev_dy || !dev_y || !dev_dx || !dev_dw) return MXFP4_ERR_NULL;
+    for (int d : {y_dtype, dx_dtype, dw_dtype})
+        if (d != MXFP4_OUT_BF16 && d != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
+    int rc = layer_args_ok(T, in_features, out_features, hadamard_mode, rounding, saved, saved_bytes, workspace,
+                           workspace_bytes, MXFP4_LAYER_FORWARD);
+    if (rc != MXFP4_OK) return rc;
+    if (workspace_bytes < mxfp4_linear_layer_bytes(T, in_features, out_features, MXFP4_LAYER_BACKWARD))
+        return MXFP4_ERR_WORKSPACE;
+    HostPipe* hp = nullptr;
+    rc = host_pipe(&hp);
+    if (rc != MXFP4_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t x_bytes = static_cast<size_t>(T) * in_features * 2;
+    const size_t w_bytes = static_cast<size_t>(out_features) * in_features * 2;
+    const size_t dy_bytes = static_cast<size_t>(T) * out_features * 2;
+    const size_t y_out = static_cast<size_t>(T) * out_features * (y_dtype == MXFP4_OUT_BF16 ? 2 : 4);
+    const size_t dx_out = static_cast<size_t>(T) * in_features * (dx_dtype == MXFP4_OUT_BF16 ? 2 : 4);
+    const size_t dw_out = static_cast<size_t>(out_features) * in_features * (dw_dtype == MXFP4_OUT_BF16 ? 2 : 4);
+#define MXFP4_TRY(call) do { if ((call) != cudaSuccess) return MXFP4_ERR_CUDA; } while (0)
+    // inputs travel on their own stream, in the order they are needed; they start once the work
+    // already queued on the caller's stream (which may still use the staging buffers) is done
+    MXFP4_TRY(cudaEventRecord(hp->start, st));
+    MXFP4_TRY(cudaStreamWaitEvent(hp->h2d, hp->start, 0));
+    MXFP4_TRY(cudaMemcpyAsync(dev_x, X_host, x_bytes, cudaMemcpyHostToDevice, hp->h2d));
+    MXFP4_TRY(cudaMemcpyAsync(dev_w, W_host, w_bytes, cudaMemcpyHostToDevice, hp->h2d));
+    MXFP4_TRY(cudaEventRecord(hp->xw, hp->h2d));
+    MXFP4_TRY(cudaMemcpyAsync(dev_dy, dY_host, dy_bytes, cudaMemcpyHostToDevice, hp->h2d));
+    MXFP4_TRY(cudaEventRecord(hp->dy, hp->h2d));
+    // compute on the caller's stream
+    MXFP4_TRY(cudaStreamWaitEvent(st, hp->xw, 0));
+    rc = mxfp4_linear_forward(dev_x, dev_w, dev_y, T, in_features, out_features, hadamard_mode, rounding, seed,
+                              y_dtype, saved, saved_bytes, workspace, workspace_bytes, stream);
+    if (rc != MXFP4_OK) return rc;
+    MXFP4_TRY(cudaEventRecord(hp->y, st));
+    MXFP4_TRY(cudaStreamWaitEvent(st, hp->dy, 0));
+    rc = linear_backward_impl(dev_dy, dev_dx, dev_dw, T, in_features, out_features, hadamard_mode, rounding, seed,
+                              dx_dtype, dw_dtype, saved, saved_bytes, workspace, workspace_bytes, stream, hp->dx);
+    if (rc != MXFP4_OK) return rc;
+    MXFP4_TRY(cudaEventRecord(hp->dw, st));
+    // results leave on a third stream, each as soon as its GEMM is done, while later inputs still arrive
+    MXFP4_TRY(cudaStreamWaitEvent(hp->d2h, hp->y, 0));
+    MXFP4_TRY(cudaMemcpyAsync(Y_host, dev_y, y_out, cudaMemcpyDeviceToHost, hp->d2h));
+    MXFP4_TRY(cudaStreamWaitEvent(hp->d2h, hp->dx, 0));
+    MXFP4_TRY(cudaMemcpyAsync(dX_host, dev_dx, dx_out, cudaMemcpyDeviceToHost, hp->d2h));
+    MXFP4_TRY(cudaStreamWaitEvent(hp->d2h, hp->dw, 0));
+    MXFP4_TRY(cudaMemcpyAsync(dW_host, dev_dw, dw_out, cudaMemcpyDeviceToHost, hp->d2h));
+    MXFP4_TRY(cudaEventRecord(hp->done, hp->d2h));
+    MXFP4_TRY(cudaStreamWaitEvent(st, hp->done, 0));
+    MXFP4_TRY(cudaStreamSynchronize(st));
+#undef MXFP4_TRY
+    return MXFP4_OK;
 }
 
 int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* out_host, int64_t T,

@@ -68,3 +68,46 @@ def test_config5_layer_stack_16384_tokens(name):
     _check_pass(0, t["X"], t["W"], 1, 0, 0, f"config 5 {name} fprop")
     _check_pass(1, t["dY"], t["W"], 1, 0, 0, f"config 5 {name} dgrad")
     _check_pass(2, t["dY"], t["X"], 1, 0, 0, f"config 5 {name} wgrad")
+
+
+@pytest.mark.parametrize("name", ["qkv", "o", "gate_up", "down"])
+def test_config5_layer_schedule_16384_tokens(name):
+    """The schedule bench.py times by default: forward + backward per linear, every tensor read
+    once by the dual-axis quantize.  Sampled output rows against the oracle; the kept column-wise
+    operands (the whole saved buffer) bit-exact for the smallest linear."""
+    t = synth.linear_tensors(name, 16384, 5)
+    X, W, dY = to_dev(t["X"]), to_dev(t["W"]), to_dev(t["dY"])
+    in_f = X.shape[1]
+    Y, saved = api.linear_forward(X, W, 1, 0, 0)
+    dX, dW = api.linear_backward(dY, saved, in_f, 1, 0, 0)
+    api.check()
+    for out, ofn, a, b, what in ((Y, oracle.linear_fprop, t["X"], t["W"], "fprop"),
+                                 (dX, oracle.linear_dgrad, t["dY"], t["W"], "dgrad"),
+                                 (dW, oracle.linear_wgrad, t["dY"], t["X"], "wgrad")):
+        rows = _rows(out.shape[0], 4321)
+        ref, S = ofn(a, b, 1, 0, 0, rows=rows)
+        got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy()
+        assert_gemm_close(got, ref, S, True, f"config 5 {name} layer schedule {what}")
+    if name == "o":
+        raw = saved.cpu().numpy()
+        r256 = lambda n: (n + 255) // 256 * 256
+        off = 0
+        for bits in (t["X"], t["W"]):
+            wc, ws = oracle.quantize(bits, 0, 1, 0, 0, 1)
+            outer, K = wc.shape[0], wc.shape[1] * 2
+            assert (raw[off:off + wc.size].reshape(wc.shape) == wc).all()
+            off += r256(wc.size)
+            sb = api.scales_bytes(outer, K)
+            assert (oracle.scales_from_tiled(raw[off:off + sb], outer, K // 32) == ws).all()
+            off += r256(sb)
+
+
+def test_config3_dual_quantize_of_the_largest_tensor():
+    """dY of gate+up at 8192 tokens (448 MiB of bf16): both orientations, whole tensors, bit-exact."""
+    t = synth.config3()
+    (cr, sr), (cc, sc) = api.quantize_dual(to_dev(t["dY"]), 1, 0, 0, tags=(0, 0))
+    api.check()
+    for codes, scales, axis in ((cr, sr, 1), (cc, sc, 0)):
+        wc, ws = oracle.quantize(t["dY"], axis, 1, 0, 0, 0)
+        assert (codes.cpu().numpy() == wc).all()
+        assert (oracle.scales_from_tiled(scales.cpu().numpy(), wc.shape[0], wc.shape[1] * 2 // 32) == ws).all()

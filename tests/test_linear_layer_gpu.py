@@ -78,3 +78,25 @@ def test_layer_argument_errors():
         api.linear_forward(bad, W, saved=torch.empty(1 << 20, dtype=torch.uint8, device="cuda"),
                            workspace=torch.empty(1 << 20, dtype=torch.uint8, device="cuda"))
     assert exc.value.status == -2
+
+
+def test_host_buffer_layer_call_matches_the_device_calls():
+    T, in_f, out_f = 416, 288, 672
+    Xb, Wb, dYb = _tensors(T, in_f, out_f, 13)
+    host = [torch.from_numpy(b.view(np.int16)).view(torch.bfloat16).pin_memory() for b in (Xb, Wb, dYb)]
+    Yh = torch.empty((T, out_f), dtype=torch.bfloat16).pin_memory()
+    dXh = torch.empty((T, in_f), dtype=torch.bfloat16).pin_memory()
+    dWh = torch.empty((out_f, in_f), dtype=torch.float32).pin_memory()
+    e = lambda shape, dt: torch.empty(shape, dtype=dt, device="cuda")
+    dev = {"x": e((T, in_f), torch.bfloat16), "w": e((out_f, in_f), torch.bfloat16), "dy": e((T, out_f), torch.bfloat16),
+           "y": e((T, out_f), torch.bfloat16), "dx": e((T, in_f), torch.bfloat16), "dw": e((out_f, in_f), torch.float32)}
+    saved = e(api.linear_layer_bytes(T, in_f, out_f, api.LAYER_SAVED), torch.uint8)
+    ws = e(max(api.linear_layer_bytes(T, in_f, out_f, w) for w in (api.LAYER_FORWARD, api.LAYER_BACKWARD)), torch.uint8)
+    for _ in range(2):                                   # twice: the second call reuses streams and events
+        api.linear_layer_host(*host, Yh, dXh, dWh, dev, saved, ws, 1, 0, 3, api.OUT_BF16, api.OUT_BF16, api.OUT_FP32)
+        api.check()
+        X, W, dY = (h.cuda() for h in host)
+        Y, sv = api.linear_forward(X, W, 1, 0, 3)
+        dX, dW = api.linear_backward(dY, sv, in_f, 1, 0, 3, api.OUT_BF16, api.OUT_FP32)
+        assert torch.equal(Yh, Y.cpu()) and torch.equal(dXh, dX.cpu()) and torch.equal(dWh, dW.cpu())
+        Yh.zero_(); dXh.zero_(); dWh.zero_()
