@@ -11,6 +11,9 @@ Passages followed: Appendix A.1 Eq. (1) (micro-scaling), Appendix A.2 (Hadamard 
 random sign flips), Appendix C (which axis each operand of Fprop / Dgrad / Wgrad is rotated
 and quantized along), Appendix D (row-wise and column-wise 32-blocks).
 Stochastic rounding: parity unpinned against the paper (it gives no definition).
+
+``mxfp8_oracle.c`` holds the 8-bit passes of the precision ladder (Table 1): the paper names the
+format only as "FP8"; the reading taken is MXFP8 (E4M3 elements, the same E8M0 block scale).
 """
 from __future__ import annotations
 
@@ -22,6 +25,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "mxfp4_oracle.c")
+_SRC8 = os.path.join(_HERE, "mxfp8_oracle.c")      # the 8-bit passes of the precision ladder
 _LIB = os.path.join(_HERE, "libmxfp4_oracle.so")
 
 HADAMARD_NONE, HADAMARD_DET, HADAMARD_RAND, HADAMARD_DET16, HADAMARD_RAND16 = 0, 1, 2, 3, 4
@@ -30,10 +34,11 @@ ROUND_RNE, ROUND_SR = 0, 1
 
 def build(force: bool = False) -> str:
     """Compile the C oracle into ``libmxfp4_oracle.so`` next to its source (gcc, OpenMP)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC),
+                                                                         os.path.getmtime(_SRC8)):
         tmp = _LIB + f".tmp{os.getpid()}"
         cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
-               "-o", tmp, _SRC, "-lm"]
+               "-o", tmp, _SRC, _SRC8, "-lm"]
         subprocess.run(cmd, check=True)
         os.replace(tmp, _LIB)
     return _LIB
@@ -63,6 +68,14 @@ def _load():
     lib.oracle_quantize.restype = ctypes.c_int
     lib.oracle_quantize_2d.argtypes = lib.oracle_quantize.argtypes
     lib.oracle_quantize_2d.restype = ctypes.c_int
+    lib.oracle_e4m3_decode.argtypes, lib.oracle_e4m3_decode.restype = [ctypes.c_uint8], ctypes.c_double
+    lib.oracle_e4m3_encode.argtypes, lib.oracle_e4m3_encode.restype = [ctypes.c_float], ctypes.c_uint8
+    lib.oracle_quantize_mxfp8.argtypes = [ctypes.POINTER(ctypes.c_uint16), i64, i64, i64, ctypes.c_int, u8p, u8p]
+    lib.oracle_quantize_mxfp8.restype = ctypes.c_int
+    lib.oracle_gemm_rows_mxfp8.argtypes = [u8p, u8p, u8p, u8p, i64, i64, i64, ctypes.c_double,
+                                           ctypes.POINTER(ctypes.c_int64), i64,
+                                           ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+    lib.oracle_gemm_rows_mxfp8.restype = ctypes.c_int
     lib.oracle_scale_offset_tiled.argtypes = [i64, i64, i64]
     lib.oracle_scale_offset_tiled.restype = i64
     lib.oracle_dequantize.argtypes = [u8p, u8p, i64, i64, ctypes.POINTER(ctypes.c_double)]
@@ -246,3 +259,65 @@ def linear_wgrad(dY, X, hadamard_mode=1, rounding=0, seed=0, rows=None):
     a = quantize(dY, 0, hadamard_mode, rounding, seed, 0)
     b = quantize(X, 0, hadamard_mode, rounding, seed, 1)
     return gemm(*a, *b, alpha=_alpha(hadamard_mode), rows=rows)
+
+
+# ----------------------------------------------------------------------------- 8-bit passes
+def e4m3_decode(code: int) -> float:
+    return float(_load().oracle_e4m3_decode(int(code)))
+
+
+def e4m3_encode(x: float) -> int:
+    return int(_load().oracle_e4m3_encode(ctypes.c_float(x)))
+
+
+def quantize_mxfp8(src_bits: np.ndarray, axis: int = 1):
+    """MXFP8 (E4M3 elements, E8M0 scale per 32 along K) of a [rows x cols] bf16 matrix.
+
+    Returns ``(codes [outer x K] uint8, scales [outer x K/32] uint8)`` for the operand view of
+    :func:`quantize`.  Round-to-nearest-even, saturating; no rotation.
+    """
+    assert src_bits.dtype == np.uint16 and src_bits.ndim == 2
+    src = np.ascontiguousarray(src_bits)
+    rows, cols = src.shape
+    outer, K = (rows, cols) if axis == 1 else (cols, rows)
+    codes = np.empty((outer, K), dtype=np.uint8)
+    scales = np.empty((outer, K // 32), dtype=np.uint8)
+    rc = _load().oracle_quantize_mxfp8(_ptr(src, ctypes.c_uint16), rows, cols, cols, axis,
+                                       _ptr(codes, ctypes.c_uint8), _ptr(scales, ctypes.c_uint8))
+    if rc != 0:
+        raise ValueError(f"oracle_quantize_mxfp8 rejected its arguments (rc={rc})")
+    return codes, scales
+
+
+def gemm_mxfp8(a_codes, a_scales, b_codes, b_scales, alpha: float = 1.0, rows=None):
+    """fp64 block-scaled product of E4M3 operands and the tolerance base S (see :func:`gemm`)."""
+    a_codes = np.ascontiguousarray(a_codes, dtype=np.uint8)
+    b_codes = np.ascontiguousarray(b_codes, dtype=np.uint8)
+    a_scales = np.ascontiguousarray(a_scales, dtype=np.uint8)
+    b_scales = np.ascontiguousarray(b_scales, dtype=np.uint8)
+    M, K = a_codes.shape
+    N, K2 = b_codes.shape
+    assert K == K2 and a_scales.shape == (M, K // 32) and b_scales.shape == (N, K // 32)
+    if rows is None:
+        rows_arr, rp, nrows = None, None, M
+    else:
+        rows_arr = np.ascontiguousarray(rows, dtype=np.int64)
+        rp, nrows = _ptr(rows_arr, ctypes.c_int64), int(rows_arr.size)
+    ref = np.empty((nrows, N), dtype=np.float64)
+    S = np.empty((nrows, N), dtype=np.float64)
+    rc = _load().oracle_gemm_rows_mxfp8(_ptr(a_codes, ctypes.c_uint8), _ptr(a_scales, ctypes.c_uint8),
+                                        _ptr(b_codes, ctypes.c_uint8), _ptr(b_scales, ctypes.c_uint8),
+                                        M, N, K, float(alpha), rp, nrows, _ptr(ref, ctypes.c_double),
+                                        _ptr(S, ctypes.c_double))
+    if rc != 0:
+        raise ValueError(f"oracle_gemm_rows_mxfp8 failed (rc={rc})")
+    return ref, S
+
+
+def linear_pass_mxfp8(pass_: int, a_bits, b_bits, rows=None):
+    """One pass of a linear layer left in 8 bits (Table 1): operand orientation as Appendix C,
+    (a, b) = (X, W) / (dY, W) / (dY, X) for pass 0 / 1 / 2."""
+    axes = ((1, 1), (1, 0), (0, 0))[pass_]
+    a = quantize_mxfp8(a_bits, axes[0])
+    b = quantize_mxfp8(b_bits, axes[1])
+    return gemm_mxfp8(*a, *b, rows=rows)
