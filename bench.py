@@ -229,9 +229,20 @@ def run_ours(args):
     dims = {n: synth.LLAMA8B_LINEARS[n] for n in names}   # (out, in)
     max_out = max(max(tokens * o, tokens * i, o * i) for o, i in dims.values())
     out_buf = torch.empty(max_out, dtype=torch.bfloat16, device="cuda")
-    ws_bytes = max(api.linear_workspace_bytes(tokens, i, o, p) for o, i in dims.values() for p in range(3))
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     lib = api.load_library()
+    # precision ladder (Table 1): the passes named in --mxfp4-passes run MXFP4, the others MXFP8
+    fp4_passes = {"fprop": 0, "dgrad": 1, "wgrad": 2}
+    chosen = [x for x in args.mxfp4_passes.split(",") if x and x != "none"]
+    if any(x not in fp4_passes for x in chosen):
+        raise SystemExit("--mxfp4-passes takes a comma-separated subset of fprop,dgrad,wgrad (or 'none')")
+    precision = [api.PRECISION_MXFP4 if name in chosen else api.PRECISION_MXFP8 for name in ("fprop", "dgrad", "wgrad")]
+    ladder = any(pr == api.PRECISION_MXFP8 for pr in precision)
+    if ladder:
+        args.schedule = "per_pass"          # the layer-level calls are MXFP4 throughout
+        args.no_e2e = args.no_configs = True  # the host-buffer call and the single-pass configs are MXFP4 only
+    ws_bytes = max(int(lib.mxfp4_linear_pass_workspace_bytes(tokens, i, o, p, precision[p]))
+                   for o, i in dims.values() for p in range(3))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
     sptr = int(stream.cuda_stream)
 
@@ -256,8 +267,8 @@ def run_ours(args):
     def step_per_pass():
         for (n, p, a, b, M, N, K) in passes:
             o, i = dims[n]
-            rc = fused[p](a.data_ptr(), b.data_ptr(), out_buf.data_ptr(), tokens, i, o, hmode, rnd, seed,
-                          api.OUT_BF16, ws.data_ptr(), ws_bytes, sptr)
+            rc = lib.mxfp4_linear_pass(p, precision[p], a.data_ptr(), b.data_ptr(), out_buf.data_ptr(), tokens, i, o,
+                                       hmode, rnd, seed, api.OUT_BF16, ws.data_ptr(), ws_bytes, sptr)
             if rc != 0:
                 raise api.Mxfp4Error(rc, "fused linear pass")
 
@@ -323,6 +334,7 @@ def run_ours(args):
 
     for rep in range(2):
         evs = []
+        fp8_evs = []
         if layer:
             for n in names:
                 o, i = dims[n]
@@ -355,6 +367,16 @@ def run_ours(args):
         else:
             for (n, p, a, b, M, N, K) in passes:
                 ax_a, ax_b = a_b_axes(p)
+                if precision[p] == api.PRECISION_MXFP8:
+                    # 8-bit pass: timed as a whole (its kernels are not the roofline's subject)
+                    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+                    ev[0].record(stream)
+                    lib.mxfp4_linear_pass(p, precision[p], a.data_ptr(), b.data_ptr(), out_buf.data_ptr(), tokens,
+                                          dims[n][1], dims[n][0], hmode, rnd, seed, api.OUT_BF16, ws.data_ptr(),
+                                          ws_bytes, sptr)
+                    ev[1].record(stream)
+                    fp8_evs.append((ev[0], ev[1], 2.0 * M * N * K))
+                    continue
                 ac, a_s, off = operand_views(ws, 0, M, K)
                 bc, b_s, _ = operand_views(ws, off, N, K)
                 ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
@@ -411,7 +433,15 @@ def run_ours(args):
         del flush
         api.check()
 
-    n_gemm = len(passes)
+    fp8_info = None
+    if ladder:
+        f8_ms = sum(a0.elapsed_time(a1) for a0, a1, _ in fp8_evs)
+        f8_fl = sum(fl for _, _, fl in fp8_evs)
+        fp8_info = {"passes": len(fp8_evs), "tflops_incl_quantize": f8_fl / (f8_ms * 1e-3) / 1e12,
+                    "format": "MXFP8 (E4M3 elements, E8M0 scale per 32), no rotation"}
+    n_gemm = max(1, len(passes) - len(fp8_evs))
+    if gemm_ms == 0.0:                      # all passes in 8 bits: nothing for the MXFP4 roofline
+        gemm_ms, gemm_flops, quant_ms, quant_bytes, n_quant = 1.0, 0.0, 1.0, 0.0, 1
     fp4_peak = 4.0 * peaks["bf16_tflops_sustained"]
     gemm_tflops = gemm_flops / (gemm_ms * 1e-3) / 1e12
     roofline = {
@@ -554,12 +584,13 @@ def run_ours(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "e2m1 (mxfp4) x e2m1, f32 accumulate",
         "data": "synthetic",
         "config": {"workload": workload_label(args.workload, tokens, args.hadamard), "passes_per_step": len(passes),
+                   "mxfp4_passes": chosen if chosen else "none (all passes MXFP8)",
                    "schedule": ("layer: forward + backward per linear, each of X, W, dY read once by the dual-axis "
                                 "quantize" if layer else "per pass: both operands of each pass quantized from bf16"),
                    "flops_per_step": flops_per_step, "out_dtype": "bf16",
                    "l2": "inputs larger than L2 (several GB per step), no flush needed",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
-        "roofline": roofline, "quantize": quantize_info,
+        "roofline": roofline, "quantize": quantize_info, "mxfp8_passes": fp8_info,
         "frac_of_nominal_fp4_peak": world and (flops_per_step / (ms_per_step * 1e-3) / 1e12) / 9000.0,
         "cpu_baseline": cpu_base, "e2e": e2e, "gpu_launches": 2 * len(passes) * args.steps,   # per linear: 3 quantize + 3 GEMM (layer) or 3 x (1 + 1)
         "clocks": clocks, "context": context, "per_config": per_config,
@@ -570,6 +601,9 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--mxfp4-passes", default="fprop,dgrad,wgrad",
+                    help="precision ladder: comma-separated passes that run MXFP4 (the rest run MXFP8); 'none' or '' "
+                         "for the all-8-bit baseline; anything but all three implies --schedule per_pass")
     ap.add_argument("--schedule", default="layer", choices=["layer", "per_pass"],
                     help="layer: mxfp4_linear_forward/backward (each tensor read once); per_pass: the three "
                          "per-pass entry points")

@@ -62,6 +62,9 @@ extern "C" {
 #define MXFP4_BLOCK_1X32 0  /* one scale per 32 elements along K (Appendix D, 1D)               */
 #define MXFP4_BLOCK_32X32 1 /* one scale per 32 operand rows x 32 elements (Appendix D, 2D)      */
 
+#define MXFP4_PRECISION_MXFP4 0 /* E2M1 elements, the method's GEMMs                              */
+#define MXFP4_PRECISION_MXFP8 1 /* E4M3 elements, the passes the ladder of Table 1 leaves in FP8  */
+
 #define MXFP4_OUT_BF16 0
 #define MXFP4_OUT_FP32 1
 
@@ -211,6 +214,34 @@ int mxfp4_linear_dgrad(const void* dY, const void* W, void* dX, int64_t T, int64
 int mxfp4_linear_wgrad(const void* dY, const void* X, void* dW, int64_t T, int64_t in_features,
                        int64_t out_features, int hadamard_mode, int rounding, uint64_t seed,
                        int out_dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The 8-bit side of the precision ladder (Table 1: Fprop, Dgrad and Wgrad are switched to MXFP4
+ * one by one; the others stay in FP8).  The paper does not say which FP8 recipe its baseline
+ * uses; this library's 8-bit passes are MXFP8 -- Eq. (1) of Appendix A.1 with E4M3 elements:
+ * one E8M0 scale 2^(floor(log2 amax) - 8) per 32 elements along the reduction axis, elements
+ * rounded to the nearest E4M3 value (ties to even, saturating at 448, sign kept on zero), no
+ * rotation and no stochastic rounding.
+ *
+ * mxfp4_quantize_fp8: as mxfp4_quantize; codes are [outer x K] bytes (one E4M3 code per element),
+ *   scales as for the 4-bit format (same size, same layouts).
+ * mxfp4_gemm_fp8: as mxfp4_gemm on such operands (tcgen05 kind::mxf8f6f4, fp32 accumulation).
+ * mxfp4_linear_pass: one pass at a chosen precision; (a, b, out) = (X, W, Y) / (dY, W, dX) /
+ *   (dY, X, dW) for MXFP4_PASS_FPROP / _DGRAD / _WGRAD.  With MXFP4_PRECISION_MXFP4 it is
+ *   mxfp4_linear_fprop / _dgrad / _wgrad; with MXFP4_PRECISION_MXFP8 hadamard_mode, rounding and
+ *   seed are ignored.  Workspace: mxfp4_linear_pass_workspace_bytes (0 for a bad argument).
+ * Errors as for the 4-bit entry points.
+ */
+int mxfp4_quantize_fp8(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis, void* codes,
+                       void* scales, int scale_layout, void* stream);
+int mxfp4_gemm_fp8(const void* a_codes, const void* a_scales, const void* b_codes, const void* b_scales,
+                   int64_t M, int64_t N, int64_t K, float alpha, void* out, int out_dtype, int64_t ld_out,
+                   void* stream);
+size_t mxfp4_linear_pass_workspace_bytes(int64_t T, int64_t in_features, int64_t out_features, int pass,
+                                         int precision);
+int mxfp4_linear_pass(int pass, int precision, const void* a, const void* b, void* out, int64_t T,
+                      int64_t in_features, int64_t out_features, int hadamard_mode, int rounding, uint64_t seed,
+                      int out_dtype, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Layer-level form of the same three passes (Appendix C), each tensor read ONCE: a linear layer

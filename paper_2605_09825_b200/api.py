@@ -19,6 +19,7 @@ SCALES_CANONICAL, SCALES_TILED = 0, 1
 BLOCK_1X32, BLOCK_32X32 = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
 LAYER_SAVED, LAYER_FORWARD, LAYER_BACKWARD = 0, 1, 2
+PRECISION_MXFP4, PRECISION_MXFP8 = 0, 1
 PASS_FPROP, PASS_DGRAD, PASS_WGRAD = 0, 1, 2
 AXIS_ROWS, AXIS_COLS = 0, 1
 
@@ -26,7 +27,8 @@ EXPORTS = (
     "mxfp4_version", "mxfp4_status_string", "mxfp4_codes_bytes", "mxfp4_scales_bytes",
     "mxfp4_quantize", "mxfp4_quantize_2d", "mxfp4_quantize_dual", "mxfp4_quantize_pair", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
     "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_layer_bytes", "mxfp4_linear_forward",
-    "mxfp4_linear_backward", "mxfp4_linear_layer_host", "mxfp4_linear_host", "mxfp4_linear_static",
+    "mxfp4_linear_backward", "mxfp4_linear_layer_host", "mxfp4_quantize_fp8", "mxfp4_gemm_fp8",
+    "mxfp4_linear_pass_workspace_bytes", "mxfp4_linear_pass", "mxfp4_linear_host", "mxfp4_linear_static",
     "mxfp4_check", "mxfp4_selftest_wait_timeout",
 )
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
@@ -86,6 +88,13 @@ def load_library() -> ctypes.CDLL:
         fn = getattr(lib, name)
         fn.argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, sz, vp]
         fn.restype = ci
+    lib.mxfp4_quantize_fp8.argtypes, lib.mxfp4_quantize_fp8.restype = [vp, i64, i64, i64, ci, vp, vp, ci, vp], ci
+    lib.mxfp4_gemm_fp8.argtypes = [vp, vp, vp, vp, i64, i64, i64, ctypes.c_float, vp, ci, i64, vp]
+    lib.mxfp4_gemm_fp8.restype = ci
+    lib.mxfp4_linear_pass_workspace_bytes.argtypes = [i64, i64, i64, ci, ci]
+    lib.mxfp4_linear_pass_workspace_bytes.restype = sz
+    lib.mxfp4_linear_pass.argtypes = [ci, ci, vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, sz, vp]
+    lib.mxfp4_linear_pass.restype = ci
     lib.mxfp4_linear_layer_bytes.argtypes, lib.mxfp4_linear_layer_bytes.restype = [i64, i64, i64, ci], sz
     lib.mxfp4_linear_forward.argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, sz, vp, sz, vp]
     lib.mxfp4_linear_forward.restype = ci
@@ -293,6 +302,66 @@ def linear_wgrad(dY, X, hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0, 
     in_f = X.shape[1]
     return _linear("mxfp4_linear_wgrad", PASS_WGRAD, dY, X, T, in_f, out_f, (out_f, in_f),
                    hadamard_mode, rounding, seed, out_dtype, workspace, out)
+
+
+def quantize_fp8(src: torch.Tensor, axis: int = AXIS_COLS, scale_layout: int = SCALES_TILED, codes=None,
+                 scales=None):
+    """``mxfp4_quantize_fp8``: MXFP8 (E4M3 + E8M0 per 32) operand of a 2-D bf16 CUDA tensor.
+    Returns ``(codes uint8 [outer, K], scales uint8 [scales_bytes])``."""
+    if src.dtype != torch.bfloat16 or src.dim() != 2 or src.stride(1) != 1:
+        raise ValueError("src must be a 2-D bf16 tensor with contiguous rows")
+    rows, cols = src.shape
+    outer, K = (rows, cols) if axis == AXIS_COLS else (cols, rows)
+    lib = load_library()
+    if K % 32 != 0 or K <= 0 or outer <= 0:
+        _raise(-2, "mxfp4_quantize_fp8")
+    if codes is None:
+        codes = torch.empty((outer, K), dtype=torch.uint8, device=src.device)
+    if scales is None:
+        scales = torch.empty(scales_bytes(outer, K, scale_layout), dtype=torch.uint8, device=src.device)
+    ld = src.stride(0) if rows > 1 else cols
+    rc = lib.mxfp4_quantize_fp8(_dev_ptr(src), rows, cols, ld, axis, _dev_ptr(codes), _dev_ptr(scales),
+                                scale_layout, _stream())
+    _raise(rc, "mxfp4_quantize_fp8")
+    return codes, scales
+
+
+def gemm_fp8(a_codes, a_scales, b_codes, b_scales, alpha: float = 1.0, out_dtype: int = OUT_BF16, out=None):
+    """``mxfp4_gemm_fp8``: ``alpha * A B^T`` from E4M3 codes [M, K], [N, K] and tiled scales."""
+    M, K = a_codes.shape
+    N, K2 = b_codes.shape
+    if K != K2:
+        raise ValueError("A and B disagree on K")
+    out = _out_tensor((M, N), out_dtype, a_codes.device, out)
+    rc = load_library().mxfp4_gemm_fp8(_dev_ptr(a_codes), _dev_ptr(a_scales), _dev_ptr(b_codes), _dev_ptr(b_scales),
+                                       M, N, K, ctypes.c_float(alpha), _dev_ptr(out), out_dtype, out.stride(0),
+                                       _stream())
+    _raise(rc, "mxfp4_gemm_fp8")
+    return out
+
+
+def linear_pass(pass_: int, precision: int, a, b, hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0,
+                out_dtype=OUT_BF16, workspace=None, out=None):
+    """``mxfp4_linear_pass``: one pass at MXFP4 or MXFP8; (a, b) = (X, W) / (dY, W) / (dY, X)."""
+    for t in (a, b):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise ValueError("inputs must be contiguous bf16 tensors")
+    if pass_ == PASS_FPROP:
+        T, in_f, out_f, shape = a.shape[0], a.shape[1], b.shape[0], (a.shape[0], b.shape[0])
+    elif pass_ == PASS_DGRAD:
+        T, out_f, in_f, shape = a.shape[0], a.shape[1], b.shape[1], (a.shape[0], b.shape[1])
+    else:
+        T, out_f, in_f, shape = a.shape[0], a.shape[1], b.shape[1], (a.shape[1], b.shape[1])
+    lib = load_library()
+    if workspace is None:
+        need = int(lib.mxfp4_linear_pass_workspace_bytes(T, in_f, out_f, pass_, precision))
+        workspace = torch.empty(max(need, 1), dtype=torch.uint8, device=a.device)
+    out = _out_tensor(shape, out_dtype, a.device, out)
+    rc = lib.mxfp4_linear_pass(pass_, precision, _dev_ptr(a), _dev_ptr(b), _dev_ptr(out), T, in_f, out_f,
+                               hadamard_mode, rounding, ctypes.c_uint64(seed), out_dtype, _dev_ptr(workspace),
+                               workspace.numel(), _stream())
+    _raise(rc, "mxfp4_linear_pass")
+    return out
 
 
 def linear_layer_bytes(T: int, in_f: int, out_f: int, which: int) -> int:

@@ -100,12 +100,15 @@ struct GemmPairParams {
 // Instruction descriptor of the pair MMA: E2M1 x E2M1, E8M0 scales, both operands K-major,
 // M = 256 (128 per CTA), N = 192.  Scale-factor ids select which byte pair of the 32-bit TMEM
 // scale column an instruction uses.
-__device__ __forceinline__ uint32_t make_idesc_mxf4_pair(uint32_t a_sf_id, uint32_t b_sf_id)
+// KIND 1 (8-bit operands): E4M3 x E4M3, whose format code under kind::mxf8f6f4 is 0, and the
+// scale-factor id selects one byte of the column.
+template <int KIND>
+__device__ __forceinline__ uint32_t make_idesc_mx_pair(uint32_t a_sf_id, uint32_t b_sf_id)
 {
     uint32_t d = 0;
     d |= b_sf_id << 4;                 // bits 4..5   B scale-factor id
-    d |= 1u << 7;                      // bits 7..9   A format: E2M1
-    d |= 1u << 10;                     // bits 10..12 B format: E2M1
+    d |= (KIND == 0 ? 1u : 0u) << 7;   // bits 7..9   A format: E2M1 (mxf4) / E4M3 (mxf8f6f4)
+    d |= (KIND == 0 ? 1u : 0u) << 10;  // bits 10..12 B format
     d |= (kPMmaN >> 3) << 17;          // bits 17..22 N / 8
     d |= 1u << 23;                     // bit 23      scale format: E8M0
     d |= (kPTileM >> 4) << 24;         // bits 24..28 M / 16
@@ -113,10 +116,18 @@ __device__ __forceinline__ uint32_t make_idesc_mxf4_pair(uint32_t a_sf_id, uint3
     return d;
 }
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
-gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                      const __grid_constant__ CUtensorMap tm_out, const GemmPairParams p)
+// The kernel body for both operand widths.  A stage is 128 bytes of codes per operand row either
+// way -- 256 four-bit or 128 eight-bit elements -- and four MMA K-steps of 32 bytes, so the
+// pipeline, the tile shape and the epilogue are shared; what differs is the instruction kind,
+// the number of 128-element scale tiles a stage covers (two / one) and how an MMA addresses its
+// scales (a byte pair of one of two columns / one byte of one column).
+template <int KIND>
+__device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CUtensorMap& tm_b,
+                                               const CUtensorMap& tm_out, const GemmPairParams& p)
 {
+    constexpr int kBlockK = KIND == 0 ? kPBlockK : kPBlockK / 2;   // elements per stage
+    constexpr int kMmaK = KIND == 0 ? 64 : 32;                     // elements per MMA
+    constexpr int kSfTilesPerStage = KIND == 0 ? 2 : 1;
     extern __shared__ uint8_t smem_raw[];
     GemmPairSmem& sm = *reinterpret_cast<GemmPairSmem*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -177,15 +188,15 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                     // codes: counted on the leader's full barrier
                     const uint32_t full_leader = map_to_cta(smem_u32(&sm.full[s]), 0);
                     mbar_arrive_expect_tx_cluster(full_leader, kPABytes + 2 * kPBSubBytes);
-                    const int32_t x = ks * (kPBlockK / 2);
+                    const int32_t x = ks * 128;                          // bytes along the code row
                     const int32_t ya = tm * kPTileM + rank * kPHalfM;
                     const int32_t yb = tn * kPTileN + rank * kPSubN;
                     tma_load_2d_pair(sm.a[s], &tm_a, full_leader, x, ya);
                     tma_load_2d_pair(sm.b[s][0], &tm_b, full_leader, x, yb);
                     tma_load_2d_pair(sm.b[s][1], &tm_b, full_leader, x, yb + kPMmaN);
                     // scales: local barrier
-                    const int kt0 = ks * 2;
-                    const int nkt = min(2, p.sf_tiles_k - kt0);
+                    const int kt0 = ks * kSfTilesPerStage;
+                    const int nkt = min(kSfTilesPerStage, p.sf_tiles_k - kt0);
                     const uint32_t sf_bytes = nkt * 512;
                     const int has_a = a_row_tile < p.sf_rows_a ? 1 : 0;
                     const int nb0 = tn * 3;
@@ -214,7 +225,9 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
             // descriptors of stage 0; a stage adds a constant, a K = 64 step adds 32 bytes
             const uint64_t a_desc0 = make_smem_desc(smem_u32(sm.a[0]), 16, 1024, 2);
             const uint64_t b_desc0 = make_smem_desc(smem_u32(sm.b[0][0]), 16, 1024, 2);
-            const uint32_t idesc0 = make_idesc_mxf4_pair(0, 0), idesc2 = make_idesc_mxf4_pair(2, 2);
+            // scale-factor ids by K-step: byte pairs 0 / 2 of alternating columns (4-bit), bytes 0..3 (8-bit)
+            const uint32_t idesc0 = make_idesc_mx_pair<KIND>(0, 0), idesc2 = make_idesc_mx_pair<KIND>(2, 2);
+            const uint32_t idesc1 = make_idesc_mx_pair<KIND>(1, 1), idesc3 = make_idesc_mx_pair<KIND>(3, 3);
             int s = 0;
             uint32_t parity = 0;
             for (int tile_it = 0; alive && tile_it < my_tiles; ++tile_it) {
@@ -234,25 +247,25 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
                         rdy_sf = mbar_test_wait(&sm.sf_ready[s1], parity1);
                     }
                     const uint32_t sf_tmem = tmem + kPTmemSfBase + s * kPTmemSfPerBuf;
-                    const int valid_k = min(kPBlockK, p.K - ks * kPBlockK);
-                    const int nmma = (valid_k + 63) / 64;
+                    const int valid_k = min(kBlockK, p.K - ks * kBlockK);
+                    const int nmma = (valid_k + kMmaK - 1) / kMmaK;
                     if (elect_one_sync()) {
                         const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(s * (kPABytes >> 4));
                         const uint64_t b_desc = b_desc0 + static_cast<uint64_t>(s * ((2 * kPBSubBytes) >> 4));
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             if (j < nmma) {
-                                // K = 64 step j: 32 bytes along the 128-byte swizzled row; two
-                                // MMAs, one per 192-column half of the tile
-                                tcgen05_mma_mxf4_pair_collect<0>(tmem, a_desc + 2 * j, b_desc + 2 * j,
-                                                                 (j & 1) ? idesc2 : idesc0, sf_tmem + (j >> 1) * 4,
-                                                                 sf_tmem + 8 + (j >> 1) * 12,
-                                                                 (ks > 0 || j > 0) ? 1u : 0u);
-                                tcgen05_mma_mxf4_pair_collect<1>(tmem + kPMmaN, a_desc + 2 * j,
-                                                                 b_desc + 2 * j + (kPBSubBytes >> 4),
-                                                                 (j & 1) ? idesc2 : idesc0, sf_tmem + (j >> 1) * 4,
-                                                                 sf_tmem + 8 + (j >> 1) * 12 + 6,
-                                                                 (ks > 0 || j > 0) ? 1u : 0u);
+                                // K-step j: 32 bytes along the 128-byte swizzled row; two MMAs, one per
+                                // 192-column half of the tile
+                                const uint32_t idesc = KIND == 0 ? ((j & 1) ? idesc2 : idesc0)
+                                                                 : (j == 0 ? idesc0 : j == 1 ? idesc1 : j == 2 ? idesc2 : idesc3);
+                                const uint32_t sfa = sf_tmem + (KIND == 0 ? (j >> 1) * 4 : 0);
+                                const uint32_t sfb = sf_tmem + 8 + (KIND == 0 ? (j >> 1) * 12 : 0);
+                                tcgen05_mma_mx_pair_collect<KIND, 0>(tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, sfa, sfb,
+                                                                     (ks > 0 || j > 0) ? 1u : 0u);
+                                tcgen05_mma_mx_pair_collect<KIND, 1>(tmem + kPMmaN, a_desc + 2 * j,
+                                                                     b_desc + 2 * j + (kPBSubBytes >> 4), idesc, sfa,
+                                                                     sfb + 6, (ks > 0 || j > 0) ? 1u : 0u);
                             }
                         }
                         // frees the shared-memory stage and its TMEM scale columns in both CTAs
@@ -420,6 +433,23 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_con
     }
 }
 
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
+gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                      const __grid_constant__ CUtensorMap tm_out, const GemmPairParams p)
+{
+    gemm_pair_body<0>(tm_a, tm_b, tm_out, p);
+}
+
+// The 8-bit GEMM of the passes the precision ladder leaves in FP8 (Table 1): E4M3 codes, one
+// byte per element, the same tiled E8M0 scales.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
+gemm_mxf8_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                      const __grid_constant__ CUtensorMap tm_out, const GemmPairParams p)
+{
+    gemm_pair_body<1>(tm_a, tm_b, tm_out, p);
+}
+
+template <int KIND>
 static int launch_gemm_pair(const void* a_codes, const void* a_scales, const void* b_codes,
                             const void* b_scales, int64_t M, int64_t N, int64_t K, float alpha, void* out,
                             int out_dtype, int64_t ld_out, int sm_count, cudaStream_t stream)
@@ -434,10 +464,12 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     } else {
         memset(&tm_out, 0, sizeof(tm_out));
     }
-    // codes as bytes: [rows x K/2], boxes of 128 bytes x 128 rows (A) / 96 rows (B), 128-byte swizzle
-    if (!make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a_codes, M, K / 2, K / 2, kPHalfM, 128,
+    // codes as bytes: [rows x K/2] (4-bit) or [rows x K] (8-bit), boxes of 128 bytes x 128 rows (A) /
+    // 96 rows (B), 128-byte swizzle
+    const int64_t row_bytes = KIND == 0 ? K / 2 : K;
+    if (!make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a_codes, M, row_bytes, row_bytes, kPHalfM, 128,
                       CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b_codes, N, K / 2, K / 2, kPSubN, 128,
+        !make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b_codes, N, row_bytes, row_bytes, kPSubN, 128,
                       CU_TENSOR_MAP_SWIZZLE_128B))
         return MXFP4_ERR_CUDA;
     GemmPairParams p;
@@ -450,7 +482,8 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     p.K = static_cast<int32_t>(K);
     p.tiles_m = static_cast<int32_t>((M + kPTileM - 1) / kPTileM);
     p.tiles_n = static_cast<int32_t>((N + kPTileN - 1) / kPTileN);
-    p.k_stages = static_cast<int32_t>((K + kPBlockK - 1) / kPBlockK);
+    constexpr int kBlockK = KIND == 0 ? kPBlockK : kPBlockK / 2;
+    p.k_stages = static_cast<int32_t>((K + kBlockK - 1) / kBlockK);
     p.sf_tiles_k = static_cast<int32_t>((K + 127) / 128);
     p.sf_rows_a = static_cast<int32_t>((M + 127) / 128);
     p.sf_rows_b = static_cast<int32_t>((N + 127) / 128);
@@ -464,14 +497,16 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(gemm_mxf4_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(KIND == 0 ? gemm_mxf4_pair_kernel : gemm_mxf8_pair_kernel,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess)
             return MXFP4_ERR_CUDA;
         attr_set[dev] = true;
     }
     const int max_clusters = sm_count / 2;
     const int clusters = static_cast<int>(total < max_clusters ? total : max_clusters);
-    gemm_mxf4_pair_kernel<<<2 * clusters, kPThreads, smem, stream>>>(tm_a, tm_b, tm_out, p);
+    if (KIND == 0) gemm_mxf4_pair_kernel<<<2 * clusters, kPThreads, smem, stream>>>(tm_a, tm_b, tm_out, p);
+    else gemm_mxf8_pair_kernel<<<2 * clusters, kPThreads, smem, stream>>>(tm_a, tm_b, tm_out, p);
     return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 

@@ -11,6 +11,7 @@
 #include "tma_host.cuh"
 #include "quantize_kernel.cuh"
 #include "quantize_dual_kernel.cuh"
+#include "quantize_fp8_kernel.cuh"
 #include "gemm_pair_kernel.cuh"
 
 namespace mxfp4 {
@@ -123,7 +124,8 @@ static void fill_quant_params(QuantParams* pp, int64_t outer, int64_t K, int had
 // Validates one tensor's arguments and fills its job (tensor maps + parameters).
 static int build_quant_job(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis,
                            int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
-                           void* codes, void* scales, int scale_layout, QuantJob* job, int block2d = 0)
+                           void* codes, void* scales, int scale_layout, QuantJob* job, int block2d = 0,
+                           int fp8 = 0)
 {
     if (!src_bf16 || !codes || !scales) return MXFP4_ERR_NULL;
     if (axis != 0 && axis != 1) return MXFP4_ERR_ENUM;
@@ -145,8 +147,11 @@ static int build_quant_job(const void* src_bf16, int64_t rows, int64_t cols, int
                                  ld_src * 2, 128, 64, CU_TENSOR_MAP_SWIZZLE_128B)
                   : make_tmap_2d(&job->tm_src, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, src_bf16, rows, cols,
                                  ld_src * 2, 128, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
-    const bool ok_codes = make_tmap_2d(&job->tm_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, outer,
-                                       K / 2, K / 2, 128, 64, CU_TENSOR_MAP_SWIZZLE_64B);
+    const bool ok_codes =
+        fp8 ? make_tmap_2d(&job->tm_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, outer, K, K, 128, 128,
+                           CU_TENSOR_MAP_SWIZZLE_128B)
+            : make_tmap_2d(&job->tm_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, outer, K / 2, K / 2, 128, 64,
+                           CU_TENSOR_MAP_SWIZZLE_64B);
     if (!ok_src || !ok_codes) return MXFP4_ERR_CUDA;
 
     QuantParams& p = job->p;
@@ -169,6 +174,38 @@ static int launch_quant_jobs(const QuantJob& j0, const QuantJob& j1, int axis0, 
     if (axis0 == 1 && axis1 == 0) return dispatch_quantize<1, 0>(hmode, sr, j0, j1, grid, st);
     if (axis0 == 0 && axis1 == 0) return dispatch_quantize<0, 0>(hmode, sr, j0, j1, grid, st);
     return MXFP4_ERR_ENUM;   // (0, 1) is never asked for: callers order row-wise first
+}
+
+template <int AXIS0, int AXIS1>
+static int launch_quantize_fp8(const QuantJob& j0, const QuantJob& j1, int grid, cudaStream_t stream)
+{
+    const size_t smem = sizeof(QuantFp8Smem) + 1024;
+    static bool attr_set[64] = {};          // the attribute is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(quantize_fp8_kernel<AXIS0, AXIS1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess)
+            return MXFP4_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    QuantJobs jobs;
+    jobs.j[0] = j0;
+    jobs.j[1] = j1;
+    quantize_fp8_kernel<AXIS0, AXIS1><<<grid, kQThreads, smem, stream>>>(jobs);
+    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+static int launch_quant_jobs_fp8(const QuantJob& j0, const QuantJob& j1, int axis0, int axis1, cudaStream_t st)
+{
+    const DeviceInfo& dev = device_info();
+    const int64_t total = static_cast<int64_t>(j0.tiles) + j1.tiles;
+    const int grid = static_cast<int>(total < dev.sm_count ? total : dev.sm_count);
+    if (j1.tiles == 0) axis1 = axis0;
+    if (axis0 == 1 && axis1 == 1) return launch_quantize_fp8<1, 1>(j0, j1, grid, st);
+    if (axis0 == 1 && axis1 == 0) return launch_quantize_fp8<1, 0>(j0, j1, grid, st);
+    if (axis0 == 0 && axis1 == 0) return launch_quantize_fp8<0, 0>(j0, j1, grid, st);
+    return MXFP4_ERR_ENUM;
 }
 
 template <int HMODE, int SR>
@@ -209,6 +246,27 @@ __global__ void selftest_wait_timeout_kernel()
 }  // namespace mxfp4
 
 using namespace mxfp4;
+
+template <int KIND>
+static int gemm_checked(const void* a_codes, const void* a_scales, const void* b_codes, const void* b_scales,
+                        int64_t M, int64_t N, int64_t K, float alpha, void* out, int out_dtype, int64_t ld_out,
+                        void* stream)
+{
+    if (!a_codes || !a_scales || !b_codes || !b_scales || !out) return MXFP4_ERR_NULL;
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 32 != 0 || ld_out < N) return MXFP4_ERR_SHAPE;
+    if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (!aligned16(a_codes) || !aligned16(a_scales) || !aligned16(b_codes) || !aligned16(b_scales) ||
+        !aligned16(out))
+        return MXFP4_ERR_ALIGN;
+    const int64_t esz = out_dtype == MXFP4_OUT_BF16 ? 2 : 4;
+    if ((ld_out * esz) % 16 != 0) return MXFP4_ERR_ALIGN;
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return MXFP4_ERR_CUDA;
+    if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
+    return launch_gemm_pair<KIND>(a_codes, a_scales, b_codes, b_scales, M, N, K, alpha, out, out_dtype, ld_out,
+                                  dev.sm_count, static_cast<cudaStream_t>(stream));
+}
 
 extern "C" {
 
@@ -344,20 +402,25 @@ int mxfp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes,
 {
     (void)workspace;
     (void)workspace_bytes;
-    if (!a_codes || !a_scales || !b_codes || !b_scales || !out) return MXFP4_ERR_NULL;
-    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
-    if (M <= 0 || N <= 0 || K <= 0 || K % 32 != 0 || ld_out < N) return MXFP4_ERR_SHAPE;
-    if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
-    if (!aligned16(a_codes) || !aligned16(a_scales) || !aligned16(b_codes) || !aligned16(b_scales) ||
-        !aligned16(out))
-        return MXFP4_ERR_ALIGN;
-    const int64_t esz = out_dtype == MXFP4_OUT_BF16 ? 2 : 4;
-    if ((ld_out * esz) % 16 != 0) return MXFP4_ERR_ALIGN;
-    const DeviceInfo& dev = device_info();
-    if (!dev.ok) return MXFP4_ERR_CUDA;
-    if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
-    return launch_gemm_pair(a_codes, a_scales, b_codes, b_scales, M, N, K, alpha, out, out_dtype, ld_out,
-                            dev.sm_count, static_cast<cudaStream_t>(stream));
+    return gemm_checked<0>(a_codes, a_scales, b_codes, b_scales, M, N, K, alpha, out, out_dtype, ld_out, stream);
+}
+
+int mxfp4_gemm_fp8(const void* a_codes, const void* a_scales, const void* b_codes, const void* b_scales,
+                   int64_t M, int64_t N, int64_t K, float alpha, void* out, int out_dtype, int64_t ld_out,
+                   void* stream)
+{
+    return gemm_checked<1>(a_codes, a_scales, b_codes, b_scales, M, N, K, alpha, out, out_dtype, ld_out, stream);
+}
+
+int mxfp4_quantize_fp8(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis, void* codes,
+                       void* scales, int scale_layout, void* stream)
+{
+    QuantJob j0, j1;
+    const int rc = build_quant_job(src_bf16, rows, cols, ld_src, axis, MXFP4_HADAMARD_NONE, MXFP4_ROUND_RNE, 0, 0u,
+                                   codes, scales, scale_layout, &j0, 0, 1);
+    if (rc != MXFP4_OK) return rc;
+    memset(&j1, 0, sizeof(j1));
+    return launch_quant_jobs_fp8(j0, j1, axis, axis, static_cast<cudaStream_t>(stream));
 }
 
 // Workspace layout of a fused pass: [A codes][A scales][B codes][B scales], each region
@@ -380,24 +443,39 @@ size_t mxfp4_linear_workspace_bytes(int64_t T, int64_t in_features, int64_t out_
            round_up(mxfp4_codes_bytes(N, K), 256) + round_up(mxfp4_scales_bytes(N, K, 1), 256);
 }
 
+static size_t pass_workspace_bytes(int64_t T, int64_t in_features, int64_t out_features, int pass, int precision)
+{
+    if (pass < 0 || pass > 2 || T <= 0 || in_features <= 0 || out_features <= 0) return 0;
+    if (precision != MXFP4_PRECISION_MXFP4 && precision != MXFP4_PRECISION_MXFP8) return 0;
+    int64_t M, N, K;
+    linear_dims(pass, T, in_features, out_features, &M, &N, &K);
+    if (K % 32 != 0) return 0;
+    const size_t mul = precision == MXFP4_PRECISION_MXFP8 ? 2 : 1;     // one byte per element instead of half
+    return round_up(mul * mxfp4_codes_bytes(M, K), 256) + round_up(mxfp4_scales_bytes(M, K, 1), 256) +
+           round_up(mul * mxfp4_codes_bytes(N, K), 256) + round_up(mxfp4_scales_bytes(N, K, 1), 256);
+}
+
 static int linear_pass(int pass, const void* a_src, const void* b_src, void* out, int64_t T,
                        int64_t in_f, int64_t out_f, int hmode, int rounding, uint64_t seed,
-                       int out_dtype, void* workspace, size_t workspace_bytes, void* stream)
+                       int out_dtype, void* workspace, size_t workspace_bytes, void* stream,
+                       int precision = MXFP4_PRECISION_MXFP4)
 {
+    const bool fp8 = precision == MXFP4_PRECISION_MXFP8;
+    const size_t cmul = fp8 ? 2 : 1;
     if (!a_src || !b_src || !out) return MXFP4_ERR_NULL;
     if (T <= 0 || in_f <= 0 || out_f <= 0) return MXFP4_ERR_SHAPE;
     if (hmode < 0 || hmode > 4 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
     int64_t M, N, K;
     linear_dims(pass, T, in_f, out_f, &M, &N, &K);
     if (K % 32 != 0 || in_f % 8 != 0 || out_f % 8 != 0) return MXFP4_ERR_SHAPE;
-    const size_t need = mxfp4_linear_workspace_bytes(T, in_f, out_f, pass);
+    const size_t need = pass_workspace_bytes(T, in_f, out_f, pass, precision);
     if (!workspace || workspace_bytes < need) return MXFP4_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MXFP4_ERR_ALIGN;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     uint8_t* a_codes = ws;
-    uint8_t* a_scales = a_codes + round_up(mxfp4_codes_bytes(M, K), 256);
+    uint8_t* a_scales = a_codes + round_up(cmul * mxfp4_codes_bytes(M, K), 256);
     uint8_t* b_codes = a_scales + round_up(mxfp4_scales_bytes(M, K, 1), 256);
-    uint8_t* b_scales = b_codes + round_up(mxfp4_codes_bytes(N, K), 256);
+    uint8_t* b_scales = b_codes + round_up(cmul * mxfp4_codes_bytes(N, K), 256);
 
     // (rows, cols, axis) of each source in its own row-major shape
     int64_t ar, ac, br, bc;
@@ -411,14 +489,17 @@ static int linear_pass(int pass, const void* a_src, const void* b_src, void* out
     }
     // both operands through one quantize launch
     QuantJob ja, jb;
+    if (fp8) hmode = MXFP4_HADAMARD_NONE, rounding = MXFP4_ROUND_RNE;    // the stabilisers belong to the 4-bit GEMMs
     int rc = build_quant_job(a_src, ar, ac, ac, a_axis, hmode, rounding, seed, 0u, a_codes, a_scales,
-                             MXFP4_SCALES_TILED, &ja);
+                             MXFP4_SCALES_TILED, &ja, 0, fp8);
     if (rc != MXFP4_OK) return rc;
     rc = build_quant_job(b_src, br, bc, bc, b_axis, hmode, rounding, seed, 1u, b_codes, b_scales,
-                         MXFP4_SCALES_TILED, &jb);
+                         MXFP4_SCALES_TILED, &jb, 0, fp8);
     if (rc != MXFP4_OK) return rc;
-    rc = launch_quant_jobs(ja, jb, a_axis, b_axis, hmode, rounding, static_cast<cudaStream_t>(stream));
+    rc = fp8 ? launch_quant_jobs_fp8(ja, jb, a_axis, b_axis, static_cast<cudaStream_t>(stream))
+             : launch_quant_jobs(ja, jb, a_axis, b_axis, hmode, rounding, static_cast<cudaStream_t>(stream));
     if (rc != MXFP4_OK) return rc;
+    if (fp8) return mxfp4_gemm_fp8(a_codes, a_scales, b_codes, b_scales, M, N, K, 1.0f, out, out_dtype, N, stream);
     // H * H^T = n * I for the +-1 matrix of order n: undo it exactly in the epilogue
     const float alpha = hmode == MXFP4_HADAMARD_NONE ? 1.0f : (hmode <= MXFP4_HADAMARD_RAND ? 0.03125f : 0.0625f);
     return mxfp4_gemm(a_codes, a_scales, b_codes, b_scales, M, N, K, alpha, out, out_dtype, N,
@@ -447,6 +528,22 @@ int mxfp4_linear_wgrad(const void* dY, const void* X, void* dW, int64_t T, int64
 {
     return linear_pass(MXFP4_PASS_WGRAD, dY, X, dW, T, in_features, out_features, hadamard_mode,
                        rounding, seed, out_dtype, workspace, workspace_bytes, stream);
+}
+
+size_t mxfp4_linear_pass_workspace_bytes(int64_t T, int64_t in_features, int64_t out_features, int pass,
+                                         int precision)
+{
+    return pass_workspace_bytes(T, in_features, out_features, pass, precision);
+}
+
+int mxfp4_linear_pass(int pass, int precision, const void* a, const void* b, void* out, int64_t T,
+                      int64_t in_features, int64_t out_features, int hadamard_mode, int rounding, uint64_t seed,
+                      int out_dtype, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (pass < 0 || pass > 2) return MXFP4_ERR_ENUM;
+    if (precision != MXFP4_PRECISION_MXFP4 && precision != MXFP4_PRECISION_MXFP8) return MXFP4_ERR_ENUM;
+    return linear_pass(pass, a, b, out, T, in_features, out_features, hadamard_mode, rounding, seed, out_dtype,
+                       workspace, workspace_bytes, stream, precision);
 }
 
 // Operand buffer = [codes][scales], each rounded up to 256 bytes.

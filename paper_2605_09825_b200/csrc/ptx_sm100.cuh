@@ -431,28 +431,30 @@ __device__ __forceinline__ void tcgen05_mma_mxf4_pair(uint32_t d_tmem, uint64_t 
 
 // Pair MMA with an A-collector hint: FILL keeps the A operand in the collector buffer for the
 // next MMA, LASTUSE consumes the kept copy (two MMAs that share A read it from shared memory once).
-template <int LAST>
-__device__ __forceinline__ void tcgen05_mma_mxf4_pair_collect(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
-                                                              uint32_t idesc, uint32_t sfa_tmem,
-                                                              uint32_t sfb_tmem, uint32_t accumulate)
+// KIND 0: 4-bit operands (kind::mxf4, K = 64, two scales per row: scale_vec::2X);
+// KIND 1: 8-bit operands (kind::mxf8f6f4, K = 32, one scale per row: scale_vec::1X).
+#define MXFP4_PAIR_MMA(KIND_STR, HINT)                                                                  \
+    asm volatile(                                                                                       \
+        "{\n\t.reg .pred P;\n\t"                                                                       \
+        "setp.ne.b32 P, %6, 0;\n\t"                                                                     \
+        "tcgen05.mma.cta_group::2." KIND_STR ".collector::a::" HINT " "                                 \
+        "[%0], %1, %2, %3, [%4], [%5], P;\n\t}"                                                         \
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate) \
+        : "memory")
+
+template <int KIND, int LAST>
+__device__ __forceinline__ void tcgen05_mma_mx_pair_collect(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                                            uint32_t idesc, uint32_t sfa_tmem,
+                                                            uint32_t sfb_tmem, uint32_t accumulate)
 {
-    if (LAST) {
-        asm volatile(
-            "{\n\t.reg .pred P;\n\t"
-            "setp.ne.b32 P, %6, 0;\n\t"
-            "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X.collector::a::lastuse "
-            "[%0], %1, %2, %3, [%4], [%5], P;\n\t}"
-            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
-            : "memory");
+    if (KIND == 0) {
+        if (LAST) MXFP4_PAIR_MMA("kind::mxf4.block_scale.scale_vec::2X", "lastuse");
+        else      MXFP4_PAIR_MMA("kind::mxf4.block_scale.scale_vec::2X", "fill");
     } else {
-        asm volatile(
-            "{\n\t.reg .pred P;\n\t"
-            "setp.ne.b32 P, %6, 0;\n\t"
-            "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X.collector::a::fill "
-            "[%0], %1, %2, %3, [%4], [%5], P;\n\t}"
-            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
-            : "memory");
+        if (LAST) MXFP4_PAIR_MMA("kind::mxf8f6f4.block_scale.scale_vec::1X", "lastuse");
+        else      MXFP4_PAIR_MMA("kind::mxf8f6f4.block_scale.scale_vec::1X", "fill");
     }
 }
+#undef MXFP4_PAIR_MMA
 
 }  // namespace mxfp4
