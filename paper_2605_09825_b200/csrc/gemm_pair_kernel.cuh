@@ -161,6 +161,10 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
     cluster_sync_all();           // both CTAs' barriers exist before anyone signals across the pair
     tcgen05_fence_after();
     const uint32_t tmem = sm.tmem_base;
+    // set-up done: let the next kernel's CTAs take SMs as they free up, and do not touch global
+    // memory before the previous kernel in the stream has completed
+    griddep_launch_dependents();
+    griddep_wait();
 
     // register budget per role (whole warpgroups): 4*32*(56 + 2*192 + 56) = 63488 <= 65536;
     // every warp of a warpgroup executes the same setmaxnreg at the top of its role
@@ -505,9 +509,9 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     }
     const int max_clusters = sm_count / 2;
     const int clusters = static_cast<int>(total < max_clusters ? total : max_clusters);
-    if (KIND == 0) gemm_mxf4_pair_kernel<<<2 * clusters, kPThreads, smem, stream>>>(tm_a, tm_b, tm_out, p);
-    else gemm_mxf8_pair_kernel<<<2 * clusters, kPThreads, smem, stream>>>(tm_a, tm_b, tm_out, p);
-    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+    return launch_kernel_pdl(KIND == 0 ? gemm_mxf4_pair_kernel : gemm_mxf8_pair_kernel, 2 * clusters, kPThreads, smem,
+                             stream, tm_a, tm_b, tm_out, p) == cudaSuccess
+               ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
 }  // namespace mxfp4

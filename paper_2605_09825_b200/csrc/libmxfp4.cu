@@ -76,8 +76,8 @@ static int launch_quantize(const QuantJob& j0, const QuantJob& j1, int grid, cud
     QuantJobs jobs;
     jobs.j[0] = j0;
     jobs.j[1] = j1;
-    quantize_kernel<AXIS0, AXIS1, HMODE, SR><<<grid, kQThreads, smem, stream>>>(jobs);
-    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+    return launch_kernel_pdl(quantize_kernel<AXIS0, AXIS1, HMODE, SR>, grid, kQThreads, smem, stream, jobs) == cudaSuccess
+               ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
 template <int AXIS0, int AXIS1>
@@ -192,8 +192,8 @@ static int launch_quantize_fp8(const QuantJob& j0, const QuantJob& j1, int grid,
     QuantJobs jobs;
     jobs.j[0] = j0;
     jobs.j[1] = j1;
-    quantize_fp8_kernel<AXIS0, AXIS1><<<grid, kQThreads, smem, stream>>>(jobs);
-    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+    return launch_kernel_pdl(quantize_fp8_kernel<AXIS0, AXIS1>, grid, kQThreads, smem, stream, jobs) == cudaSuccess
+               ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
 static int launch_quant_jobs_fp8(const QuantJob& j0, const QuantJob& j1, int axis0, int axis1, cudaStream_t st)
@@ -221,8 +221,8 @@ static int launch_quantize_dual(const QuantDualJob& job, int grid, cudaStream_t 
             return MXFP4_ERR_CUDA;
         attr_set[dev] = true;
     }
-    quantize_dual_kernel<HMODE, SR><<<grid, kQThreads, smem, stream>>>(job);
-    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+    return launch_kernel_pdl(quantize_dual_kernel<HMODE, SR>, grid, kQThreads, smem, stream, job) == cudaSuccess
+               ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
 static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -24,6 +24,23 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p)
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// Programmatic dependent launch: every kernel of the library is launched with the
+// programmatic-stream-serialization attribute, so its CTAs may start (barrier set-up, TMEM
+// allocation, descriptor prefetch) while the previous kernel in the stream is still draining.
+// griddep_wait() returns once that previous kernel has completed and its writes are visible;
+// every kernel executes it before its first global-memory access, which keeps stream order
+// transitive.  griddep_launch_dependents() lets the next kernel's CTAs be scheduled as soon as
+// SMs free up.  Both are no-ops for a kernel launched without the attribute.
+__device__ __forceinline__ void griddep_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+__device__ __forceinline__ void griddep_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ uint32_t elect_one_sync()
 {
     uint32_t pred = 0;

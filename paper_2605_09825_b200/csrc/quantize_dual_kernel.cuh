@@ -100,6 +100,8 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
         fence_barrier_init();
     }
     __syncthreads();
+    griddep_launch_dependents();
+    griddep_wait();        // no global-memory access before the previous kernel in the stream is done
 
     if (tid >= kQConsumers) {
         // ------------------------------------------------------------ producer warp

@@ -394,6 +394,8 @@ quantize_kernel(const __grid_constant__ QuantJobs jobs)
         fence_barrier_init();
     }
     __syncthreads();
+    griddep_launch_dependents();
+    griddep_wait();        // no global-memory access before the previous kernel in the stream is done
 
     if (tid >= kQConsumers) {
         // ------------------------------------------------------------ producer warp

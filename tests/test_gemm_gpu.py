@@ -174,3 +174,14 @@ def test_ragged_n_with_padded_leading_dimension(M, N, K, ld, out_dtype):
     ref, S = oracle.gemm(ac, asc, bc, bsc, alpha=0.5)
     assert_gemm_close(big[:, :N].float().cpu().numpy(), ref, S, out_dtype == api.OUT_BF16, "ragged N")
     assert (big[:, N:] == 7.0).all()
+
+
+def test_plain_stream_order_launches_still_work():
+    """MXFP4_PDL=0 turns the programmatic-dependent-launch attribute off; same results."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-c", "import __graft_entry__ as g; g.smoke()"], cwd=root,
+                         env=dict(os.environ, MXFP4_PDL="0"), capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, res.stdout + res.stderr
