@@ -501,22 +501,27 @@ def run_ours(args):
                    "dy": torch.empty(big(lambda o, i: tokens * o), dtype=torch.bfloat16, device="cuda"),
                    "y": out_buf, "dx": out_buf2,
                    "dw": torch.empty(big(lambda o, i: o * i), dtype=torch.bfloat16, device="cuda")}
-            host_out = {"y": out_host,
-                        "dx": torch.empty(big(lambda o, i: tokens * i), dtype=torch.bfloat16).pin_memory(),
-                        "dw": torch.empty(big(lambda o, i: o * i), dtype=torch.bfloat16).pin_memory()}
+            # every linear's results land in host buffers of their own (nothing is overwritten)
+            host_out = {n: {"y": torch.empty(tokens * o, dtype=torch.bfloat16).pin_memory(),
+                            "dx": torch.empty(tokens * i, dtype=torch.bfloat16).pin_memory(),
+                            "dw": torch.empty(o * i, dtype=torch.bfloat16).pin_memory()}
+                        for n, (o, i) in dims.items()}
 
         def e2e_step_layer():
             for n in names:
                 o, i = dims[n]
                 h = pin[n]
                 rc = lib.mxfp4_linear_layer_host(
-                    h["X"].data_ptr(), h["W"].data_ptr(), h["dY"].data_ptr(), host_out["y"].data_ptr(),
-                    host_out["dx"].data_ptr(), host_out["dw"].data_ptr(), tokens, i, o, hmode, rnd, seed,
+                    h["X"].data_ptr(), h["W"].data_ptr(), h["dY"].data_ptr(), host_out[n]["y"].data_ptr(),
+                    host_out[n]["dx"].data_ptr(), host_out[n]["dw"].data_ptr(), tokens, i, o, hmode, rnd, seed,
                     api.OUT_BF16, api.OUT_BF16, api.OUT_BF16, stg["x"].data_ptr(), stg["w"].data_ptr(),
                     stg["dy"].data_ptr(), stg["y"].data_ptr(), stg["dx"].data_ptr(), stg["dw"].data_ptr(),
-                    saved.data_ptr(), saved_bytes, lws.data_ptr(), lws_bytes, sptr)
+                    saved.data_ptr(), saved_bytes, lws.data_ptr(), lws_bytes, sptr, 0)
                 if rc != 0:
                     raise api.Mxfp4Error(rc, "mxfp4_linear_layer_host")
+            rc = lib.mxfp4_linear_layer_host_drain(sptr)      # all results of the step are in host memory
+            if rc != 0:
+                raise api.Mxfp4Error(rc, "mxfp4_linear_layer_host_drain")
 
         e2e_step = e2e_step_layer if layer else e2e_step_per_pass
 
@@ -532,7 +537,8 @@ def run_ours(args):
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
                "ms_per_step": e2e_ms / n_e2e,
                "note": ("mxfp4_linear_layer_host per linear: pinned X, W, dY copied in once each, Y, dX, dW "
-                        "copied out, copies overlapped with each other and the kernels, drained each call"
+                        "copied out to their own host buffers, copies overlapped with each other, with the kernels and "
+                        "across the linears of a step, drained once per step"
                         if layer else
                         "mxfp4_linear_host per pass: pinned host inputs copied in, result copied out, "
                         "stream drained each call")}

@@ -293,7 +293,12 @@ int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* ou
  * once each (the per-pass form copies every tensor twice), on a copy stream of the library's
  * own in the order they are needed; the kernels run on `stream`; Y, dX and dW return on a second
  * copy stream, each as soon as its GEMM has finished, so results flow out while dY still flows
- * in.  The call returns after everything has drained: the three host outputs are valid.
+ * in.  With drain != 0 the call returns after everything has drained: the three host outputs are
+ * valid.  With drain == 0 it returns as soon as the work is queued, so that the next layer's
+ * inputs travel while this layer's results are still on their way back (the next call orders
+ * itself after this one wherever the two share a staging buffer); the host outputs of all
+ * undrained calls are valid after mxfp4_linear_layer_host_drain(stream), and the host inputs must
+ * stay untouched until then.
  *   dev_x, dev_w, dev_dy    device staging for the bf16 inputs ([T x in], [out x in], [T x out]);
  *   dev_y, dev_dx, dev_dw   device staging for the outputs; all six distinct;
  *   saved, workspace        as for forward / backward; workspace must cover the larger of
@@ -305,7 +310,9 @@ int mxfp4_linear_layer_host(const void* X_host, const void* W_host, const void* 
                             void* dX_host, void* dW_host, int64_t T, int64_t in_features, int64_t out_features,
                             int hadamard_mode, int rounding, uint64_t seed, int y_dtype, int dx_dtype, int dw_dtype,
                             void* dev_x, void* dev_w, void* dev_dy, void* dev_y, void* dev_dx, void* dev_dw,
-                            void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream);
+                            void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream,
+                            int drain);
+int mxfp4_linear_layer_host_drain(void* stream);
 
 /*
  * mxfp4_linear_static -- the fused passes for callers that cannot allocate device memory.

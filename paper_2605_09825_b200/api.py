@@ -27,7 +27,7 @@ EXPORTS = (
     "mxfp4_version", "mxfp4_status_string", "mxfp4_codes_bytes", "mxfp4_scales_bytes",
     "mxfp4_quantize", "mxfp4_quantize_2d", "mxfp4_quantize_dual", "mxfp4_quantize_pair", "mxfp4_gemm", "mxfp4_linear_workspace_bytes", "mxfp4_linear_fprop",
     "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_layer_bytes", "mxfp4_linear_forward",
-    "mxfp4_linear_backward", "mxfp4_linear_layer_host", "mxfp4_quantize_fp8", "mxfp4_gemm_fp8",
+    "mxfp4_linear_backward", "mxfp4_linear_layer_host", "mxfp4_linear_layer_host_drain", "mxfp4_quantize_fp8", "mxfp4_gemm_fp8",
     "mxfp4_linear_pass_workspace_bytes", "mxfp4_linear_pass", "mxfp4_linear_host", "mxfp4_linear_static",
     "mxfp4_check", "mxfp4_selftest_wait_timeout",
 )
@@ -101,8 +101,9 @@ def load_library() -> ctypes.CDLL:
     lib.mxfp4_linear_backward.argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, ci, vp, sz, vp, sz, vp]
     lib.mxfp4_linear_backward.restype = ci
     lib.mxfp4_linear_layer_host.argtypes = [vp] * 6 + [i64, i64, i64, ci, ci, u64, ci, ci, ci] + [vp] * 6 + \
-        [vp, sz, vp, sz, vp]
+        [vp, sz, vp, sz, vp, ci]
     lib.mxfp4_linear_layer_host.restype = ci
+    lib.mxfp4_linear_layer_host_drain.argtypes, lib.mxfp4_linear_layer_host_drain.restype = [vp], ci
     lib.mxfp4_linear_host.argtypes = [ci, vp, vp, vp, i64, i64, i64, ci, ci, u64, ci, vp, vp, vp, vp,
                                       sz, vp]
     lib.mxfp4_linear_host.restype = ci
@@ -416,7 +417,7 @@ def linear_backward(dY, saved, in_f: int, hadamard_mode=HADAMARD_DET, rounding=R
 
 def linear_layer_host(X_host, W_host, dY_host, Y_host, dX_host, dW_host, dev: dict, saved, workspace,
                       hadamard_mode=HADAMARD_DET, rounding=ROUND_RNE, seed=0, y_dtype=OUT_BF16,
-                      dx_dtype=OUT_BF16, dw_dtype=OUT_BF16):
+                      dx_dtype=OUT_BF16, dw_dtype=OUT_BF16, drain=True):
     """``mxfp4_linear_layer_host``: forward + backward of one linear from host (ideally pinned)
     tensors into host tensors; ``dev`` maps "x", "w", "dy", "y", "dx", "dw" to device staging."""
     T, in_f = X_host.shape
@@ -426,8 +427,13 @@ def linear_layer_host(X_host, W_host, dY_host, Y_host, dX_host, dW_host, dev: di
         dW_host.data_ptr(), T, in_f, out_f, hadamard_mode, rounding, ctypes.c_uint64(seed), y_dtype, dx_dtype,
         dw_dtype, _dev_ptr(dev["x"]), _dev_ptr(dev["w"]), _dev_ptr(dev["dy"]), _dev_ptr(dev["y"]),
         _dev_ptr(dev["dx"]), _dev_ptr(dev["dw"]), _dev_ptr(saved), saved.numel(), _dev_ptr(workspace),
-        workspace.numel(), _stream())
+        workspace.numel(), _stream(), 1 if drain else 0)
     _raise(rc, "mxfp4_linear_layer_host")
+
+
+def linear_layer_host_drain():
+    """Wait for every undrained ``linear_layer_host`` call on the current stream."""
+    _raise(load_library().mxfp4_linear_layer_host_drain(_stream()), "mxfp4_linear_layer_host_drain")
 
 
 def linear_host(pass_: int, a_host: torch.Tensor, b_host: torch.Tensor, out_host: torch.Tensor, T: int,

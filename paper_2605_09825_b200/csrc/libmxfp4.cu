@@ -685,11 +685,14 @@ static int host_pipe(HostPipe** out)
     return MXFP4_OK;
 }
 
+int mxfp4_linear_layer_host_drain(void* stream);
+
 int mxfp4_linear_layer_host(const void* X_host, const void* W_host, const void* dY_host, void* Y_host,
                             void* dX_host, void* dW_host, int64_t T, int64_t in_features, int64_t out_features,
                             int hadamard_mode, int rounding, uint64_t seed, int y_dtype, int dx_dtype, int dw_dtype,
                             void* dev_x, void* dev_w, void* dev_dy, void* dev_y, void* dev_dx, void* dev_dw,
-                            void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream)
+                            void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream,
+                            int drain)
 {
     if (!X_host || !W_host || !dY_host || !Y_host || !dX_host || !dW_host) return MXFP4_ERR_NULL;
     if (!dev_x || !dev_w || !dev_dy || !dev_y || !dev_dx || !dev_dw) return MXFP4_ERR_NULL;
@@ -720,8 +723,10 @@ int mxfp4_linear_layer_host(const void* X_host, const void* W_host, const void* 
     MXFP4_TRY(cudaEventRecord(hp->xw, hp->h2d));
     MXFP4_TRY(cudaMemcpyAsync(dev_dy, dY_host, dy_bytes, cudaMemcpyHostToDevice, hp->h2d));
     MXFP4_TRY(cudaEventRecord(hp->dy, hp->h2d));
-    // compute on the caller's stream
+    // compute on the caller's stream; the output staging buffers may still be on their way to the
+    // host from the previous call (a no-op wait the first time)
     MXFP4_TRY(cudaStreamWaitEvent(st, hp->xw, 0));
+    MXFP4_TRY(cudaStreamWaitEvent(st, hp->done, 0));
     rc = mxfp4_linear_forward(dev_x, dev_w, dev_y, T, in_features, out_features, hadamard_mode, rounding, seed,
                               y_dtype, saved, saved_bytes, workspace, workspace_bytes, stream);
     if (rc != MXFP4_OK) return rc;
@@ -739,9 +744,18 @@ int mxfp4_linear_layer_host(const void* X_host, const void* W_host, const void* 
     MXFP4_TRY(cudaStreamWaitEvent(hp->d2h, hp->dw, 0));
     MXFP4_TRY(cudaMemcpyAsync(dW_host, dev_dw, dw_out, cudaMemcpyDeviceToHost, hp->d2h));
     MXFP4_TRY(cudaEventRecord(hp->done, hp->d2h));
-    MXFP4_TRY(cudaStreamWaitEvent(st, hp->done, 0));
-    MXFP4_TRY(cudaStreamSynchronize(st));
 #undef MXFP4_TRY
+    return drain ? mxfp4_linear_layer_host_drain(stream) : MXFP4_OK;
+}
+
+int mxfp4_linear_layer_host_drain(void* stream)
+{
+    HostPipe* hp = nullptr;
+    const int rc = host_pipe(&hp);
+    if (rc != MXFP4_OK) return rc;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess ||
+        cudaStreamSynchronize(hp->h2d) != cudaSuccess || cudaStreamSynchronize(hp->d2h) != cudaSuccess)
+        return MXFP4_ERR_CUDA;
     return MXFP4_OK;
 }
 

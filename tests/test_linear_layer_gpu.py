@@ -100,3 +100,29 @@ def test_host_buffer_layer_call_matches_the_device_calls():
         dX, dW = api.linear_backward(dY, sv, in_f, 1, 0, 3, api.OUT_BF16, api.OUT_FP32)
         assert torch.equal(Yh, Y.cpu()) and torch.equal(dXh, dX.cpu()) and torch.equal(dWh, dW.cpu())
         Yh.zero_(); dXh.zero_(); dWh.zero_()
+
+
+def test_undrained_host_calls_overlap_and_keep_their_results():
+    """Three layers queued without draining, sharing one set of staging buffers: every layer's
+    host outputs must be that layer's results once the drain returns."""
+    T, in_f, out_f = 416, 288, 672
+    e = lambda shape, dt: torch.empty(shape, dtype=dt, device="cuda")
+    dev = {"x": e((T, in_f), torch.bfloat16), "w": e((out_f, in_f), torch.bfloat16), "dy": e((T, out_f), torch.bfloat16),
+           "y": e((T, out_f), torch.bfloat16), "dx": e((T, in_f), torch.bfloat16), "dw": e((out_f, in_f), torch.bfloat16)}
+    saved = e(api.linear_layer_bytes(T, in_f, out_f, api.LAYER_SAVED), torch.uint8)
+    ws = e(max(api.linear_layer_bytes(T, in_f, out_f, w) for w in (api.LAYER_FORWARD, api.LAYER_BACKWARD)), torch.uint8)
+    layers = []
+    for k in range(3):
+        bits = _tensors(T, in_f, out_f, 100 + k)
+        host = [torch.from_numpy(b.view(np.int16)).view(torch.bfloat16).pin_memory() for b in bits]
+        outs = [torch.zeros(s_, dtype=torch.bfloat16).pin_memory() for s_ in ((T, out_f), (T, in_f), (out_f, in_f))]
+        layers.append((host, outs))
+    for host, outs in layers:
+        api.linear_layer_host(*host, *outs, dev, saved, ws, 1, 0, 3, drain=False)
+    api.linear_layer_host_drain()
+    api.check()
+    for host, outs in layers:
+        X, W, dY = (h.cuda() for h in host)
+        Y, sv = api.linear_forward(X, W, 1, 0, 3)
+        dX, dW = api.linear_backward(dY, sv, in_f, 1, 0, 3)
+        assert torch.equal(outs[0], Y.cpu()) and torch.equal(outs[1], dX.cpu()) and torch.equal(outs[2], dW.cpu())
