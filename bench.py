@@ -469,6 +469,10 @@ def run_ours(args):
                      "frac": quant_gbs / peaks["hbm_gbs"], "bytes_per_element": q_bytes_per_element,
                      "avg_launch_ms": quant_ms / n_quant, "launches_per_step": n_quant,
                      "traffic": traffic_per_element * quant_bytes / q_bytes_per_element / n_quant}
+    if layer:
+        # the same quantized operands cost two single-axis launches (5.0625 B/element) in the per-pass
+        # schedule: this launch's rate in those terms, for comparison with that schedule's figure
+        quantize_info["as_two_single_axis_passes_gbs"] = quant_gbs * 5.0625 / 3.0625
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region
     e2e = None
