@@ -20,6 +20,14 @@
  *     per byte, element k even in bits 3:0 and k odd in bits 7:4.  A code is
  *     (sign << 3) | magnitude with magnitudes 0..7 = {0, 0.5, 1, 1.5, 2, 3, 4, 6}.
  *   - A scale byte b means 2^(b - 127).
+ *   - Launches use programmatic dependent launch: a kernel's set-up may overlap the tail of the
+ *     previous kernel in the stream, and every kernel waits for that kernel's completion before
+ *     it touches global memory, so stream order is what a caller observes.  MXFP4_PDL=0 in the
+ *     environment (read once) selects plain launches.
+ *   - Host threads: per-device state (function attributes, the copy streams and events of the
+ *     host-buffer layer call, the static scratch address) is created on first use without a
+ *     lock; make the first call on a device from one thread, and do not run two host-buffer
+ *     layer calls on the same device at the same time.
  */
 #ifndef MXFP4_H_
 #define MXFP4_H_
