@@ -57,6 +57,16 @@ def run(pass_name: str = "wgrad", tokens: int = 4096, linear: str = "down", seed
         got = fn(a, b, hmode, rnd, seed, api.OUT_FP32)
         api.check()
         out[name] = round(snr_db(got, ref), 3)
+    # the 32 x 32 block strategy (Appendix D) and the 8-bit format of the ladder's other passes,
+    # from explicit quantize + GEMM calls (operand orientation per pass as in the wrappers)
+    pass_id = {"fprop": api.PASS_FPROP, "dgrad": api.PASS_DGRAD, "wgrad": api.PASS_WGRAD}[pass_name]
+    ax_a, ax_b = ((1, 1), (1, 0), (0, 0))[pass_id]
+    for name, hmode, alpha in (("none_32x32", api.HADAMARD_NONE, 1.0), ("det_h32_32x32", api.HADAMARD_DET, 1.0 / 32)):
+        qa = api.quantize(a, ax_a, hmode, api.ROUND_RNE, seed, 0, block_shape=api.BLOCK_32X32)
+        qb = api.quantize(b, ax_b, hmode, api.ROUND_RNE, seed, 1, block_shape=api.BLOCK_32X32)
+        out[name] = round(snr_db(api.gemm(*qa, *qb, alpha, api.OUT_FP32), ref), 3)
+    out["mxfp8"] = round(snr_db(api.linear_pass(pass_id, api.PRECISION_MXFP8, a, b, out_dtype=api.OUT_FP32), ref), 3)
+    api.check()
     return {"pass": pass_name, "linear": linear, "tokens": tokens, "seed": seed, "snr_db": out,
             "inputs": "synthetic: dY Student-t(3)*1e-3, X |N|*N (down) or N(0,1)+outlier channels, W N(0,0.02^2)"}
 
