@@ -323,6 +323,7 @@ def run_ours(args):
 
     gemm_ms = gemm_flops = quant_ms = quant_bytes = 0.0
     n_quant = 0
+    gemm_by_shape = {}      # per launch, M x N x K -> TFLOP/s inside the step (tile and wave effects show here)
     r256 = lambda v: (v + 255) // 256 * 256
 
     def operand_views(buf, off, outer, K):
@@ -362,8 +363,9 @@ def run_ours(args):
                 api.gemm(dyt_c, dyt_s, xt_c, xt_s, alpha, api.OUT_BF16, out=out_buf2[: o * i].view(o, i))
                 ev[7].record(stream)
                 evs.append(([(ev[0], ev[1], T * i), (ev[1], ev[2], o * i), (ev[4], ev[5], T * o)],
-                            [(ev[2], ev[3], 2.0 * T * o * i), (ev[5], ev[6], 2.0 * T * o * i),
-                             (ev[6], ev[7], 2.0 * T * o * i)]))
+                            [(ev[2], ev[3], 2.0 * T * o * i, f"{n} fprop {T}x{o}x{i}"),
+                             (ev[5], ev[6], 2.0 * T * o * i, f"{n} dgrad {T}x{i}x{o}"),
+                             (ev[6], ev[7], 2.0 * T * o * i, f"{n} wgrad {o}x{i}x{T}")]))
         else:
             for (n, p, a, b, M, N, K) in passes:
                 ax_a, ax_b = a_b_axes(p)
@@ -385,7 +387,8 @@ def run_ours(args):
                 ev[1].record(stream)
                 api.gemm(ac, a_s, bc, b_s, alpha, api.OUT_BF16, out=out_buf[: M * N].view(M, N))
                 ev[2].record(stream)
-                evs.append(([(ev[0], ev[1], (M + N) * K)], [(ev[1], ev[2], 2.0 * M * N * K)]))
+                evs.append(([(ev[0], ev[1], (M + N) * K)],
+                            [(ev[1], ev[2], 2.0 * M * N * K, f"{n} {('fprop', 'dgrad', 'wgrad')[p]} {M}x{N}x{K}")]))
         torch.cuda.synchronize()
         if rep == 0:
             continue   # first decomposed pass is a warm-up
@@ -394,9 +397,10 @@ def run_ours(args):
                 quant_ms += a0.elapsed_time(a1)
                 quant_bytes += elems * q_bytes_per_element
                 n_quant += 1
-            for a0, a1, fl in gs:
+            for a0, a1, fl, label in gs:
                 gemm_ms += a0.elapsed_time(a1)
                 gemm_flops += fl
+                gemm_by_shape[label] = round(fl / (a0.elapsed_time(a1) * 1e-3) / 1e12, 1)
     clocks = sampler.stop(t_begin, t_end)
     api.check()
 
@@ -457,6 +461,7 @@ def run_ours(args):
         "peak_source": f"4 x sustained cuBLAS bf16 ({peaks['source']}); burst would be "
                        f"{4.0 * peaks['bf16_tflops']:.0f}, nominal dense FP4 9000",
         "flops_per_launch": gemm_flops / n_gemm, "avg_launch_ms": gemm_ms / n_gemm,
+        "tflops_by_launch": gemm_by_shape,
     }
     quant_gbs = quant_bytes / (quant_ms * 1e-3) / 1e9
     # ncu, single-axis kernel on a 117.4 M-element tensor: 234.9 MB read + 45.4 MB written = 2.39 B
