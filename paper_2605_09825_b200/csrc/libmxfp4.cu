@@ -270,7 +270,7 @@ static int gemm_checked(const void* a_codes, const void* a_scales, const void* b
 
 extern "C" {
 
-int mxfp4_version(void) { return 100; }
+int mxfp4_version(void) { return 103; }   // 1.3: + pair/dual/2D quantize, layer-level calls, 8-bit passes
 
 const char* mxfp4_status_string(int status)
 {
