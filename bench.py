@@ -31,6 +31,7 @@ import subprocess
 import sys
 import threading
 import time
+import zlib
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
@@ -222,8 +223,11 @@ def run_ours(args):
 
     # ---- inputs: seeded synthetic, generated on the host, then resident in HBM
     host, dev_in = {}, {}
+    checksums = {}
     for n in names:
         t = synth.linear_tensors(n, tokens, 5)
+        if rank == 0 and not args.no_checksums:
+            checksums[n] = {k: f"{zlib.crc32(memoryview(np.ascontiguousarray(v)).cast('B')):08x}" for k, v in t.items()}
         host[n] = {k: torch.from_numpy(v.view(np.int16)).view(torch.bfloat16) for k, v in t.items()}
         dev_in[n] = {k: v.cuda() for k, v in host[n].items()}
     dims = {n: synth.LLAMA8B_LINEARS[n] for n in names}   # (out, in)
@@ -605,6 +609,7 @@ def run_ours(args):
                    "schedule": ("layer: forward + backward per linear, each of X, W, dY read once by the dual-axis "
                                 "quantize" if layer else "per pass: both operands of each pass quantized from bf16"),
                    "flops_per_step": flops_per_step, "out_dtype": "bf16",
+                   "input_crc32": checksums,
                    "l2": "inputs larger than L2 (several GB per step), no flush needed",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "roofline": roofline, "quantize": quantize_info, "mxfp8_passes": fp8_info,
@@ -618,6 +623,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--no-checksums", action="store_true", help="skip the CRC-32 of the input tensors")
     ap.add_argument("--mxfp4-passes", default="fprop,dgrad,wgrad",
                     help="precision ladder: comma-separated passes that run MXFP4 (the rest run MXFP8); 'none' or '' "
                          "for the all-8-bit baseline; anything but all three implies --schedule per_pass")
