@@ -19,11 +19,23 @@
 namespace mxfp4 {
 
 constexpr int kQDStages = 4;
+// Consumer-group width per variant.  256: two groups of 256 threads on alternate tiles, double-
+// buffered staging.  128: four groups of 128 threads, each thread doing a tile's blocks in two
+// sub-passes, single-buffered staging -- four different phases per scheduler instead of two, which
+// keeps the FMA and ALU pipes busier for the deterministic rotations (7-9 % faster there) but
+// costs the un-rotated, HBM-bound variant 10 % and changes nothing for the others.
+template <int HMODE, int SR>
+struct QuantDualShape {
+    static constexpr int kGroupThreads = ((HMODE == 1 || HMODE == 3) && SR == 0) ? 128 : 256;
+    static constexpr int kGroups = kQConsumers / kGroupThreads;
+    static constexpr int kSub = 256 / kGroupThreads;
+    static constexpr int kBufs = kGroups == 2 ? 2 : 1;
+};
 
 struct QuantDualSmem {
     alignas(1024) uint8_t stage[kQDStages][kQStageBytes];
-    alignas(1024) uint8_t code_tile[2][2][2][kQCodeTileBytes];   // [group][double buffer][orientation]
-    alignas(128) uint8_t scale_tile[2][2][2][kQScaleTileBytes];
+    alignas(1024) uint8_t code_tile[8][kQCodeTileBytes];     // [(group * buffers + buffer) * 2 + orientation]
+    alignas(128) uint8_t scale_tile[8][kQScaleTileBytes];
     alignas(8) uint64_t full[kQDStages];
     uint64_t empty[kQDStages];
     int abort_flag;
@@ -84,6 +96,9 @@ template <int HMODE, int SR>
 __global__ void __launch_bounds__(kQThreads, 1)
 quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
 {
+    using Shape = QuantDualShape<HMODE, SR>;
+    constexpr int kQDGroupThreads = Shape::kGroupThreads, kQDGroups = Shape::kGroups, kQDSub = Shape::kSub,
+                  kQDBufs = Shape::kBufs;
     extern __shared__ uint8_t smem_raw[];
     QuantDualSmem& sm = *reinterpret_cast<QuantDualSmem*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -95,7 +110,7 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
         sm.abort_flag = 0;
         for (int s = 0; s < kQDStages; ++s) {
             mbar_init(&sm.full[s], 1);
-            mbar_init(&sm.empty[s], kQConsumers / 64);      // the 8 warps of one consumer group
+            mbar_init(&sm.empty[s], kQDGroupThreads / 32);  // the warps of one consumer group
         }
         fence_barrier_init();
     }
@@ -122,12 +137,8 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
     }
 
     // ---------------------------------------------------------------- consumers
-    const int grp = tid >> 8;          // consumer group: takes tiles grp, grp + 2, ...
-    const int t = tid & 255;
-    const int kbh = t >> 7;            // row-wise: blocks kbh and kbh + 2 of source row o
-    const int o = t & 127;
-    const int kbc = t >> 6;            // column-wise: block kbc of source columns 2*jc, 2*jc + 1
-    const int jc = t & 63;
+    const int grp = tid / kQDGroupThreads;     // consumer group: takes tiles grp, grp + kQDGroups, ...
+    const int t = tid % kQDGroupThreads;
     // the 16 lanes that share a 32-column group (a 32 x 32 region of the transposed operand)
     const uint32_t half_mask = (tid & 16) ? 0xFFFF0000u : 0x0000FFFFu;
     const QuantParams& pr = job.pr;
@@ -138,64 +149,79 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
     }
 
     int trip = 0;
-    for (int it = grp; it < my_tiles; it += 2, ++trip) {
+    for (int it = grp; it < my_tiles; it += kQDGroups, ++trip) {
         const int tile = blockIdx.x + it * gridDim.x;
         const int tr = tile / job.tiles_c, tc = tile % job.tiles_c;
         const int s = it % kQDStages;
         const uint32_t round = it / kQDStages;
-        const int buf = trip & 1;
+        const int slot = (grp * kQDBufs + (kQDBufs == 2 ? (trip & 1) : 0)) * 2;   // staging tiles of this trip
         const bool ok = mbar_wait(&sm.full[s], round & 1, &sm.abort_flag);
+        if (kQDBufs == 1) {
+            // single staging buffer: last trip's stores must have read it before anyone rewrites it
+            if (t == 0) bulk_wait_group_read<0>();
+            asm volatile("barrier.cta.sync %0, %1;" ::"r"(grp + 1), "n"(kQDGroupThreads) : "memory");
+        }
 
         float2 P0[16], P1[16];
         uint32_t packed[4], byte;
-
-        // ---- row-wise operand: operand row = source row, K = columns
-        if (ok) {
-            load_block<1, HMODE>(&sm.stage[s][0], kbh, o, pr.sign_mask, P0);
-            load_block<1, HMODE>(&sm.stage[s][0], kbh + 2, o, pr.sign_mask, P1);
-        } else {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
-        }
-        {
-            const uint64_t e_row = static_cast<uint64_t>(tr * 128 + o) * static_cast<uint64_t>(pr.K);
-            uint8_t* ct = &sm.code_tile[grp][buf][0][0];
-            uint8_t* st = &sm.scale_tile[grp][buf][0][0];
-            quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tc * 4 + kbh) * 32), pr, packed, byte);
-            stage_block(ct, st, pr, o, kbh, tr, tc, packed, byte, ok);
-            quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tc * 4 + kbh + 2) * 32), pr, packed, byte);
-            stage_block(ct, st, pr, o, kbh + 2, tr, tc, packed, byte, ok);
-        }
+        for (int u = 0; u < kQDSub; ++u) {
+            const int tv = t + u * kQDGroupThreads;     // position in the 256-thread layout of a tile
+            const int kbh = tv >> 7;                    // row-wise: blocks kbh and kbh + 2 of source row o
+            const int o = tv & 127;
+            const int kbc = tv >> 6;                    // column-wise: block kbc of source columns 2*jc, 2*jc + 1
+            const int jc = tv & 63;
 
-        // ---- column-wise operand: operand row = source column, K = rows
-        if (ok) {
-            load_column_blocks<HMODE>(&sm.stage[s][0], kbc, jc, pc.sign_mask, P0, P1);
-        } else {
+            // ---- row-wise operand: operand row = source row, K = columns
+            if (ok) {
+                load_block<1, HMODE>(&sm.stage[s][0], kbh, o, pr.sign_mask, P0);
+                load_block<1, HMODE>(&sm.stage[s][0], kbh + 2, o, pr.sign_mask, P1);
+            } else {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
-        }
-        // the stage is in registers now: hand it back to the producer
-        __syncwarp();
-        if ((tid & 31) == 0) mbar_arrive(&sm.empty[s]);
-        {
-            float amax0 = rotate_and_amax<HMODE>(P0);
-            float amax1 = rotate_and_amax<HMODE>(P1);
-            if (pc.block2d) amax0 = amax1 = lanes_max(half_mask, fmaxf(amax0, amax1));
-            const uint64_t e_blk = static_cast<uint64_t>((tr * 4 + kbc) * 32);
-            const uint64_t e_row = static_cast<uint64_t>(tc * 128 + 2 * jc) * static_cast<uint64_t>(pc.K);
-            uint8_t* ct = &sm.code_tile[grp][buf][1][0];
-            uint8_t* st = &sm.scale_tile[grp][buf][1][0];
-            scale_round_pack<SR>(P0, amax0, e_row + e_blk, pc, packed, byte);
-            stage_block(ct, st, pc, 2 * jc, kbc, tc, tr, packed, byte, ok);
-            scale_round_pack<SR>(P1, amax1, e_row + static_cast<uint64_t>(pc.K) + e_blk, pc, packed, byte);
-            stage_block(ct, st, pc, 2 * jc + 1, kbc, tc, tr, packed, byte, ok);
+                for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
+            }
+            {
+                const uint64_t e_row = static_cast<uint64_t>(tr * 128 + o) * static_cast<uint64_t>(pr.K);
+                uint8_t* ct = &sm.code_tile[slot][0];
+                uint8_t* st = &sm.scale_tile[slot][0];
+                quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tc * 4 + kbh) * 32), pr, packed, byte);
+                stage_block(ct, st, pr, o, kbh, tr, tc, packed, byte, ok);
+                quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tc * 4 + kbh + 2) * 32), pr, packed, byte);
+                stage_block(ct, st, pr, o, kbh + 2, tr, tc, packed, byte, ok);
+            }
+
+            // ---- column-wise operand: operand row = source column, K = rows
+            if (ok) {
+                load_column_blocks<HMODE>(&sm.stage[s][0], kbc, jc, pc.sign_mask, P0, P1);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
+            }
+            if (u == kQDSub - 1) {
+                // the stage is in registers now: hand it back to the producer
+                __syncwarp();
+                if ((tid & 31) == 0) mbar_arrive(&sm.empty[s]);
+            }
+            {
+                float amax0 = rotate_and_amax<HMODE>(P0);
+                float amax1 = rotate_and_amax<HMODE>(P1);
+                if (pc.block2d) amax0 = amax1 = lanes_max(half_mask, fmaxf(amax0, amax1));
+                const uint64_t e_blk = static_cast<uint64_t>((tr * 4 + kbc) * 32);
+                const uint64_t e_row = static_cast<uint64_t>(tc * 128 + 2 * jc) * static_cast<uint64_t>(pc.K);
+                uint8_t* ct = &sm.code_tile[slot + 1][0];
+                uint8_t* st = &sm.scale_tile[slot + 1][0];
+                scale_round_pack<SR>(P0, amax0, e_row + e_blk, pc, packed, byte);
+                stage_block(ct, st, pc, 2 * jc, kbc, tc, tr, packed, byte, ok);
+                scale_round_pack<SR>(P1, amax1, e_row + static_cast<uint64_t>(pc.K) + e_blk, pc, packed, byte);
+                stage_block(ct, st, pc, 2 * jc + 1, kbc, tc, tr, packed, byte, ok);
+            }
         }
 
         fence_proxy_async_smem();
-        // the stores this group issued one trip ago must have drained their buffers before the
-        // next trip (which every thread of the group reaches only through the barrier below)
-        // overwrites them
-        if (t == 0) bulk_wait_group_read<0>();
+        // double-buffered staging: the stores this group issued one trip ago must have drained
+        // their buffers before the next trip (which every thread of the group reaches only
+        // through the barrier below) overwrites them
+        if (kQDBufs == 2 && t == 0) bulk_wait_group_read<0>();
         uint32_t any_fail;
         asm volatile(
             "{\n\t.reg .pred P, Q;\n\t"
@@ -203,17 +229,17 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
             "barrier.cta.red.or.pred P, %2, %3, Q;\n\t"
             "selp.u32 %0, 1, 0, P;\n\t}"
             : "=r"(any_fail)
-            : "r"(ok ? 0u : 1u), "r"(grp + 1), "n"(kQConsumers / 2)
+            : "r"(ok ? 0u : 1u), "r"(grp + 1), "n"(kQDGroupThreads)
             : "memory");
         if (any_fail) break;
         if (t == 0) {
-            tma_store_2d(&job.tm_codes_row, &sm.code_tile[grp][buf][0][0], tc * 64, tr * 128);
-            tma_store_2d(&job.tm_codes_col, &sm.code_tile[grp][buf][1][0], tr * 64, tc * 128);
+            tma_store_2d(&job.tm_codes_row, &sm.code_tile[slot][0], tc * 64, tr * 128);
+            tma_store_2d(&job.tm_codes_col, &sm.code_tile[slot + 1][0], tr * 64, tc * 128);
             if (pr.scale_layout == 1) {
                 bulk_store_1d(pr.scales + (static_cast<int64_t>(tr) * pr.tiles_k + tc) * kQScaleTileBytes,
-                              &sm.scale_tile[grp][buf][0][0], kQScaleTileBytes);
+                              &sm.scale_tile[slot][0], kQScaleTileBytes);
                 bulk_store_1d(pc.scales + (static_cast<int64_t>(tc) * pc.tiles_k + tr) * kQScaleTileBytes,
-                              &sm.scale_tile[grp][buf][1][0], kQScaleTileBytes);
+                              &sm.scale_tile[slot + 1][0], kQScaleTileBytes);
             }
             bulk_commit_group();
         }
