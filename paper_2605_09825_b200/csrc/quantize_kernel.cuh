@@ -38,8 +38,8 @@ constexpr int kQScaleTileBytes = 512;
 
 struct QuantSmem {
     alignas(1024) uint8_t stage[kQStages][kQStageBytes];
-    alignas(1024) uint8_t code_tile[2][2][kQCodeTileBytes];    // [consumer group][double buffer]
-    alignas(128) uint8_t scale_tile[2][2][kQScaleTileBytes];
+    alignas(1024) uint8_t code_tile[4][kQCodeTileBytes];       // [consumer group * buffers + buffer]
+    alignas(128) uint8_t scale_tile[4][kQScaleTileBytes];
     alignas(8) uint64_t full[kQStages];
     uint64_t empty[kQStages];
     int abort_flag;
@@ -297,12 +297,112 @@ __device__ __forceinline__ void issue_tile_load(const CUtensorMap* tm_src, const
     }
 }
 
+// Consumer-group width per variant.  256: two groups of 256 threads on alternate tiles,
+// double-buffered staging.  128: four groups of 128 threads, each thread doing a tile's blocks in
+// two sub-passes, single-buffered staging: four different phases per scheduler instead of two keep
+// the FMA and ALU pipes busier for the deterministic rotations; the other variants (HBM-bound
+// without rotation, integer-bound with stochastic rounding) do not gain from it.
+template <int HMODE, int SR>
+struct QuantShape {
+    static constexpr int kGroupThreads = ((HMODE == 1 || HMODE == 3) && SR == 0) ? 128 : 256;
+    static constexpr int kGroups = kQConsumers / kGroupThreads;
+    static constexpr int kSub = 256 / kGroupThreads;
+    static constexpr int kBufs = kGroups == 2 ? 2 : 1;
+};
+
+// Four groups of 128 threads: the same work per tile in two sub-passes per thread.
+template <int AXIS, int HMODE, int SR>
+__device__ __forceinline__ bool consume_tile_narrow(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
+                                             int tile, int it, int trip, int grp, int t)
+{
+    using Shape = QuantShape<HMODE, SR>;
+    const int s = it % kQStages;
+    const uint32_t round = it / kQStages;
+    const int slot = grp * Shape::kBufs + (Shape::kBufs == 2 ? (trip & 1) : 0);   // staging tile of this trip
+    int to, tk;
+    tile_coords<AXIS>(p, tile, to, tk);
+
+    const bool ok = mbar_wait(&sm.full[s], round & 1, &sm.abort_flag);
+    if (Shape::kBufs == 1) {
+        // single staging buffer: last trip's store must have read it before anyone rewrites it
+        if (t == 0) bulk_wait_group_read<0>();
+        asm volatile("barrier.cta.sync %0, %1;" ::"r"(grp + 1), "n"(Shape::kGroupThreads) : "memory");
+    }
+
+#pragma unroll
+    for (int u = 0; u < Shape::kSub; ++u) {
+        const int tv = t + u * Shape::kGroupThreads;   // position in the 256-thread layout of a tile
+        const int kbh = tv >> 7;                       // this thread's blocks along K: kbh and kbh + 2
+        const int o = tv & 127;                        // operand row inside the tile
+        float2 P0[16], P1[16];
+        if (ok) {
+            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.sign_mask, P0);
+            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.sign_mask, P1);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
+        }
+        if (u == Shape::kSub - 1) {
+            // the stage is in registers now: hand it back to the producer
+            __syncwarp();
+            if ((t & 31) == 0) mbar_arrive(&sm.empty[s]);
+        }
+
+        const uint64_t e_row = static_cast<uint64_t>(to * kQTileO + o) * static_cast<uint64_t>(p.K);
+        uint32_t packed0[4], packed1[4], byte0, byte1;
+        quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tk * 4 + kbh) * 32), p, packed0, byte0);
+        quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tk * 4 + kbh + 2) * 32), p, packed1, byte1);
+
+        // stage the results: codes in the 64-byte swizzle the TMA store expects
+        uint8_t* ct = &sm.code_tile[slot][o * 64];
+        *reinterpret_cast<uint4*>(ct + ((kbh ^ ((o >> 1) & 3)) * 16)) =
+            make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]);
+        *reinterpret_cast<uint4*>(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16)) =
+            make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]);
+        if (p.scale_layout == 1) {
+            uint8_t* st = &sm.scale_tile[slot][(o & 31) * 16 + (o >> 5) * 4];
+            st[kbh] = static_cast<uint8_t>(byte0);
+            st[kbh + 2] = static_cast<uint8_t>(byte1);
+        } else if (ok) {
+            const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
+            const int64_t tg = static_cast<int64_t>(tk) * 4 + kbh;
+            if (og < p.outer && tg < p.nt) p.scales[og * p.nt + tg] = static_cast<uint8_t>(byte0);
+            if (og < p.outer && tg + 2 < p.nt) p.scales[og * p.nt + tg + 2] = static_cast<uint8_t>(byte1);
+        }
+    }
+    fence_proxy_async_smem();
+    // double-buffered staging: the store this group issued one trip ago must have drained its
+    // buffer before the next trip (which every thread of the group reaches only through the
+    // barrier below) overwrites it
+    if (Shape::kBufs == 2 && t == 0) bulk_wait_group_read<0>();
+    uint32_t any_fail;
+    asm volatile(
+        "{\n\t.reg .pred P, Q;\n\t"
+        "setp.ne.u32 Q, %1, 0;\n\t"
+        "barrier.cta.red.or.pred P, %2, %3, Q;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(any_fail)
+        : "r"(ok ? 0u : 1u), "r"(grp + 1), "n"(Shape::kGroupThreads)
+        : "memory");
+    if (any_fail) return false;
+    if (t == 0) {
+        tma_store_2d(tm_codes, &sm.code_tile[slot][0], tk * (kQTileK / 2), to * kQTileO);
+        if (p.scale_layout == 1)
+            bulk_store_1d(p.scales + (static_cast<int64_t>(to) * p.tiles_k + tk) * kQScaleTileBytes,
+                          &sm.scale_tile[slot][0], kQScaleTileBytes);
+        bulk_commit_group();
+    }
+    return true;
+}
+
 // One tile of one job, as seen by a consumer thread: wait for the stage, rotate + quantize this
 // thread's two blocks, stage codes and scales, and (thread 0 of the group) store them.  `p` and
 // `tm_codes` refer to kernel parameters, so every field is a constant-bank operand.  Returns
 // false when a wait gave up (the group leaves the kernel).
+// Two groups of 256 threads: a thread handles two blocks of its group's tile (the form every
+// variant but the deterministic rotations uses).
 template <int AXIS, int HMODE, int SR>
-__device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
+__device__ __forceinline__ bool consume_tile_wide(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
                                              int tile, int it, int trip, int grp, int t)
 {
     const int kbh = t >> 7;            // this thread's blocks along K: kbh and kbh + 2
@@ -333,13 +433,13 @@ __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p
     quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tk * 4 + kbh + 2) * 32), p, packed1, byte1);
 
     // stage the results: codes in the 64-byte swizzle the TMA store expects
-    uint8_t* ct = &sm.code_tile[grp][buf][o * 64];
+    uint8_t* ct = &sm.code_tile[grp * 2 + buf][o * 64];
     *reinterpret_cast<uint4*>(ct + ((kbh ^ ((o >> 1) & 3)) * 16)) =
         make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]);
     *reinterpret_cast<uint4*>(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16)) =
         make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]);
     if (p.scale_layout == 1) {
-        uint8_t* st = &sm.scale_tile[grp][buf][(o & 31) * 16 + (o >> 5) * 4];
+        uint8_t* st = &sm.scale_tile[grp * 2 + buf][(o & 31) * 16 + (o >> 5) * 4];
         st[kbh] = static_cast<uint8_t>(byte0);
         st[kbh + 2] = static_cast<uint8_t>(byte1);
     } else if (ok) {
@@ -364,19 +464,29 @@ __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p
         : "memory");
     if (any_fail) return false;
     if (t == 0) {
-        tma_store_2d(tm_codes, &sm.code_tile[grp][buf][0], tk * (kQTileK / 2), to * kQTileO);
+        tma_store_2d(tm_codes, &sm.code_tile[grp * 2 + buf][0], tk * (kQTileK / 2), to * kQTileO);
         if (p.scale_layout == 1)
             bulk_store_1d(p.scales + (static_cast<int64_t>(to) * p.tiles_k + tk) * kQScaleTileBytes,
-                          &sm.scale_tile[grp][buf][0], kQScaleTileBytes);
+                          &sm.scale_tile[grp * 2 + buf][0], kQScaleTileBytes);
         bulk_commit_group();
     }
     return true;
+}
+
+template <int AXIS, int HMODE, int SR>
+__device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
+                                             int tile, int it, int trip, int grp, int t)
+{
+    if (QuantShape<HMODE, SR>::kGroups == 2)
+        return consume_tile_wide<AXIS, HMODE, SR>(sm, p, tm_codes, tile, it, trip, grp, t);
+    return consume_tile_narrow<AXIS, HMODE, SR>(sm, p, tm_codes, tile, it, trip, grp, t);
 }
 
 template <int AXIS0, int AXIS1, int HMODE, int SR>
 __global__ void __launch_bounds__(kQThreads, 1)
 quantize_kernel(const __grid_constant__ QuantJobs jobs)
 {
+    using Shape = QuantShape<HMODE, SR>;
     extern __shared__ uint8_t smem_raw[];
     QuantSmem& sm = *reinterpret_cast<QuantSmem*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -389,7 +499,7 @@ quantize_kernel(const __grid_constant__ QuantJobs jobs)
         sm.abort_flag = 0;
         for (int s = 0; s < kQStages; ++s) {
             mbar_init(&sm.full[s], 1);
-            mbar_init(&sm.empty[s], kQConsumers / 64);      // the 8 warps of one consumer group
+            mbar_init(&sm.empty[s], Shape::kGroupThreads / 32);   // the warps of one consumer group
         }
         fence_barrier_init();
     }
@@ -418,8 +528,8 @@ quantize_kernel(const __grid_constant__ QuantJobs jobs)
     }
 
     // ---------------------------------------------------------------- consumers
-    const int grp = tid >> 8;          // consumer group: takes tiles grp, grp + 2, ...
-    const int t = tid & 255;
+    const int grp = tid / Shape::kGroupThreads;     // consumer group: takes tiles grp, grp + kGroups, ...
+    const int t = tid % Shape::kGroupThreads;
     if (t == 0) {
         tma_prefetch_desc(&jobs.j[0].tm_codes);
         if (jobs.j[1].tiles > 0) tma_prefetch_desc(&jobs.j[1].tm_codes);
@@ -429,14 +539,14 @@ quantize_kernel(const __grid_constant__ QuantJobs jobs)
     // through a loop specialised for that job's axis and parameters
     int it = grp, trip = 0;
     bool alive = true;
-    for (; it < my_tiles; it += 2, ++trip) {
+    for (; it < my_tiles; it += Shape::kGroups, ++trip) {
         const int gtile = blockIdx.x + it * gridDim.x;
         if (gtile >= tiles0) break;
         alive = consume_tile<AXIS0, HMODE, SR>(sm, jobs.j[0].p, &jobs.j[0].tm_codes, gtile, it, trip, grp, t);
         if (!alive) break;
     }
     if (alive) {
-        for (; it < my_tiles; it += 2, ++trip) {
+        for (; it < my_tiles; it += Shape::kGroups, ++trip) {
             const int gtile = blockIdx.x + it * gridDim.x;
             if (!consume_tile<AXIS1, HMODE, SR>(sm, jobs.j[1].p, &jobs.j[1].tm_codes, gtile - tiles0, it, trip,
                                                 grp, t))
