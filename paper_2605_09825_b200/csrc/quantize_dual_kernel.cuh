@@ -23,7 +23,8 @@ constexpr int kQDStages = 4;
 // buffered staging.  128: four groups of 128 threads, each thread doing a tile's blocks in two
 // sub-passes, single-buffered staging -- four different phases per scheduler instead of two, which
 // keeps the FMA and ALU pipes busier for the deterministic rotations (7-9 % faster there) but
-// costs the un-rotated, HBM-bound variant 10 % and changes nothing for the others.
+// costs the un-rotated variant and the stochastic-rounding ones 5-20 % here (the kernel has
+// less register headroom than the single-axis one) and changes nothing for the randomized rotations.
 template <int HMODE, int SR>
 struct QuantDualShape {
     static constexpr int kGroupThreads = ((HMODE == 1 || HMODE == 3) && SR == 0) ? 128 : 256;

