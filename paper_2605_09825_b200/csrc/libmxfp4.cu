@@ -117,6 +117,9 @@ static void fill_quant_params(QuantParams* pp, int64_t outer, int64_t K, int had
         const uint32_t m16 = host_sign_mask(seed) & 0xFFFFu;   // same 16 signs for both halves
         p.sign_mask = m16 | (m16 << 16);
     }
+    for (int i = 0; i < 16; ++i)
+        p.signs.pair[i] = (((p.sign_mask >> (2 * i)) & 1u) << 15) | (((p.sign_mask >> (2 * i + 1)) & 1u) << 31);
+    for (int k = 0; k < 32; ++k) p.signs.word[k] = ((p.sign_mask >> k) & 1u) ? 0x80008000u : 0u;
     p.scale_layout = scale_layout;
     p.block2d = block2d;
 }

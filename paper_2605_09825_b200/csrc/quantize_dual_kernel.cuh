@@ -27,7 +27,7 @@ constexpr int kQDStages = 4;
 // less register headroom than the single-axis one) and changes nothing for the randomized rotations.
 template <int HMODE, int SR>
 struct QuantDualShape {
-    static constexpr int kGroupThreads = ((HMODE == 1 || HMODE == 3) && SR == 0) ? 128 : 256;
+    static constexpr int kGroupThreads = (HMODE != 0 && SR == 0) ? 128 : 256;
     static constexpr int kGroups = kQConsumers / kGroupThreads;
     static constexpr int kSub = 256 / kGroupThreads;
     static constexpr int kBufs = kGroups == 2 ? 2 : 1;
@@ -56,7 +56,7 @@ struct QuantDualJob {
 // applied on the way in.  Element (r, c) of the tile sits at
 //   (c / 64) * 16384 + r * 128 + (((c % 64) / 8) ^ (r % 8)) * 16 + (c % 8) * 2.
 template <int HMODE>
-__device__ __forceinline__ void load_column_blocks(const uint8_t* stage, int kb, int jc, uint32_t sign_mask,
+__device__ __forceinline__ void load_column_blocks(const uint8_t* stage, int kb, int jc, const QuantSigns& sg,
                                                    float2 (&PA)[16], float2 (&PB)[16])
 {
     const int w = jc & 31;                                  // 4-byte word inside the 128-byte row
@@ -64,14 +64,18 @@ __device__ __forceinline__ void load_column_blocks(const uint8_t* stage, int kb,
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
         const int r0 = 2 * i, r1 = 2 * i + 1;               // rows of the block; (kb*32 + r) % 8 == r % 8
-        const uint32_t w0 = *reinterpret_cast<const uint32_t*>(stage + ((base ^ ((r0 & 7) << 4)) + r0 * 128));
-        const uint32_t w1 = *reinterpret_cast<const uint32_t*>(stage + ((base ^ ((r1 & 7) << 4)) + r1 * 128));
-        if (HMODE == 1 || HMODE == 3) {
+        uint32_t w0 = *reinterpret_cast<const uint32_t*>(stage + ((base ^ ((r0 & 7) << 4)) + r0 * 128));
+        uint32_t w1 = *reinterpret_cast<const uint32_t*>(stage + ((base ^ ((r1 & 7) << 4)) + r1 * 128));
+        if (HMODE == 2 || HMODE == 4) {                     // element r of both columns shares its sign
+            w0 ^= sg.word[r0];
+            w1 ^= sg.word[r1];
+        }
+        if (HMODE != 0) {
             PA[i] = first_stage_pair_bf16(w0, __uint_as_float(w1 << 16));
             PB[i] = first_stage_pair_bf16(w0 >> 16, __uint_as_float(w1 & 0xFFFF0000u));
         } else {
-            PA[i] = first_stage_pair<HMODE>(i, w0 << 16, w1 << 16, sign_mask);
-            PB[i] = first_stage_pair<HMODE>(i, w0 & 0xFFFF0000u, w1 & 0xFFFF0000u, sign_mask);
+            PA[i] = make_float2(__uint_as_float(w0 << 16), __uint_as_float(w1 << 16));
+            PB[i] = make_float2(__uint_as_float(w0 & 0xFFFF0000u), __uint_as_float(w1 & 0xFFFF0000u));
         }
     }
 }
@@ -175,8 +179,8 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
 
             // ---- row-wise operand: operand row = source row, K = columns
             if (ok) {
-                load_block<1, HMODE>(&sm.stage[s][0], kbh, o, pr.sign_mask, P0);
-                load_block<1, HMODE>(&sm.stage[s][0], kbh + 2, o, pr.sign_mask, P1);
+                load_block<1, HMODE>(&sm.stage[s][0], kbh, o, pr.signs, P0);
+                load_block<1, HMODE>(&sm.stage[s][0], kbh + 2, o, pr.signs, P1);
             } else {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
@@ -193,7 +197,7 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
 
             // ---- column-wise operand: operand row = source column, K = rows
             if (ok) {
-                load_column_blocks<HMODE>(&sm.stage[s][0], kbc, jc, pc.sign_mask, P0, P1);
+                load_column_blocks<HMODE>(&sm.stage[s][0], kbc, jc, pc.signs, P0, P1);
             } else {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);

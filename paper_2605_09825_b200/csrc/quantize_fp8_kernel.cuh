@@ -66,8 +66,8 @@ __device__ __forceinline__ bool consume_tile_fp8(QuantFp8Smem& sm, const QuantPa
     const bool ok = mbar_wait(&sm.full[s], round & 1, &sm.abort_flag);
     float2 P0[16], P1[16];
     if (ok) {
-        load_block<AXIS, 0>(&sm.stage[s][0], kbh, o, 0u, P0);
-        load_block<AXIS, 0>(&sm.stage[s][0], kbh + 2, o, 0u, P1);
+        load_block<AXIS, 0>(&sm.stage[s][0], kbh, o, p.signs, P0);
+        load_block<AXIS, 0>(&sm.stage[s][0], kbh + 2, o, p.signs, P1);
     } else {
 #pragma unroll
         for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);

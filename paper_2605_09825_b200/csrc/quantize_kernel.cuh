@@ -45,7 +45,18 @@ struct QuantSmem {
     int abort_flag;
 };
 
+// Sign diagonal of the randomized rotation as XOR words for raw bf16 data (all zero otherwise):
+// pair[i] flips elements 2i (bit 15) and 2i+1 (bit 31) of a word holding two consecutive elements;
+// word[k] = 0x80008000 if element k is flipped, for words holding element k of two columns (or
+// one zero-extended element).  Built on the host from the 32-bit mask; read as constant-bank
+// operands, so a flip costs one logic instruction per loaded word.
+struct QuantSigns {
+    uint32_t pair[16];
+    uint32_t word[32];
+};
+
 struct QuantParams {
+    QuantSigns signs;
     uint8_t* scales;
     int64_t outer, K;        // operand view
     int64_t nt;              // K / 32
@@ -109,19 +120,6 @@ __device__ __forceinline__ void fwht32_pair_stage(float2 (&P)[16])
     }
 }
 
-// Pair (element 2i, element 2i+1) of a block from the two fp32 bit patterns: optional sign
-// diagonal, then the h = 1 butterfly (the pair's halves are each other's partners).
-template <int HMODE>
-__device__ __forceinline__ float2 first_stage_pair(int i, uint32_t lo_bits, uint32_t hi_bits, uint32_t sign_mask)
-{
-    if (HMODE == 2 || HMODE == 4) {
-        lo_bits ^= (sign_mask << (31 - 2 * i)) & 0x80000000u;
-        hi_bits ^= (sign_mask << (30 - 2 * i)) & 0x80000000u;
-    }
-    const float a = __uint_as_float(lo_bits), b = __uint_as_float(hi_bits);
-    return HMODE != 0 ? make_float2(__fadd_rn(a, b), __fsub_rn(a, b)) : make_float2(a, b);
-}
-
 // Eight E2M1 codes (one 32-bit word of packed output) from eight floats, round-to-nearest-even,
 // saturating; v0 lands in bits 3:0, v7 in bits 31:28.
 __device__ __forceinline__ uint32_t cvt_e2m1x8(float v0, float v1, float v2, float v3, float v4,
@@ -163,12 +161,15 @@ __device__ __forceinline__ float2 first_stage_pair_bf16(uint32_t a_bits, float b
     return make_float2(s, d);
 }
 
-// One 32-element block out of a shared-memory stage into registers as 16 pairs (sign diagonal
-// and first butterfly stage applied on the way in).
+// One 32-element block out of a shared-memory stage into registers as 16 pairs.  The sign
+// diagonal of the randomized modes is applied to the raw bf16 bits (a sign flip commutes with the
+// exact widening), after which every rotated mode takes the same mixed-precision first butterfly
+// stage; without rotation the pair is just widened.
 template <int AXIS, int HMODE>
-__device__ __forceinline__ void load_block(const uint8_t* stage, int kb, int o, uint32_t sign_mask,
+__device__ __forceinline__ void load_block(const uint8_t* stage, int kb, int o, const QuantSigns& sg,
                                            float2 (&P)[16])
 {
+    constexpr bool kRand = HMODE == 2 || HMODE == 4;
     if (AXIS == 1) {
         const uint8_t* base = stage + (kb >> 1) * (kQStageBytes / 2) + o * 128;
 #pragma unroll
@@ -177,20 +178,25 @@ __device__ __forceinline__ void load_block(const uint8_t* stage, int kb, int o, 
             const uint4 q = *reinterpret_cast<const uint4*>(base + chunk);
             const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                P[4 * j + i] = (HMODE == 1 || HMODE == 3)
-                                   ? first_stage_pair_bf16(w[i], __uint_as_float(w[i] & 0xFFFF0000u))
-                                   : first_stage_pair<HMODE>(4 * j + i, w[i] * 65536u, w[i] & 0xFFFF0000u, sign_mask);
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t wv = kRand ? (w[i] ^ sg.pair[4 * j + i]) : w[i];
+                P[4 * j + i] = HMODE != 0 ? first_stage_pair_bf16(wv, __uint_as_float(wv & 0xFFFF0000u))
+                                          : make_float2(__uint_as_float(wv << 16), __uint_as_float(wv & 0xFFFF0000u));
+            }
         }
     } else {
         const uint16_t* base = reinterpret_cast<const uint16_t*>(stage) + (kb * 32) * 128 + o;
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
-            P[i] = (HMODE == 1 || HMODE == 3)
-                       ? first_stage_pair_bf16(base[(2 * i) * 128],
-                                               __uint_as_float(static_cast<uint32_t>(base[(2 * i + 1) * 128]) * 65536u))
-                       : first_stage_pair<HMODE>(i, static_cast<uint32_t>(base[(2 * i) * 128]) * 65536u,
-                                                 static_cast<uint32_t>(base[(2 * i + 1) * 128]) * 65536u, sign_mask);
+        for (int i = 0; i < 16; ++i) {
+            // zero-extended elements; the flip word's upper half falls off in the shift / the 16-bit operand
+            uint32_t a = base[(2 * i) * 128], b = base[(2 * i + 1) * 128];
+            if (kRand) {
+                a ^= sg.word[2 * i];
+                b ^= sg.word[2 * i + 1];
+            }
+            P[i] = HMODE != 0 ? first_stage_pair_bf16(a, __uint_as_float(b << 16))
+                              : make_float2(__uint_as_float(a << 16), __uint_as_float(b << 16));
+        }
     }
 }
 
@@ -339,8 +345,8 @@ __device__ __forceinline__ bool consume_tile_narrow(QuantSmem& sm, const QuantPa
         const int o = tv & 127;                        // operand row inside the tile
         float2 P0[16], P1[16];
         if (ok) {
-            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.sign_mask, P0);
-            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.sign_mask, P1);
+            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.signs, P0);
+            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.signs, P1);
         } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
@@ -419,8 +425,8 @@ __device__ __forceinline__ bool consume_tile_wide(QuantSmem& sm, const QuantPara
 
     float2 P0[16], P1[16];
     if (ok) {
-        load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.sign_mask, P0);
-        load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.sign_mask, P1);
+        load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.signs, P0);
+        load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.signs, P1);
     } else {
 #pragma unroll
         for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
