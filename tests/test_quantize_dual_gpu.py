@@ -118,3 +118,49 @@ def test_dual_rejects_bad_arguments():
     with pytest.raises(api.Mxfp4Error) as exc:
         api.quantize_dual(to_dev(random_bits(rng, 64, 64)), block_shape=2)
     assert exc.value.status == -4
+
+
+def test_dual_special_values_in_both_orientations():
+    """Every finite bf16 pattern as the only non-zero element of its row-wise block AND of its
+    column-wise block (so no rotation overflows), plus a region of negative zeros: sub-normal block
+    maxima, the scale clamp, signed zeros and saturation reach both paths of the kernel."""
+    pats = np.array([p for p in range(1 << 16) if ((p >> 7) & 0xFF) != 0xFF], dtype=np.uint16)
+    rows, cols = 8192 + 32, 256
+    bits = np.zeros((rows, cols), dtype=np.uint16)
+    k = np.arange(len(pats))
+    r, cb = k // 8, k % 8                                    # one pattern per (row, 32-column block) ...
+    bits[r, cb * 32 + r % 32] = pats                         # ... and per (32-row group, column)
+    bits[-32:, :] = 0x8000                                   # a region of negative zeros
+    for hmode, rnd in ((0, 0), (1, 0), (3, 1), (2, 0)):
+        (cr, sr), (cc, sc) = api.quantize_dual(to_dev(bits), hmode, rnd, 5)
+        api.check()
+        _assert_operand(cr, sr, *oracle.quantize(bits, 1, hmode, rnd, 5, 0), what=f"row-wise mode {hmode}")
+        _assert_operand(cc, sc, *oracle.quantize(bits, 0, hmode, rnd, 5, 1), what=f"column-wise mode {hmode}")
+
+
+def test_dual_canary_bytes_around_all_four_outputs():
+    import torch
+    rng = np.random.default_rng(31)
+    rows, cols = 224, 160
+    src = to_dev(random_bits(rng, rows, cols))
+    pad = 4096
+    sizes = (api.codes_bytes(rows, cols), api.scales_bytes(rows, cols), api.codes_bytes(cols, rows),
+             api.scales_bytes(cols, rows))
+    bufs = [torch.full((n + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda") for n in sizes]
+    view = lambda b, n: b[pad:pad + n]
+    api.quantize_dual(src, 1, 0, 0,
+                      out_row=(view(bufs[0], sizes[0]).view(rows, cols // 2), view(bufs[1], sizes[1])),
+                      out_col=(view(bufs[2], sizes[2]).view(cols, rows // 2), view(bufs[3], sizes[3])))
+    api.check()
+    for b, n in zip(bufs, sizes):
+        assert (b[:pad] == 0xA5).all() and (b[pad + n:] == 0xA5).all()
+
+
+def test_dual_is_reproducible_run_to_run():
+    t = synth.config1()
+    a = api.quantize_dual(to_dev(t["X"]), 2, 1, 7)
+    b = api.quantize_dual(to_dev(t["X"]), 2, 1, 7)
+    api.check()
+    import torch
+    for (x0, x1), (y0, y1) in zip(a, b):
+        assert torch.equal(x0, y0) and torch.equal(x1, y1)
