@@ -118,7 +118,9 @@ size_t mxfp4_scales_bytes(int64_t outer, int64_t K, int scale_layout);
  *   operand_tag  decorrelates the stochastic-rounding streams of different operands.
  *   codes        out, [outer x K/2] bytes, 16-byte aligned.
  *   scales       out, mxfp4_scales_bytes(outer, K, scale_layout) bytes, 16-byte aligned.
- * Inputs must be finite.
+ * Inputs must be finite; with a rotation the 32-term (16-term) sums of a block must stay finite
+ * in fp32 too, i.e. magnitudes below about 1e37 (overflowing blocks are outside the contract: the
+ * result is then unspecified, never a fault).
  */
 int mxfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis,
                    int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
