@@ -94,7 +94,7 @@ struct GemmPairParams {
     int32_t sf_rows_b;          // ceil(N / 128)
     float alpha;
     int32_t out_fp32;
-    int32_t n_tma;              // bf16 output: columns written by TMA stores (N rounded down to 8)
+    int32_t n_tma;              // columns written by TMA stores: N rounded down to a 16-byte granule (8 bf16 / 4 fp32)
 };
 
 // Instruction descriptor of the pair MMA: E2M1 x E2M1, E8M0 scales, both operands K-major,
@@ -340,23 +340,38 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
                     }
+                    // three passes of 32 columns: the warp lays its 32 rows x 128 bytes out in the
+                    // 128-byte swizzle and one lane hands the box to a TMA store, as for bf16
 #pragma unroll
                     for (int c = 0; c < 3; ++c) {
                         const int64_t col0 = colbase + round * 96 + c * 32;
-                        if (row >= p.M || col0 >= p.N) continue;
-                        float* dst = static_cast<float*>(p.out) + row * p.ld_out + col0;
-                        if (col0 + 32 <= p.N) {
+                        if (lane == 0) bulk_wait_group_read<0>();
+                        __syncwarp();
 #pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                reinterpret_cast<float4*>(dst)[i] =
-                                    make_float4(__uint_as_float(r[c][4 * i]) * p.alpha,
-                                                __uint_as_float(r[c][4 * i + 1]) * p.alpha,
-                                                __uint_as_float(r[c][4 * i + 2]) * p.alpha,
-                                                __uint_as_float(r[c][4 * i + 3]) * p.alpha);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (col0 + i < p.N) dst[i] = __uint_as_float(r[c][i]) * p.alpha;
+                        for (int q = 0; q < 8; ++q)
+                            *reinterpret_cast<float4*>(stg + lane * 128 + ((q ^ (lane & 7)) * 16)) =
+                                make_float4(__uint_as_float(r[c][4 * q]) * p.alpha, __uint_as_float(r[c][4 * q + 1]) * p.alpha,
+                                            __uint_as_float(r[c][4 * q + 2]) * p.alpha,
+                                            __uint_as_float(r[c][4 * q + 3]) * p.alpha);
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (p.n_tma < p.N) {
+                            // N is not a multiple of 4: the tensor map ends at the last full 16-byte
+                            // granule; the one to three columns after it come from the staged row
+                            const int64_t rc = p.n_tma - col0;
+                            if (rc >= 0 && rc < 32 && row < p.M) {
+                                const int q = static_cast<int>(rc >> 2);
+                                const float4 v = *reinterpret_cast<const float4*>(stg + lane * 128 + ((q ^ (lane & 7)) * 16));
+                                const float e[4] = {v.x, v.y, v.z, v.w};
+                                float* dst = static_cast<float*>(p.out) + row * p.ld_out + p.n_tma;
+                                for (int k = 0; k < 3; ++k)
+                                    if (p.n_tma + k < p.N) dst[k] = e[k];
+                            }
+                        }
+                        if (lane == 0 && row0 < p.M && col0 < p.n_tma) {
+                            tma_store_2d_hint(&tm_out, stg, static_cast<int32_t>(col0), static_cast<int32_t>(row0),
+                                              store_policy);
+                            bulk_commit_group();
                         }
                     }
                 }
@@ -459,10 +474,12 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
                             int out_dtype, int64_t ld_out, int sm_count, cudaStream_t stream)
 {
     CUtensorMap tm_a, tm_b, tm_out;
-    // bf16 output through TMA stores of 64 columns x 32 rows (fp32 output is stored directly)
-    const int64_t n_tma = out_dtype == MXFP4_OUT_BF16 ? (N & ~static_cast<int64_t>(7)) : 0;
+    // output through TMA stores of 128-byte x 32-row boxes: 64 bf16 or 32 fp32 columns
+    const bool bf16_out = out_dtype == MXFP4_OUT_BF16;
+    const int64_t n_tma = bf16_out ? (N & ~static_cast<int64_t>(7)) : (N & ~static_cast<int64_t>(3));
     if (n_tma > 0) {
-        if (!make_tmap_2d(&tm_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, out, M, n_tma, ld_out * 2, 32, 64,
+        if (!make_tmap_2d(&tm_out, bf16_out ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                          bf16_out ? 2 : 4, out, M, n_tma, ld_out * (bf16_out ? 2 : 4), 32, bf16_out ? 64 : 32,
                           CU_TENSOR_MAP_SWIZZLE_128B))
             return MXFP4_ERR_CUDA;
     } else {
