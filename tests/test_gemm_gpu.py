@@ -161,9 +161,11 @@ def test_an_expired_bounded_wait_is_reported_and_the_context_stays_usable():
 
 
 @pytest.mark.parametrize("M,N,K,ld,out_dtype", [(130, 100, 32, 104, api.OUT_BF16), (257, 50, 160, 52, api.OUT_FP32),
-                                                (64, 385, 64, 392, api.OUT_BF16), (300, 769, 288, 776, api.OUT_FP32)])
+                                                (64, 385, 64, 392, api.OUT_BF16), (300, 769, 288, 776, api.OUT_FP32),
+                                                (33, 3, 32, 4, api.OUT_FP32), (40, 7, 64, 8, api.OUT_BF16),
+                                                (129, 391, 96, 392, api.OUT_FP32)])
 def test_ragged_n_with_padded_leading_dimension(M, N, K, ld, out_dtype):
-    # N is not a multiple of the 8-element store granule; the columns between N and ld must stay untouched
+    # N is not a multiple of the 16-byte store granule (8 bf16 / 4 fp32), down to N smaller than one granule; the columns between N and ld must stay untouched
     rng = np.random.default_rng(M + N + K)
     ac, asc, bc, bsc = _random_operands(rng, M, N, K)
     dt = torch.bfloat16 if out_dtype == api.OUT_BF16 else torch.float32
