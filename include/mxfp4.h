@@ -306,7 +306,8 @@ int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* ou
  * in.  With drain != 0 the call returns after everything has drained: the three host outputs are
  * valid.  With drain == 0 it returns as soon as the work is queued, so that the next layer's
  * inputs travel while this layer's results are still on their way back (the next call orders
- * itself after this one wherever the two share a staging buffer); the host outputs of all
+ * itself after this one wherever the two share a staging buffer, provided both use the same
+ * `stream`); the host outputs of all
  * undrained calls are valid after mxfp4_linear_layer_host_drain(stream), and the host inputs must
  * stay untouched until then.
  *   dev_x, dev_w, dev_dy    device staging for the bf16 inputs ([T x in], [out x in], [T x out]);
