@@ -6,6 +6,7 @@ from fractions import Fraction
 import numpy as np
 
 import oracle
+from conftest import read_golden_lines
 from test_oracle_pins import (GRID, bf16_bits, bf16_fraction, expected_scale_byte, nearest_code, unpack)
 
 
@@ -43,20 +44,21 @@ def test_2d_blocks_are_transpose_invariant_without_rotation():
 
 
 def test_hand_worked_region_with_one_outlier():
-    """32 x 32 of ones with one 48: the region's largest magnitude is 48 = 1.5 * 2^5, so the
-    scale is 2^(5-2) = 8 (byte 130) for every row; 48 / 8 = 6 -> code 7, 1 / 8 = 0.125 -> code 0
-    (below the 0.25 midpoint).  Per-row blocks would give the other rows scale 2^-2 and code 6."""
+    """The region worked by hand in tests/golden/worked_blocks_32x32_and_mxfp8.txt: 32 x 32 of ones
+    with one 48."""
+    g = [ln.split() for ln in read_golden_lines("worked_blocks_32x32_and_mxfp8.txt") if ln.startswith("region32x32")][0]
+    byte2d, code48, code1_2d, byte1d, code1_1d = (int(x) for x in g[1:])
     vals = np.full((32, 32), bf16_bits(1.0), dtype=np.uint16)
     vals[5, 9] = bf16_bits(48.0)
     codes, scales = oracle.quantize(vals, 1, 0, 0, block2d=True)
-    assert (scales == 130).all()
+    assert (scales == byte2d).all()
     nib = _nibbles(codes)
-    assert nib[5, 9] == 7
-    nib[5, 9] = 0
-    assert (nib == 0).all()
+    assert nib[5, 9] == code48
+    nib[5, 9] = code1_2d
+    assert (nib == code1_2d).all()
     codes1, scales1 = oracle.quantize(vals, 1, 0, 0)
-    assert scales1[5, 0] == 130 and (np.delete(scales1[:, 0], 5) == 125).all()
-    assert (np.delete(_nibbles(codes1), 5, axis=0) == 6).all()
+    assert scales1[5, 0] == byte2d and (np.delete(scales1[:, 0], 5) == byte1d).all()
+    assert (np.delete(_nibbles(codes1), 5, axis=0) == code1_1d).all()
 
 
 def test_brute_force_in_rational_arithmetic_with_a_ragged_last_region():

@@ -7,6 +7,7 @@ import numpy as np
 import torch
 
 import oracle
+from conftest import read_golden_lines
 from test_oracle_pins import bf16_bits, bf16_fraction, floor_log2
 
 
@@ -74,14 +75,13 @@ def test_encode_is_the_nearest_grid_point_ties_to_even_and_saturates():
 
 
 def test_hand_worked_block():
-    """Block maximum 3 = 1.5 * 2^1 -> scale 2^(1-8) (byte 120); 3 / 2^-7 = 384 = 1.5 * 2^8 ->
-    code (8+7)<<3 | 4 = 0x7C.  1 -> 128 = 2^7 -> 0x70.  -0.75 -> -96 = -1.5 * 2^6 -> 0xEC.
-    2^-15 -> 2^-8 = 2 sub-normal steps -> 0x02.  2^-17 -> 2^-10 = half a step, tie -> 0."""
+    """The block worked by hand in tests/golden/worked_blocks_32x32_and_mxfp8.txt."""
+    g = [ln.split() for ln in read_golden_lines("worked_blocks_32x32_and_mxfp8.txt") if ln.startswith("mxfp8_block")][0]
     vals = [3.0, 1.0, -0.75, 2.0 ** -15, 2.0 ** -17] + [0.0] * 27
     bits = np.array([[bf16_bits(v) for v in vals]], dtype=np.uint16)
     codes, scales = oracle.quantize_mxfp8(bits, 1)
-    assert scales[0, 0] == 120
-    assert codes[0, :5].tolist() == [0x7C, 0x70, 0xEC, 0x02, 0x00]
+    assert scales[0, 0] == int(g[1])
+    assert codes[0, :5].tolist() == [int(x, 16) for x in g[2:7]]
     assert (codes[0, 5:] == 0).all()
 
 
