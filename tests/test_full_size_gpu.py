@@ -111,3 +111,30 @@ def test_config3_dual_quantize_of_the_largest_tensor():
         wc, ws = oracle.quantize(t["dY"], axis, 1, 0, 0, 0)
         assert (codes.cpu().numpy() == wc).all()
         assert (oracle.scales_from_tiled(scales.cpu().numpy(), wc.shape[0], wc.shape[1] * 2 // 32) == ws).all()
+
+
+def test_eight_times_the_benchmark_token_count():
+    """131072 tokens (1 GiB of bf16 activations, 2^29 elements): index arithmetic beyond the
+    benchmark's sizes.  Dual-axis quantize bit-exact on the whole tensor in both orientations,
+    Fprop and Wgrad outputs on sampled rows."""
+    T, in_f, out_f = 131072, 4096, 1024
+    t = synth.linear_tensors("o", T, 6)                  # X [T x 4096], W, dY [T x 4096]
+    Xb, Wb, dYb = t["X"], np.ascontiguousarray(t["W"][:out_f]), np.ascontiguousarray(t["dY"][:, :out_f])
+    X, W, dY = to_dev(Xb), to_dev(Wb), to_dev(dYb)
+    (cr, sr), (cc, sc) = api.quantize_dual(X, 1, 0, 0, tags=(0, 1))
+    api.check()
+    for codes, scales, axis, tag in ((cr, sr, 1, 0), (cc, sc, 0, 1)):
+        wc, ws = oracle.quantize(Xb, axis, 1, 0, 0, tag)
+        assert (codes.cpu().numpy() == wc).all()
+        assert (oracle.scales_from_tiled(scales.cpu().numpy(), wc.shape[0], wc.shape[1] * 2 // 32) == ws).all()
+        del wc, ws
+    del cr, sr, cc, sc
+    Y, saved = api.linear_forward(X, W, 1, 0, 0)
+    dX, dW = api.linear_backward(dY, saved, in_f, 1, 0, 0, api.OUT_BF16, api.OUT_FP32)
+    api.check()
+    rows = _rows(T, 99, n_random=8)
+    ref, S = oracle.linear_fprop(Xb, Wb, 1, 0, 0, rows=rows)
+    assert_gemm_close(Y[torch.from_numpy(rows).cuda()].float().cpu().numpy(), ref, S, True, "fprop at 131072 tokens")
+    rows = _rows(out_f, 98, n_random=4)
+    ref, S = oracle.linear_wgrad(dYb, Xb, 1, 0, 0, rows=rows)
+    assert_gemm_close(dW[torch.from_numpy(rows).cuda()].cpu().numpy(), ref, S, False, "wgrad over 131072 tokens")
