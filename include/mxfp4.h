@@ -72,6 +72,7 @@ extern "C" {
 
 #define MXFP4_PRECISION_MXFP4 0 /* E2M1 elements, the method's GEMMs                              */
 #define MXFP4_PRECISION_MXFP8 1 /* E4M3 elements, the passes the ladder of Table 1 leaves in FP8  */
+#define MXFP4_PRECISION_MXFP4_32X32 2 /* MXFP4 with Appendix D's 32 x 32 blocks for both operands */
 
 #define MXFP4_OUT_BF16 0
 #define MXFP4_OUT_FP32 1
@@ -238,7 +239,8 @@ int mxfp4_linear_wgrad(const void* dY, const void* X, void* dW, int64_t T, int64
  * mxfp4_gemm_fp8: as mxfp4_gemm on such operands (tcgen05 kind::mxf8f6f4, fp32 accumulation).
  * mxfp4_linear_pass: one pass at a chosen precision; (a, b, out) = (X, W, Y) / (dY, W, dX) /
  *   (dY, X, dW) for MXFP4_PASS_FPROP / _DGRAD / _WGRAD.  With MXFP4_PRECISION_MXFP4 it is
- *   mxfp4_linear_fprop / _dgrad / _wgrad; with MXFP4_PRECISION_MXFP8 hadamard_mode, rounding and
+ *   mxfp4_linear_fprop / _dgrad / _wgrad; MXFP4_PRECISION_MXFP4_32X32 is the same pass with both
+ *   operands quantized by mxfp4_quantize_2d; with MXFP4_PRECISION_MXFP8 hadamard_mode, rounding and
  *   seed are ignored.  Workspace: mxfp4_linear_pass_workspace_bytes (0 for a bad argument).
  * Errors as for the 4-bit entry points.
  */

@@ -19,7 +19,7 @@ SCALES_CANONICAL, SCALES_TILED = 0, 1
 BLOCK_1X32, BLOCK_32X32 = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
 LAYER_SAVED, LAYER_FORWARD, LAYER_BACKWARD = 0, 1, 2
-PRECISION_MXFP4, PRECISION_MXFP8 = 0, 1
+PRECISION_MXFP4, PRECISION_MXFP8, PRECISION_MXFP4_32X32 = 0, 1, 2
 PASS_FPROP, PASS_DGRAD, PASS_WGRAD = 0, 1, 2
 AXIS_ROWS, AXIS_COLS = 0, 1
 

@@ -449,7 +449,7 @@ size_t mxfp4_linear_workspace_bytes(int64_t T, int64_t in_features, int64_t out_
 static size_t pass_workspace_bytes(int64_t T, int64_t in_features, int64_t out_features, int pass, int precision)
 {
     if (pass < 0 || pass > 2 || T <= 0 || in_features <= 0 || out_features <= 0) return 0;
-    if (precision != MXFP4_PRECISION_MXFP4 && precision != MXFP4_PRECISION_MXFP8) return 0;
+    if (precision < MXFP4_PRECISION_MXFP4 || precision > MXFP4_PRECISION_MXFP4_32X32) return 0;
     int64_t M, N, K;
     linear_dims(pass, T, in_features, out_features, &M, &N, &K);
     if (K % 32 != 0) return 0;
@@ -464,6 +464,7 @@ static int linear_pass(int pass, const void* a_src, const void* b_src, void* out
                        int precision = MXFP4_PRECISION_MXFP4)
 {
     const bool fp8 = precision == MXFP4_PRECISION_MXFP8;
+    const int b2d = precision == MXFP4_PRECISION_MXFP4_32X32 ? 1 : 0;    // Appendix D's 32 x 32 blocks
     const size_t cmul = fp8 ? 2 : 1;
     if (!a_src || !b_src || !out) return MXFP4_ERR_NULL;
     if (T <= 0 || in_f <= 0 || out_f <= 0) return MXFP4_ERR_SHAPE;
@@ -494,10 +495,10 @@ static int linear_pass(int pass, const void* a_src, const void* b_src, void* out
     QuantJob ja, jb;
     if (fp8) hmode = MXFP4_HADAMARD_NONE, rounding = MXFP4_ROUND_RNE;    // the stabilisers belong to the 4-bit GEMMs
     int rc = build_quant_job(a_src, ar, ac, ac, a_axis, hmode, rounding, seed, 0u, a_codes, a_scales,
-                             MXFP4_SCALES_TILED, &ja, 0, fp8);
+                             MXFP4_SCALES_TILED, &ja, b2d, fp8);
     if (rc != MXFP4_OK) return rc;
     rc = build_quant_job(b_src, br, bc, bc, b_axis, hmode, rounding, seed, 1u, b_codes, b_scales,
-                         MXFP4_SCALES_TILED, &jb, 0, fp8);
+                         MXFP4_SCALES_TILED, &jb, b2d, fp8);
     if (rc != MXFP4_OK) return rc;
     rc = fp8 ? launch_quant_jobs_fp8(ja, jb, a_axis, b_axis, static_cast<cudaStream_t>(stream))
              : launch_quant_jobs(ja, jb, a_axis, b_axis, hmode, rounding, static_cast<cudaStream_t>(stream));
@@ -544,7 +545,7 @@ int mxfp4_linear_pass(int pass, int precision, const void* a, const void* b, voi
                       int out_dtype, void* workspace, size_t workspace_bytes, void* stream)
 {
     if (pass < 0 || pass > 2) return MXFP4_ERR_ENUM;
-    if (precision != MXFP4_PRECISION_MXFP4 && precision != MXFP4_PRECISION_MXFP8) return MXFP4_ERR_ENUM;
+    if (precision < MXFP4_PRECISION_MXFP4 || precision > MXFP4_PRECISION_MXFP4_32X32) return MXFP4_ERR_ENUM;
     return linear_pass(pass, a, b, out, T, in_features, out_features, hadamard_mode, rounding, seed, out_dtype,
                        workspace, workspace_bytes, stream, precision);
 }

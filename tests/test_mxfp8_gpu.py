@@ -103,7 +103,7 @@ def test_linear_pass_at_4_bits_is_the_per_pass_entry_point():
     a = api.linear_pass(api.PASS_FPROP, api.PRECISION_MXFP4, X, W, 1, 0, 3)
     assert torch.equal(a, api.linear_fprop(X, W, 1, 0, 3))
     with pytest.raises(api.Mxfp4Error) as exc:
-        api.linear_pass(api.PASS_FPROP, 2, X, W)
+        api.linear_pass(api.PASS_FPROP, 3, X, W)
     assert exc.value.status == -4
 
 

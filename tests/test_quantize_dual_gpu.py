@@ -164,3 +164,25 @@ def test_dual_is_reproducible_run_to_run():
     import torch
     for (x0, x1), (y0, y1) in zip(a, b):
         assert torch.equal(x0, y0) and torch.equal(x1, y1)
+
+
+@pytest.mark.parametrize("pass_", [0, 1, 2])
+def test_passes_with_32x32_blocks(pass_):
+    """mxfp4_linear_pass with 32 x 32 blocks: bit-identical to quantize_2d + gemm, and within
+    tolerance of the oracle's 2D quantization followed by its fp64 GEMM."""
+    import torch
+    from gpu_util import assert_gemm_close
+    rng = np.random.default_rng(60 + pass_)
+    T, in_f, out_f = 416, 288, 672
+    X, W, dY = _mixed_bits(rng, T, in_f), _mixed_bits(rng, out_f, in_f), _mixed_bits(rng, T, out_f)
+    a, b = ((X, W), (dY, W), (dY, X))[pass_]
+    axes = ((1, 1), (1, 0), (0, 0))[pass_]
+    out = api.linear_pass(pass_, api.PRECISION_MXFP4_32X32, to_dev(a), to_dev(b), 1, 0, 3, api.OUT_FP32)
+    qa = api.quantize(to_dev(a), axes[0], 1, 0, 3, 0, block_shape=api.BLOCK_32X32)
+    qb = api.quantize(to_dev(b), axes[1], 1, 0, 3, 1, block_shape=api.BLOCK_32X32)
+    assert torch.equal(out, api.gemm(*qa, *qb, 1.0 / 32, api.OUT_FP32))
+    api.check()
+    oa = oracle.quantize(a, axes[0], 1, 0, 3, 0, block2d=True)
+    ob = oracle.quantize(b, axes[1], 1, 0, 3, 1, block2d=True)
+    ref, S = oracle.gemm(*oa, *ob, alpha=1.0 / 32)
+    assert_gemm_close(out.cpu().numpy(), ref, S, False, f"32x32 pass {pass_}")
