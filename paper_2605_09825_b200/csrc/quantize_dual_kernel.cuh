@@ -6,9 +6,10 @@
 // of 2 bytes per element by one: 3.06 instead of 5.06 bytes of traffic per element.
 //
 // Same skeleton as the single-axis kernel: persistent CTAs, a TMA producer warp filling a ring
-// of 128 x 128 source tiles (two 128-row x 64-column boxes in the 128-byte swizzle), two
-// consumer groups of 256 threads on alternate tiles.  Per tile a thread first handles two
-// row-wise blocks (its source row, block columns kbh and kbh + 2), then two column-wise blocks:
+// of 128 x 128 source tiles (two 128-row x 64-column boxes in the 128-byte swizzle), consumer
+// groups on alternate tiles (two of 256 threads or four of 128, see QuantDualShape).  Per tile
+// and sub-pass a thread first handles two row-wise blocks (its source row, block columns kbh and
+// kbh + 2), then two column-wise blocks:
 // it reads 32 rows of one 4-byte word, i.e. of two adjacent source columns, which gives it the
 // same block of two neighbouring operand rows of the transposed operand.  Each orientation has
 // its own staged code / scale tile and its own TMA store.

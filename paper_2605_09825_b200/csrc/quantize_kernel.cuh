@@ -3,11 +3,11 @@
 //
 // Work unit: a tile of 128 operand rows x 128 elements along K (4 MX blocks).  A producer warp
 // streams source tiles into a ring of shared-memory stages with TMA.  The 512 consumer threads
-// form two groups of 256 that take alternate tiles; a thread handles two 32-element blocks of
-// its group's tile, one after the other, each entirely in registers, so the five butterfly
-// stages (as packed fp32x2 operations), the block maximum and the rounding need no cross-lane
-// traffic.  The two groups synchronise only among themselves, so they sit in different phases
-// (one in its integer/convert instructions while the other is in its floating-point ones)
+// form groups (four of 128 threads, see QuantShape) that take alternate tiles; a thread handles
+// 32-element blocks of its group's tile two at a time, each entirely in registers, so the five
+// butterfly stages (as packed fp32x2 operations), the block maximum and the rounding need no
+// cross-lane traffic.  The groups synchronise only among themselves, so they sit in different
+// phases (one in its integer/convert instructions while another is in its floating-point ones)
 // instead of all sixteen warps queueing on the same pipe at the same time.
 // Results leave through shared memory: packed codes as a 128 x 64-byte tile written by a TMA
 // store (which also clips ragged edges), scales as one contiguous 512-byte tile.
