@@ -138,3 +138,16 @@ def test_eight_times_the_benchmark_token_count():
     rows = _rows(out_f, 98, n_random=4)
     ref, S = oracle.linear_wgrad(dYb, Xb, 1, 0, 0, rows=rows)
     assert_gemm_close(dW[torch.from_numpy(rows).cuda()].cpu().numpy(), ref, S, False, "wgrad over 131072 tokens")
+
+
+@pytest.mark.parametrize("hmode,rnd", [(1, 0), (2, 0), (0, 1)])
+def test_config4_dual_quantize_variants(hmode, rnd):
+    """Config 4's X [8192 x 14336] (post-SwiGLU-like) through the dual-axis kernel for the three
+    variants of that configuration, whole tensor, both orientations, bit-exact."""
+    t = synth.config4()
+    (cr, sr), (cc, sc) = api.quantize_dual(to_dev(t["X"]), hmode, rnd, 7, tags=(0, 1))
+    api.check()
+    for codes, scales, axis, tag in ((cr, sr, 1, 0), (cc, sc, 0, 1)):
+        wc, ws = oracle.quantize(t["X"], axis, hmode, rnd, 7, tag)
+        assert (codes.cpu().numpy() == wc).all()
+        assert (oracle.scales_from_tiled(scales.cpu().numpy(), wc.shape[0], wc.shape[1] * 2 // 32) == ws).all()
