@@ -514,17 +514,28 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     const int64_t total = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
     if (total > 0x3FFFFFFF) return MXFP4_ERR_SHAPE;
     const size_t smem = sizeof(GemmPairSmem) + 1024;
-    static bool attr_set[64] = {};          // the attribute is per device
+    static int resident_clusters[64] = {};  // per device: CTA pairs that can be resident at once (0 = not asked yet)
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
-    if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(KIND == 0 ? gemm_mxf4_pair_kernel : gemm_mxf8_pair_kernel,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(smem)) != cudaSuccess)
+    if (resident_clusters[dev] == 0) {
+        auto kernel = KIND == 0 ? gemm_mxf4_pair_kernel : gemm_mxf8_pair_kernel;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
+            cudaSuccess)
             return MXFP4_ERR_CUDA;
-        attr_set[dev] = true;
+        // the persistent grid must not exceed what the device can hold at once (a partitioned or
+        // shared device may offer fewer pairs than SMs / 2); fall back to SMs / 2 if the query fails
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(sm_count & ~1), 1, 1);
+        cfg.blockDim = dim3(kPThreads, 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            n = sm_count / 2;
+        }
+        resident_clusters[dev] = n < sm_count / 2 ? n : sm_count / 2;
     }
-    const int max_clusters = sm_count / 2;
+    const int max_clusters = resident_clusters[dev];
     const int clusters = static_cast<int>(total < max_clusters ? total : max_clusters);
     return launch_kernel_pdl(KIND == 0 ? gemm_mxf4_pair_kernel : gemm_mxf8_pair_kernel, 2 * clusters, kPThreads, smem,
                              stream, tm_a, tm_b, tm_out, p) == cudaSuccess
