@@ -159,6 +159,63 @@ def aggregate_over_ranks(elapsed_ms: float, world: int) -> float:
     return float(t.item())
 
 
+def sweep_quantize_variants(dev_in, peaks, api, reps: int = 10):
+    """GB/s of every quantizer variant -- {no rotation, deterministic H32, randomized H32} x {RNE,
+    stochastic rounding} x {row-wise, column-wise, dual-axis} -- on the activations of config 2
+    (X 8192 x 4096), the gradient of config 3 (dY 8192 x 28672) and the activations of config 4
+    (X 8192 x 14336): the first 8192 tokens of this step's tensors, which follow those recipes.
+    Single launches, CUDA events, a 256 MB buffer rewritten before each so that nothing comes from
+    L2; median of `reps` after 3 warm-ups.  Algorithmic bytes: 2.53125 per element single-axis,
+    3.0625 dual-axis."""
+    import torch
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    tensors = {"config 2 X 8192x4096": dev_in["qkv"]["X"][:8192],
+               "config 3 dY 8192x28672": dev_in["gate_up"]["dY"][:8192],
+               "config 4 X 8192x14336": dev_in["down"]["X"][:8192]}
+    hbm = peaks["hbm_gbs"]
+    out = {"unit": "GB/s of algorithmic bytes", "peak": hbm, "peak_source": peaks["source"] + " copy bandwidth",
+           "timing": f"single launches, L2 rewritten before each, median of {reps}", "cases": {}}
+
+    def timed(fn):
+        ts = []
+        for r in range(3 + reps):
+            flush.fill_(r & 0xFF)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            if r >= 3:
+                ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts)
+
+    for tname, x in tensors.items():
+        rows, cols = x.shape
+        n = rows * cols
+        buf = {1: (torch.empty((rows, cols // 2), dtype=torch.uint8, device="cuda"),
+                   torch.empty(api.scales_bytes(rows, cols), dtype=torch.uint8, device="cuda")),
+               0: (torch.empty((cols, rows // 2), dtype=torch.uint8, device="cuda"),
+                   torch.empty(api.scales_bytes(cols, rows), dtype=torch.uint8, device="cuda"))}
+        table = {}
+        for hname, hmode in (("none", api.HADAMARD_NONE), ("h32", api.HADAMARD_DET), ("rh32", api.HADAMARD_RAND)):
+            for rname, rnd in (("rne", api.ROUND_RNE), ("sr", api.ROUND_SR)):
+                for axis, aname in ((1, "row"), (0, "col")):
+                    c, sc = buf[axis]
+                    ms = timed(lambda: api.quantize(x, axis, hmode, rnd, 7, 0, codes=c, scales=sc))
+                    gbs = n * 2.53125 / (ms * 1e-3) / 1e9
+                    table[f"{aname} {hname} {rname}"] = {"us": round(ms * 1e3, 1), "gbs": round(gbs, 1),
+                                                         "frac": round(gbs / hbm, 3)}
+                ms = timed(lambda: api.quantize_dual(x, hmode, rnd, 7, out_row=buf[1], out_col=buf[0]))
+                gbs = n * 3.0625 / (ms * 1e-3) / 1e9
+                table[f"dual {hname} {rname}"] = {"us": round(ms * 1e3, 1), "gbs": round(gbs, 1),
+                                                  "frac": round(gbs / hbm, 3)}
+        out["cases"][tname] = table
+        del buf
+    del flush
+    api.check()
+    return out
+
+
 # --------------------------------------------------------------------------- oracle arm
 def oracle_sample(steps: int, warmup: int):
     """Time the CPU oracle on a bounded sample: the QKV Fprop restricted to 2048 tokens."""
@@ -327,8 +384,10 @@ def run_ours(args):
 
     gemm_ms = gemm_flops = quant_ms = quant_bytes = 0.0
     n_quant = 0
-    gemm_by_shape = {}      # per launch, M x N x K -> TFLOP/s inside the step (tile and wave effects show here)
+    gemm_times = {}         # per launch of the step, label -> (flops, [ms per repetition])
+    quant_times = {}        # per quantize launch of the step, index -> (bytes, [ms per repetition])
     r256 = lambda v: (v + 255) // 256 * 256
+    n_dec = max(2, args.decomposed_reps + 1)          # the first decomposed pass is a warm-up
 
     def operand_views(buf, off, outer, K):
         """(codes, scales, next offset) inside a byte buffer, as the library lays operands out."""
@@ -337,7 +396,7 @@ def run_ours(args):
         sb = api.scales_bytes(outer, K)
         return c, buf[off: off + sb], off + r256(sb)
 
-    for rep in range(2):
+    for rep in range(n_dec):
         evs = []
         fp8_evs = []
         if layer:
@@ -396,17 +455,31 @@ def run_ours(args):
         torch.cuda.synchronize()
         if rep == 0:
             continue   # first decomposed pass is a warm-up
+        qi = 0
         for qs, gs in evs:
             for a0, a1, elems in qs:
-                quant_ms += a0.elapsed_time(a1)
-                quant_bytes += elems * q_bytes_per_element
-                n_quant += 1
+                quant_times.setdefault(qi, (elems * q_bytes_per_element, []))[1].append(a0.elapsed_time(a1))
+                qi += 1
             for a0, a1, fl, label in gs:
-                gemm_ms += a0.elapsed_time(a1)
-                gemm_flops += fl
-                gemm_by_shape[label] = round(fl / (a0.elapsed_time(a1) * 1e-3) / 1e12, 1)
+                gemm_times.setdefault(label, (fl, []))[1].append(a0.elapsed_time(a1))
+    # medians over the repetitions, per launch; the step's totals are sums of those medians
+    gemm_by_shape = {}
+    for label, (fl, ts) in gemm_times.items():
+        med = statistics.median(ts)
+        gemm_ms += med
+        gemm_flops += fl
+        gemm_by_shape[label] = round(fl / (med * 1e-3) / 1e12, 1)
+    for _, (nbytes, ts) in quant_times.items():
+        quant_ms += statistics.median(ts)
+        quant_bytes += nbytes
+        n_quant += 1
     clocks = sampler.stop(t_begin, t_end)
     api.check()
+
+    # ---- every quantizer variant on the config-2/3/4 tensors (single launches, L2 rewritten before each)
+    quantize_variants = None
+    if args.workload == "layer_stack" and not args.no_variants and not ladder:
+        quantize_variants = sweep_quantize_variants(dev_in, peaks, api)
 
     # ---- the single-pass configurations (8192 tokens), fused call, L2 flushed between repetitions
     per_config = {}
@@ -452,20 +525,45 @@ def run_ours(args):
     n_gemm = max(1, len(passes) - len(fp8_evs))
     if gemm_ms == 0.0:                      # all passes in 8 bits: nothing for the MXFP4 roofline
         gemm_ms, gemm_flops, quant_ms, quant_bytes, n_quant = 1.0, 0.0, 1.0, 0.0, 1
-    fp4_peak = 4.0 * peaks["bf16_tflops_sustained"]
+    # Peak for the contraction: the measured cuBLAS bf16 rate x the nominal FP4 : bf16 ratio (9 : 2.25).
+    # The timed region lasts a fraction of a second, so the BURST figure is the one that applies;
+    # the sustained figure (seconds under the power cap) and the nominal 9 PFLOP/s are given beside it.
+    fp4_peak = 4.0 * peaks["bf16_tflops"]
+    fp4_peak_sustained = 4.0 * peaks["bf16_tflops_sustained"]
     gemm_tflops = gemm_flops / (gemm_ms * 1e-3) / 1e12
+    sm_mhz = clocks.get("sm_mhz") or 0.0
+    sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    # tensor-pipe issue ceiling at the clock sampled during the timed region: a 256 x 192 x 64 pair
+    # MMA takes 96 cycles on two SMs = 32768 flop per clock per SM
+    pipe_peak = 32768.0 * sm_count * sm_mhz * 1e6 / 1e12 if sm_mhz else None
+    step_tflops = flops_per_step / (elapsed_ms / args.steps * 1e-3) / 1e12
     roofline = {
         "kernel": "gemm_mxf4_pair_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak,
-        "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak, "traffic": None,
-        "traffic_captured": {"dram_bytes": 81.3e6, "algorithmic_bytes": 130.1e6,
-                             "launch": "8192x6144x4096 (QKV Fprop at 8192 tokens), ncu, profiles/",
-                             "note": "DRAM traffic does not scale with flops (operands are re-read from "
-                                     "L2, the output is partly still in L2 at kernel end), so no "
-                                     "per-launch figure is extrapolated for the 12 shapes of this step"},
-        "peak_source": f"4 x sustained cuBLAS bf16 ({peaks['source']}); burst would be "
-                       f"{4.0 * peaks['bf16_tflops']:.0f}, nominal dense FP4 9000",
+        "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak,
+        "peak_source": f"4 x burst cuBLAS bf16 ({peaks['source']}: {peaks['bf16_tflops']:.1f}); the timed region is "
+                       f"{elapsed_ms * 1e-3:.2f} s, so the burst figure applies",
+        "frac_of_4x_sustained_bf16": gemm_tflops / fp4_peak_sustained, "peak_4x_sustained_bf16": fp4_peak_sustained,
+        "frac_of_nominal_fp4": gemm_tflops / 9000.0, "peak_nominal_fp4": 9000.0,
+        "frac_of_tensor_pipe_at_sampled_clock": (gemm_tflops / pipe_peak) if pipe_peak else None,
+        "tensor_pipe_peak_at_sampled_clock": pipe_peak, "sampled_sm_mhz": sm_mhz or None,
+        # ncu, one launch of the 8192 x 6144 x 4096 GEMM (QKV Fprop at 8192 tokens; profiles/): DRAM
+        # bytes of THAT launch, not scaled to this step's shapes (operands are re-read from L2 and
+        # part of the output is still in L2 at kernel end, so traffic does not follow the flops)
+        "traffic": 81.3e6,
+        "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one captured 8192x6144x4096 launch "
+                        "(algorithmic bytes of that launch 130.1e6); not scaled to the 12 shapes of this step",
         "flops_per_launch": gemm_flops / n_gemm, "avg_launch_ms": gemm_ms / n_gemm,
+        "launch_timing": f"median of {n_dec - 1} repetitions per launch, CUDA events on the launching stream",
         "tflops_by_launch": gemm_by_shape,
+        "fused_path": {"tflops": step_tflops, "frac_of_nominal_fp4": step_tflops / 9000.0,
+                       "frac_of_4x_burst_bf16": step_tflops / fp4_peak,
+                       "frac_of_4x_sustained_bf16": step_tflops / fp4_peak_sustained,
+                       "note": "the whole step (quantize + GEMM launches) against the same peaks; target 0.60 of nominal"},
+        "decomposed": {"gemm_ms": gemm_ms, "quantize_ms": quant_ms, "sum_ms": gemm_ms + quant_ms,
+                       "ms_per_step": elapsed_ms / args.steps,
+                       "note": "sum of per-launch medians with an event between launches; the events keep a "
+                               "launch's set-up from overlapping the previous launch's tail (programmatic "
+                               "dependent launch), so the sum exceeds the step time by a few per cent"},
     }
     quant_gbs = quant_bytes / (quant_ms * 1e-3) / 1e9
     # ncu, single-axis kernel on a 117.4 M-element tensor: 234.9 MB read + 45.4 MB written = 2.39 B
@@ -612,7 +710,8 @@ def run_ours(args):
                    "input_crc32": checksums,
                    "l2": "inputs larger than L2 (several GB per step), no flush needed",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
-        "roofline": roofline, "quantize": quantize_info, "mxfp8_passes": fp8_info,
+        "roofline": roofline, "quantize": quantize_info, "quantize_variants": quantize_variants,
+        "mxfp8_passes": fp8_info,
         "frac_of_nominal_fp4_peak": world and (flops_per_step / (ms_per_step * 1e-3) / 1e12) / 9000.0,
         "cpu_baseline": cpu_base, "e2e": e2e, "gpu_launches": 2 * len(passes) * args.steps,   # per linear: 3 quantize + 3 GEMM (layer) or 3 x (1 + 1)
         "clocks": clocks, "context": context, "per_config": per_config,
@@ -639,6 +738,9 @@ def main():
     ap.add_argument("--no-context", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true")
+    ap.add_argument("--no-variants", action="store_true", help="skip the per-variant quantize table")
+    ap.add_argument("--decomposed-reps", type=int, default=20,
+                    help="repetitions of the per-launch timed step (medians feed the roofline)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

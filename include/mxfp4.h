@@ -24,10 +24,11 @@
  *     previous kernel in the stream, and every kernel waits for that kernel's completion before
  *     it touches global memory, so stream order is what a caller observes.  MXFP4_PDL=0 in the
  *     environment (read once) selects plain launches.
- *   - Host threads: per-device state (function attributes, the copy streams and events of the
- *     host-buffer layer call, the static scratch address) is created on first use without a
- *     lock; make the first call on a device from one thread, and do not run two host-buffer
- *     layer calls on the same device at the same time.
+ *   - Host threads: per-device state (function attributes, the resident-grid size, the copy
+ *     streams and events of the host-buffer layer call, the static scratch address) is created
+ *     on first use, once per device, and that set-up is safe against several host threads
+ *     making their first call at the same time.  The host-buffer layer calls of one device
+ *     share one set of copy streams and events: do not run two of them at the same time.
  */
 #ifndef MXFP4_H_
 #define MXFP4_H_
@@ -108,14 +109,16 @@ size_t mxfp4_scales_bytes(int64_t outer, int64_t K, int scale_layout);
  *                MXFP4_AXIS_ROWS: operand[o][k] = src[k][o], outer = cols, K = rows -- the
  *                transposed operand Dgrad (W^T) and Wgrad (dY^T, X^T) need, written directly
  *                with no separate transpose pass.
- *   K must be a multiple of 32.  For MXFP4_AXIS_ROWS, cols must be a multiple of 8.
+ *   K must be a multiple of 32; outer may be any positive number (cols need not be a multiple
+ *                of 8 for MXFP4_AXIS_ROWS: only ld_src has that rule).
  *   hadamard_mode, rounding, seed: each 32-block v becomes H*v (mode 1) or H*(D*v) (mode 2,
  *                D the +-1 diagonal drawn from `seed`) in fp32 with a fixed five-stage
  *                butterfly; modes 3 / 4 rotate each half of the block with its own 16-point
  *                transform instead (the same butterfly without its last stage); the block scale is 2^(floor(log2 amax) - 2); elements are rounded
  *                to E2M1 with saturation at 6.  With MXFP4_ROUND_SR each element uses 8 bits
- *                of Philox4x32-10(key = seed, counter = (e>>4, 0, operand_tag, 0)), e the
- *                element's index o*K + k in the operand view.
+ *                of Philox4x32-10(key = (lo32(seed), hi32(seed)), counter = (lo32(g), hi32(g),
+ *                operand_tag, 0)) with g = e >> 4 and e the element's 64-bit index o*K + k in
+ *                the operand view: byte (e & 3) of output word ((e & 15) >> 2).
  *   operand_tag  decorrelates the stochastic-rounding streams of different operands.
  *   codes        out, [outer x K/2] bytes, 16-byte aligned.
  *   scales       out, mxfp4_scales_bytes(outer, K, scale_layout) bytes, 16-byte aligned.

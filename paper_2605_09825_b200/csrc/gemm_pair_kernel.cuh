@@ -40,6 +40,8 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "../../include/mxfp4.h"
 #include "ptx_sm100.cuh"
 #include "tma_host.cuh"
@@ -514,14 +516,17 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     const int64_t total = static_cast<int64_t>(p.tiles_m) * p.tiles_n;
     if (total > 0x3FFFFFFF) return MXFP4_ERR_SHAPE;
     const size_t smem = sizeof(GemmPairSmem) + 1024;
-    static int resident_clusters[64] = {};  // per device: CTA pairs that can be resident at once (0 = not asked yet)
+    // per device, set up once however many host threads arrive together: the shared-memory
+    // attribute and the number of CTA pairs that can be resident at once
+    static int resident_clusters[64] = {};
+    static std::once_flag once[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
-    if (resident_clusters[dev] == 0) {
+    std::call_once(once[dev], [&] {
         auto kernel = KIND == 0 ? gemm_mxf4_pair_kernel : gemm_mxf8_pair_kernel;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
             cudaSuccess)
-            return MXFP4_ERR_CUDA;
+            return;                                     // resident_clusters stays 0: reported below
         // the persistent grid must not exceed what the device can hold at once (a partitioned or
         // shared device may offer fewer pairs than SMs / 2); fall back to SMs / 2 if the query fails
         cudaLaunchConfig_t cfg = {};
@@ -534,7 +539,8 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
             n = sm_count / 2;
         }
         resident_clusters[dev] = n < sm_count / 2 ? n : sm_count / 2;
-    }
+    });
+    if (resident_clusters[dev] <= 0) return MXFP4_ERR_CUDA;
     const int max_clusters = resident_clusters[dev];
     const int clusters = static_cast<int>(total < max_clusters ? total : max_clusters);
     return launch_kernel_pdl(KIND == 0 ? gemm_mxf4_pair_kernel : gemm_mxf8_pair_kernel, 2 * clusters, kPThreads, smem,

@@ -6,6 +6,8 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "../../include/mxfp4.h"
 #include "ptx_sm100.cuh"
 #include "tma_host.cuh"
@@ -18,29 +20,67 @@ namespace mxfp4 {
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+constexpr int kMaxDevices = 64;      // size of the per-device tables below
+
 struct DeviceInfo {
     int sm_count = 0;
     int cc_major = 0;
     bool ok = false;
 };
 
+// Per-device set-up that runs once however many host threads reach it at the same time: the
+// first caller on a device runs `f` (which returns a status code), the others wait for it, and
+// everybody gets that status.  One instance per table (device properties, a kernel's
+// shared-memory attribute, the copy streams of the host-buffer call, ...).
+struct PerDeviceOnce {
+    std::once_flag flag[kMaxDevices];
+    int status[kMaxDevices] = {};
+    template <class F>
+    int run(int dev, F&& f)
+    {
+        std::call_once(flag[dev], [&] { status[dev] = f(); });
+        return status[dev];
+    }
+};
+
+// Ordinal of the current device, or -1 if it cannot be had or lies beyond the tables.
+static int current_device()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+
 static const DeviceInfo& device_info()
 {
-    static DeviceInfo info[64];
-    static bool init[64] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64) dev = 0;
-    if (!init[dev]) {
+    static DeviceInfo info[kMaxDevices];
+    static PerDeviceOnce once;
+    static const DeviceInfo none;
+    const int dev = current_device();
+    if (dev < 0) return none;
+    once.run(dev, [&] {
         cudaDeviceProp prop;
         if (cudaGetDeviceProperties(&prop, dev) == cudaSuccess) {
             info[dev].sm_count = prop.multiProcessorCount;
             info[dev].cc_major = prop.major;
             info[dev].ok = true;
         }
-        init[dev] = true;
-    }
+        return 0;
+    });
     return info[dev];
+}
+
+// Raises a kernel's dynamic shared-memory limit on the current device, once per device.
+template <class Kernel>
+static int ensure_smem_attribute(PerDeviceOnce& once, Kernel kernel, size_t smem)
+{
+    const int dev = current_device();
+    if (dev < 0) return MXFP4_ERR_CUDA;
+    return once.run(dev, [&] {
+        return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) ==
+                       cudaSuccess
+                   ? MXFP4_OK : MXFP4_ERR_CUDA;
+    });
 }
 
 // Host copy of the counter-based generator, used only for the 32-bit sign mask of the
@@ -63,16 +103,9 @@ template <int AXIS0, int AXIS1, int HMODE, int SR>
 static int launch_quantize(const QuantJob& j0, const QuantJob& j1, int grid, cudaStream_t stream)
 {
     const size_t smem = sizeof(QuantSmem) + 1024;
-    static bool attr_set[64] = {};          // the attribute is per device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
-    if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(quantize_kernel<AXIS0, AXIS1, HMODE, SR>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(smem)) != cudaSuccess)
-            return MXFP4_ERR_CUDA;
-        attr_set[dev] = true;
-    }
+    static PerDeviceOnce once;               // the attribute is per device
+    const int rc = ensure_smem_attribute(once, quantize_kernel<AXIS0, AXIS1, HMODE, SR>, smem);
+    if (rc != MXFP4_OK) return rc;
     QuantJobs jobs;
     jobs.j[0] = j0;
     jobs.j[1] = j1;
@@ -183,15 +216,9 @@ template <int AXIS0, int AXIS1>
 static int launch_quantize_fp8(const QuantJob& j0, const QuantJob& j1, int grid, cudaStream_t stream)
 {
     const size_t smem = sizeof(QuantFp8Smem) + 1024;
-    static bool attr_set[64] = {};          // the attribute is per device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
-    if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(quantize_fp8_kernel<AXIS0, AXIS1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(smem)) != cudaSuccess)
-            return MXFP4_ERR_CUDA;
-        attr_set[dev] = true;
-    }
+    static PerDeviceOnce once;               // the attribute is per device
+    const int rc = ensure_smem_attribute(once, quantize_fp8_kernel<AXIS0, AXIS1>, smem);
+    if (rc != MXFP4_OK) return rc;
     QuantJobs jobs;
     jobs.j[0] = j0;
     jobs.j[1] = j1;
@@ -215,15 +242,9 @@ template <int HMODE, int SR>
 static int launch_quantize_dual(const QuantDualJob& job, int grid, cudaStream_t stream)
 {
     const size_t smem = sizeof(QuantDualSmem) + 1024;
-    static bool attr_set[64] = {};          // the attribute is per device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
-    if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(quantize_dual_kernel<HMODE, SR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(smem)) != cudaSuccess)
-            return MXFP4_ERR_CUDA;
-        attr_set[dev] = true;
-    }
+    static PerDeviceOnce once;               // the attribute is per device
+    const int rc = ensure_smem_attribute(once, quantize_dual_kernel<HMODE, SR>, smem);
+    if (rc != MXFP4_OK) return rc;
     return launch_kernel_pdl(quantize_dual_kernel<HMODE, SR>, grid, kQThreads, smem, stream, job) == cudaSuccess
                ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
@@ -273,7 +294,7 @@ static int gemm_checked(const void* a_codes, const void* a_scales, const void* b
 
 extern "C" {
 
-int mxfp4_version(void) { return 103; }   // 1.3: + pair/dual/2D quantize, layer-level calls, 8-bit passes
+int mxfp4_version(void) { return 104; }   // 1.4: thread-safe first calls, argument checks before any enqueue
 
 const char* mxfp4_status_string(int status)
 {
@@ -461,7 +482,7 @@ static size_t pass_workspace_bytes(int64_t T, int64_t in_features, int64_t out_f
 static int linear_pass(int pass, const void* a_src, const void* b_src, void* out, int64_t T,
                        int64_t in_f, int64_t out_f, int hmode, int rounding, uint64_t seed,
                        int out_dtype, void* workspace, size_t workspace_bytes, void* stream,
-                       int precision = MXFP4_PRECISION_MXFP4)
+                       int precision = MXFP4_PRECISION_MXFP4, bool validate_only = false)
 {
     const bool fp8 = precision == MXFP4_PRECISION_MXFP8;
     const int b2d = precision == MXFP4_PRECISION_MXFP4_32X32 ? 1 : 0;    // Appendix D's 32 x 32 blocks
@@ -472,9 +493,14 @@ static int linear_pass(int pass, const void* a_src, const void* b_src, void* out
     int64_t M, N, K;
     linear_dims(pass, T, in_f, out_f, &M, &N, &K);
     if (K % 32 != 0 || in_f % 8 != 0 || out_f % 8 != 0) return MXFP4_ERR_SHAPE;
+    // everything the GEMM would reject is checked here, before the quantize launch
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
+    if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
     const size_t need = pass_workspace_bytes(T, in_f, out_f, pass, precision);
     if (!workspace || workspace_bytes < need) return MXFP4_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MXFP4_ERR_ALIGN;
+    if (!aligned16(a_src) || !aligned16(b_src) || !aligned16(out)) return MXFP4_ERR_ALIGN;
+    if (validate_only) return MXFP4_OK;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     uint8_t* a_codes = ws;
     uint8_t* a_scales = a_codes + round_up(cmul * mxfp4_codes_bytes(M, K), 256);
@@ -595,6 +621,8 @@ int mxfp4_linear_forward(const void* X, const void* W, void* Y, int64_t T, int64
                          void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream)
 {
     if (!X || !W || !Y) return MXFP4_ERR_NULL;
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
+    if (!aligned16(X) || !aligned16(W) || !aligned16(Y)) return MXFP4_ERR_ALIGN;
     int rc = layer_args_ok(T, in_features, out_features, hadamard_mode, rounding, saved, saved_bytes, workspace,
                            workspace_bytes, MXFP4_LAYER_FORWARD);
     if (rc != MXFP4_OK) return rc;
@@ -626,6 +654,9 @@ static int linear_backward_impl(const void* dY, void* dX, void* dW, int64_t T, i
                                 size_t workspace_bytes, void* stream, cudaEvent_t after_dx)
 {
     if (!dY || !dX || !dW) return MXFP4_ERR_NULL;
+    for (int d : {dx_dtype, dw_dtype})
+        if (d != MXFP4_OUT_BF16 && d != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
+    if (!aligned16(dY) || !aligned16(dX) || !aligned16(dW)) return MXFP4_ERR_ALIGN;
     int rc = layer_args_ok(T, in_features, out_features, hadamard_mode, rounding, saved, saved_bytes, workspace,
                            workspace_bytes, MXFP4_LAYER_BACKWARD);
     if (rc != MXFP4_OK) return rc;
@@ -672,11 +703,13 @@ struct HostPipe {
 
 static int host_pipe(HostPipe** out)
 {
-    static HostPipe pipes[64] = {};
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
+    static HostPipe pipes[kMaxDevices] = {};
+    static PerDeviceOnce once;
+    const int dev = current_device();
+    if (dev < 0) return MXFP4_ERR_CUDA;
     HostPipe& p = pipes[dev];
-    if (!p.ready) {
+    *out = &p;
+    return once.run(dev, [&] {
         if (cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking) != cudaSuccess ||
             cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking) != cudaSuccess)
             return MXFP4_ERR_CUDA;
@@ -684,9 +717,8 @@ static int host_pipe(HostPipe** out)
         for (cudaEvent_t* e : evs)
             if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return MXFP4_ERR_CUDA;
         p.ready = true;
-    }
-    *out = &p;
-    return MXFP4_OK;
+        return MXFP4_OK;
+    });
 }
 
 int mxfp4_linear_layer_host_drain(void* stream);
@@ -707,6 +739,10 @@ int mxfp4_linear_layer_host(const void* X_host, const void* W_host, const void* 
     if (rc != MXFP4_OK) return rc;
     if (workspace_bytes < mxfp4_linear_layer_bytes(T, in_features, out_features, MXFP4_LAYER_BACKWARD))
         return MXFP4_ERR_WORKSPACE;
+    for (const void* q : {static_cast<const void*>(dev_x), static_cast<const void*>(dev_w),
+                          static_cast<const void*>(dev_dy), static_cast<const void*>(dev_y),
+                          static_cast<const void*>(dev_dx), static_cast<const void*>(dev_dw)})
+        if (!aligned16(q)) return MXFP4_ERR_ALIGN;      // before the first copy is enqueued
     HostPipe* hp = nullptr;
     rc = host_pipe(&hp);
     if (rc != MXFP4_OK) return rc;
@@ -780,6 +816,10 @@ int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* ou
     int64_t M, N, K;
     linear_dims(pass, T, in_features, out_features, &M, &N, &K);
     const size_t out_bytes = static_cast<size_t>(M) * N * (out_dtype == MXFP4_OUT_BF16 ? 2 : 4);
+    // argument errors are reported before the first copy is enqueued
+    const int vrc = linear_pass(pass, dev_a, dev_b, dev_out, T, in_features, out_features, hadamard_mode, rounding,
+                                seed, out_dtype, workspace, workspace_bytes, stream, MXFP4_PRECISION_MXFP4, true);
+    if (vrc != MXFP4_OK) return vrc;
     if (cudaMemcpyAsync(dev_a, a_host, a_elems * 2, cudaMemcpyHostToDevice, st) != cudaSuccess ||
         cudaMemcpyAsync(dev_b, b_host, b_elems * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return MXFP4_ERR_CUDA;
@@ -801,17 +841,19 @@ static __device__ __align__(256) uint8_t g_static_scratch[MXFP4_STATIC_SCRATCH_B
 
 static int static_scratch_address(uint8_t** out)
 {
-    static uint8_t* cached[64] = {};
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MXFP4_ERR_CUDA;
-    if (!cached[dev]) {
+    static uint8_t* cached[kMaxDevices] = {};
+    static PerDeviceOnce once;
+    const int dev = current_device();
+    if (dev < 0) return MXFP4_ERR_CUDA;
+    const int rc = once.run(dev, [&] {
         uint8_t* ptr = nullptr;
         if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess || !ptr)
             return MXFP4_ERR_CUDA;
         cached[dev] = ptr;
-    }
+        return MXFP4_OK;
+    });
     *out = cached[dev];
-    return MXFP4_OK;
+    return rc;
 }
 
 int mxfp4_linear_static(int pass, const void* a, const void* b, void* out, int64_t T,

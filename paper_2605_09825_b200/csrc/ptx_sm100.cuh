@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk[.tensor]), tcgen05
-// (TMEM allocation, MMA, commit, ld, cp) and the bounded-wait discipline every kernel of this
+// (TMEM allocation, MMA, commit, ld, st) and the bounded-wait discipline every kernel of this
 // library follows: no wait spins forever; a wait that runs out records a status word and
 // makes every later wait of the CTA return at once.
 #pragma once
@@ -205,24 +205,6 @@ __device__ __forceinline__ void bulk_wait_group()
 }
 
 // ---------------------------------------------------------------- tcgen05 / TMEM
-__device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t ncols)
-{
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(smem_result)), "r"(ncols)
-                 : "memory");
-}
-
-__device__ __forceinline__ void tmem_relinquish()
-{
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
-{
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
-                 : "memory");
-}
-
 __device__ __forceinline__ void tcgen05_fence_before()
 {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -231,38 +213,6 @@ __device__ __forceinline__ void tcgen05_fence_before()
 __device__ __forceinline__ void tcgen05_fence_after()
 {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-
-// Arrive on `bar` when all tcgen05 operations issued so far by this thread have completed.
-__device__ __forceinline__ void tcgen05_commit(uint64_t* bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                 ::"r"(smem_u32(bar))
-                 : "memory");
-}
-
-// Block-scaled FP4 MMA: D[tmem] (+)= A[smem] * B[smem]^T with E8M0 scales in TMEM, two scale
-// blocks (of 32) per K = 64 instruction.
-__device__ __forceinline__ void tcgen05_mma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
-                                                 uint32_t idesc, uint32_t sfa_tmem,
-                                                 uint32_t sfb_tmem, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "setp.ne.b32 P, %6, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X "
-        "[%0], %1, %2, %3, [%4], [%5], P;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem),
-        "r"(accumulate)
-        : "memory");
-}
-
-// Copy 32 rows x 16 bytes of shared memory into 4 TMEM columns, replicated to all four
-// 32-lane quadrants (the arrangement scale factors need).
-__device__ __forceinline__ void tcgen05_cp_32x128b_warpx4(uint32_t taddr, uint64_t smem_desc)
-{
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(smem_desc)
-                 : "memory");
 }
 
 // 32 lanes x 32 consecutive 32-bit columns -> 32 registers per thread (lane = thread's row).
@@ -431,22 +381,8 @@ __device__ __forceinline__ void tcgen05_commit_pair(uint64_t* bar, uint16_t cta_
         : "memory");
 }
 
-// Pair MMA: 256 x N x 64 across the two CTAs (each holds 128 rows of A and N/2 rows of B).
-__device__ __forceinline__ void tcgen05_mma_mxf4_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
-                                                      uint32_t idesc, uint32_t sfa_tmem,
-                                                      uint32_t sfb_tmem, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "setp.ne.b32 P, %6, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X "
-        "[%0], %1, %2, %3, [%4], [%5], P;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem),
-        "r"(accumulate)
-        : "memory");
-}
-
-// Pair MMA with an A-collector hint: FILL keeps the A operand in the collector buffer for the
+// Pair MMA, 256 x N x 64 (or x 32) across the two CTAs (each holds 128 rows of A and N/2 rows of B):
+// D[tmem] (+)= A[smem] * B[smem]^T with E8M0 scales in TMEM.  A-collector hint: FILL keeps the A operand in the collector buffer for the
 // next MMA, LASTUSE consumes the kept copy (two MMAs that share A read it from shared memory once).
 // KIND 0: 4-bit operands (kind::mxf4, K = 64, two scales per row: scale_vec::2X);
 // KIND 1: 8-bit operands (kind::mxf8f6f4, K = 32, one scale per row: scale_vec::1X).

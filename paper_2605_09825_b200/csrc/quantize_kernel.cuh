@@ -307,21 +307,21 @@ __device__ __forceinline__ void issue_tile_load(const CUtensorMap* tm_src, const
 // with a single staging buffer per group.  Each scheduler then holds one warp of every group --
 // four different phases instead of the two that two groups of 256 threads give -- which keeps the
 // FMA and ALU pipes busier: 5-10 % faster for the rotations and for stochastic rounding, no
-// change for the un-rotated variant.  (The two-group form is kept below for comparison builds.)
-#ifndef MXFP4_Q_GROUP_THREADS
-#define MXFP4_Q_GROUP_THREADS 128
-#endif
+// change for the un-rotated variant.
 template <int HMODE, int SR>
 struct QuantShape {
-    static constexpr int kGroupThreads = MXFP4_Q_GROUP_THREADS;
+    static constexpr int kGroupThreads = 128;
     static constexpr int kGroups = kQConsumers / kGroupThreads;
     static constexpr int kSub = 256 / kGroupThreads;
     static constexpr int kBufs = kGroups == 2 ? 2 : 1;
 };
 
-// Four groups of 128 threads: the same work per tile in two sub-passes per thread.
+// One tile of one job, as seen by a consumer thread: wait for the stage, rotate + quantize this
+// thread's blocks (two at a time, two sub-passes), stage codes and scales, and (thread 0 of the
+// group) store them.  `p` and `tm_codes` refer to kernel parameters, so every field is a
+// constant-bank operand.  Returns false when a wait gave up (the group leaves the kernel).
 template <int AXIS, int HMODE, int SR>
-__device__ __forceinline__ bool consume_tile_narrow(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
+__device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
                                              int tile, int it, int trip, int grp, int t)
 {
     using Shape = QuantShape<HMODE, SR>;
@@ -402,92 +402,6 @@ __device__ __forceinline__ bool consume_tile_narrow(QuantSmem& sm, const QuantPa
         bulk_commit_group();
     }
     return true;
-}
-
-// One tile of one job, as seen by a consumer thread: wait for the stage, rotate + quantize this
-// thread's two blocks, stage codes and scales, and (thread 0 of the group) store them.  `p` and
-// `tm_codes` refer to kernel parameters, so every field is a constant-bank operand.  Returns
-// false when a wait gave up (the group leaves the kernel).
-// Two groups of 256 threads: a thread handles two blocks of its group's tile.
-template <int AXIS, int HMODE, int SR>
-__device__ __forceinline__ bool consume_tile_wide(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
-                                             int tile, int it, int trip, int grp, int t)
-{
-    const int kbh = t >> 7;            // this thread's blocks along K: kbh and kbh + 2
-    const int o = t & 127;             // operand row inside the tile
-    const int s = it % kQStages;
-    const uint32_t round = it / kQStages;
-    const int buf = trip & 1;
-    int to, tk;
-    tile_coords<AXIS>(p, tile, to, tk);
-
-    const bool ok = mbar_wait(&sm.full[s], round & 1, &sm.abort_flag);
-
-    float2 P0[16], P1[16];
-    if (ok) {
-        load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.signs, P0);
-        load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.signs, P1);
-    } else {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
-    }
-    // the stage is in registers now: hand it back to the producer
-    __syncwarp();
-    if ((t & 31) == 0) mbar_arrive(&sm.empty[s]);
-
-    const uint64_t e_row = static_cast<uint64_t>(to * kQTileO + o) * static_cast<uint64_t>(p.K);
-    uint32_t packed0[4], packed1[4], byte0, byte1;
-    quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tk * 4 + kbh) * 32), p, packed0, byte0);
-    quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tk * 4 + kbh + 2) * 32), p, packed1, byte1);
-
-    // stage the results: codes in the 64-byte swizzle the TMA store expects
-    uint8_t* ct = &sm.code_tile[grp * 2 + buf][o * 64];
-    *reinterpret_cast<uint4*>(ct + ((kbh ^ ((o >> 1) & 3)) * 16)) =
-        make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]);
-    *reinterpret_cast<uint4*>(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16)) =
-        make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]);
-    if (p.scale_layout == 1) {
-        uint8_t* st = &sm.scale_tile[grp * 2 + buf][(o & 31) * 16 + (o >> 5) * 4];
-        st[kbh] = static_cast<uint8_t>(byte0);
-        st[kbh + 2] = static_cast<uint8_t>(byte1);
-    } else if (ok) {
-        const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
-        const int64_t tg = static_cast<int64_t>(tk) * 4 + kbh;
-        if (og < p.outer && tg < p.nt) p.scales[og * p.nt + tg] = static_cast<uint8_t>(byte0);
-        if (og < p.outer && tg + 2 < p.nt) p.scales[og * p.nt + tg + 2] = static_cast<uint8_t>(byte1);
-    }
-    fence_proxy_async_smem();
-    // the store this group issued one trip ago must have drained its buffer before the next
-    // trip (which every thread of the group reaches only through the barrier below)
-    // overwrites it
-    if (t == 0) bulk_wait_group_read<0>();
-    uint32_t any_fail;
-    asm volatile(
-        "{\n\t.reg .pred P, Q;\n\t"
-        "setp.ne.u32 Q, %1, 0;\n\t"
-        "barrier.cta.red.or.pred P, %2, %3, Q;\n\t"
-        "selp.u32 %0, 1, 0, P;\n\t}"
-        : "=r"(any_fail)
-        : "r"(ok ? 0u : 1u), "r"(grp + 1), "n"(kQConsumers / 2)
-        : "memory");
-    if (any_fail) return false;
-    if (t == 0) {
-        tma_store_2d(tm_codes, &sm.code_tile[grp * 2 + buf][0], tk * (kQTileK / 2), to * kQTileO);
-        if (p.scale_layout == 1)
-            bulk_store_1d(p.scales + (static_cast<int64_t>(to) * p.tiles_k + tk) * kQScaleTileBytes,
-                          &sm.scale_tile[grp * 2 + buf][0], kQScaleTileBytes);
-        bulk_commit_group();
-    }
-    return true;
-}
-
-template <int AXIS, int HMODE, int SR>
-__device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
-                                             int tile, int it, int trip, int grp, int t)
-{
-    if (QuantShape<HMODE, SR>::kGroups == 2)
-        return consume_tile_wide<AXIS, HMODE, SR>(sm, p, tm_codes, tile, it, trip, grp, t);
-    return consume_tile_narrow<AXIS, HMODE, SR>(sm, p, tm_codes, tile, it, trip, grp, t);
 }
 
 template <int AXIS0, int AXIS1, int HMODE, int SR>

@@ -17,16 +17,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 inline EncodeTiledFn encode_tiled_fn()
 {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
+    // looked up once (initialisation of a function-local static is thread-safe)
+    static const EncodeTiledFn fn = [] {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) !=
                 cudaSuccess ||
             q != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
+            return static_cast<EncodeTiledFn>(nullptr);
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
     return fn;
 }
 
@@ -53,12 +53,11 @@ inline bool make_tmap_2d(CUtensorMap* map, CUtensorMapDataType dtype, uint32_t e
 // ptx_sm100.cuh).  MXFP4_PDL=0 in the environment turns the attribute off (plain stream order).
 inline bool pdl_enabled()
 {
-    static int cached = -1;
-    if (cached < 0) {
+    static const bool on = [] {
         const char* e = getenv("MXFP4_PDL");
-        cached = (e && e[0] == '0') ? 0 : 1;
-    }
-    return cached == 1;
+        return !(e && e[0] == '0');
+    }();
+    return on;
 }
 
 template <typename... KArgs, typename... Args>

@@ -37,7 +37,8 @@ def assert_gemm_close(out, ref, S, bf16: bool, what=""):
     tol = 1e-5 * S + (2.0 ** -8 * np.abs(ref) if bf16 else 0.0)
     # denormal-range outputs can differ by one fp32 ulp of the smallest normal
     tol = tol + 1e-38
-    bad = np.abs(out - ref) > tol
+    # written so that a NaN or an infinity in `out` fails (a NaN compares false either way round)
+    bad = ~(np.abs(out - ref) <= tol)
     if bad.any():
         idx = np.argwhere(bad)[:8]
         msg = [f"{what}: {bad.sum()} of {bad.size} elements out of tolerance"]

@@ -75,3 +75,27 @@ def test_argument_errors_come_back_as_status_codes(lib):
     assert f(p, p, p, 128, 128, 128, 1, 0, 0, 0, None, 0, None) == -5         # no workspace
     assert f(p, p, p, 128, 100, 128, 1, 0, 0, 0, p, 1 << 15, None) == -2      # in % 32
     assert f(None, p, p, 128, 128, 128, 1, 0, 0, 0, p, 1 << 15, None) == -1
+
+
+def test_output_errors_are_found_before_the_quantize_launch(lib):
+    """What the GEMM at the end of a fused pass would reject (output dtype, output alignment) and
+    what the second tensor of a layer call would trip over are reported by checks that run before
+    the first launch or copy: they come back even on a machine without a GPU."""
+    buf = ctypes.create_string_buffer(1 << 17)
+    p = (ctypes.addressof(buf) + 255) & ~255
+    ws = 1 << 16
+    f = lib.mxfp4_linear_fprop
+    assert f(p, p, p, 128, 128, 128, 1, 0, 0, 7, p, ws, None) == -4            # out_dtype
+    assert f(p, p, p + 4, 128, 128, 128, 1, 0, 0, 0, p, ws, None) == -3        # out alignment
+    assert f(p, p + 2, p, 128, 128, 128, 1, 0, 0, 0, p, ws, None) == -3        # second operand alignment
+    h = lib.mxfp4_linear_host
+    assert h(0, p, p, p, 128, 128, 128, 1, 0, 0, 9, p, p, p, p, ws, None) == -4
+    assert h(0, p, p, p, 128, 128, 128, 1, 0, 0, 0, p, p + 8, p, p, ws, None) == -3
+    assert h(0, p, p, p, 128, 128, 128, 1, 0, 0, 0, p, p, p, p, 16, None) == -5
+    fw = lib.mxfp4_linear_forward
+    big = 1 << 16
+    assert fw(p, p + 2, p, 64, 64, 64, 1, 0, 0, 0, p, big, p, big, None) == -3  # W misaligned
+    assert fw(p, p, p, 64, 64, 64, 1, 0, 0, 5, p, big, p, big, None) == -4      # out_dtype
+    bw = lib.mxfp4_linear_backward
+    assert bw(p, p, p + 6, 64, 64, 64, 1, 0, 0, 0, 0, p, big, p, big, None) == -3
+    assert bw(p, p, p, 64, 64, 64, 1, 0, 0, 0, 3, p, big, p, big, None) == -4

@@ -364,6 +364,25 @@ def test_sr_worked_tile_and_sign_masks():
     assert oracle.sign_mask(0) == int(g["sign_mask_seed0"][0], 16)
 
 
+def test_sr_comparison_is_strict_at_equality():
+    """u = (u8 + 1/2)/256 equal to frac stays down.  The random byte comes from the generator's
+    published first vector, the expected codes from the hand derivation in the golden file."""
+    g = _sr_golden()
+    kat = [int(x, 16) for x in read_golden_lines("philox4x32_10_kat.txt")[0].split()]
+    assert kat[:6] == [0] * 6
+    u8 = (kat[6] >> 16) & 0xFF                       # element 2: byte 2 of word 0
+    assert u8 == int(g["strict_u8_element2"][0], 16) == 39
+    for n in (78, 79, 80):
+        assert Fraction(n, 512) == Fraction(n, 1024) / Fraction(1, 2)          # frac between 0 and 0.5
+        want = 1 if Fraction(2 * u8 + 1, 512) < Fraction(n, 512) else 0
+        assert want == int(g[f"strict_n{n}_code"][0])
+        vals = [4.0, 0.0, n / 1024] + [0.0] * 29
+        codes, scales = oracle.quantize(bits_row(vals), 1, rounding=1, seed=0, tag=0)
+        got = unpack(codes[0])
+        assert int(scales[0, 0]) == 127 and got[0] == 6 and got[2] == want, (n, got[:4])
+        assert all(c == 0 for i, c in enumerate(got) if i not in (0, 2))
+
+
 def test_sr_is_unbiased_and_never_moves_grid_points():
     # row o of a [rows x 32] matrix uses element indices 32*o .. 32*o+31: fresh bits per row
     rows = 1 << 15

@@ -60,6 +60,21 @@ def test_narrow_column_wise_sources():
     _check(random_bits(rng, 4128, 8), 0, 2, 0)      # K = 4128 = 32 tiles + one block
 
 
+def test_column_wise_source_whose_width_is_not_a_multiple_of_8():
+    """Only the leading dimension has the multiple-of-8 rule: a 100-column view of a 104-wide
+    buffer gives a 100-row transposed operand."""
+    rng = np.random.default_rng(8)
+    full = random_bits(rng, 96, 104)
+    view = to_dev(full)[:, :100]
+    sub = np.ascontiguousarray(full[:, :100])
+    for hmode, rnd in ((1, 0), (0, 1)):
+        codes, scales = api.quantize(view, 0, hmode, rnd, 7, 1)
+        api.check()
+        wc, ws = oracle.quantize(sub, 0, hmode, rnd, 7, 1)
+        assert np.array_equal(codes.cpu().numpy(), wc)
+        assert np.array_equal(oracle.scales_from_tiled(scales.cpu().numpy(), 100, 3), ws)
+
+
 def test_one_row_axis1():
     rng = np.random.default_rng(5)
     _check(random_bits(rng, 1, 64), 1, 1, 0)
@@ -106,6 +121,23 @@ def test_rounding_ties_and_saturation_on_device():
                      -3.5, -5.0, 7.5, -7.5, 0.0, -0.0, 0.1, -0.1, 5.5, -5.5] + [0.0] * 9, dtype=np.float32)
     bits = (vals.view(np.uint32) >> 16).astype(np.uint16)[None, :]
     _check(bits, 1, 0, 0)
+
+
+def test_stochastic_rounding_equality_stays_down_on_device():
+    """Seed 0, tag 0, row 0: element 2 draws u8 = 39 (published first vector of the generator), so
+    79/1024 sits exactly on the threshold (512 * frac = 2 * u8 + 1) and stays at code 0 while
+    80/1024 rounds up; both axes, against the oracle (whose own answer a CPU pin derives by hand)."""
+    for n, want in ((78, 0), (79, 0), (80, 1)):
+        vals = np.zeros((32, 32), dtype=np.float32)
+        vals[0, 0], vals[0, 2] = 4.0, n / 1024
+        bits = (vals.view(np.uint32) >> 16).astype(np.uint16)
+        codes, _, _ = gpu_quantize(bits, 1, 0, 1, 0, 0)
+        assert codes[0, 1] & 0xF == want and codes[0, 0] == 0x06
+        _check(bits, 1, 0, 1, seed=0, tag=0)
+        # column-wise: the same block as column 0 of the transposed source
+        codes, _, _ = gpu_quantize(np.ascontiguousarray(bits.T), 0, 0, 1, 0, 0)
+        assert codes[0, 1] & 0xF == want and codes[0, 0] == 0x06
+        _check(np.ascontiguousarray(bits.T), 0, 0, 1, seed=0, tag=0)
 
 
 def test_results_are_reproducible_run_to_run():

@@ -61,3 +61,27 @@ def test_two_calls_in_a_row_match_the_workspace_entry_points():
     again1 = api.linear_static(api.PASS_FPROP, X1, W1, T1, IN1, OUT1, api.HADAMARD_DET, api.ROUND_RNE, 3)
     api.check()
     assert torch.equal(again1, want1)
+
+
+@pytest.mark.gpu
+def test_ragged_shapes_after_a_call_that_left_other_bytes_everywhere():
+    """Shapes that are multiples of neither the scale tile (128 rows x 128 elements) nor the GEMM
+    tile, right after a larger call with stochastic rounding has left its operands all over the
+    array: the padding rows and blocks of the scale tiles and the code rows past M and N that the
+    GEMM's tile loads touch must all come from this call, so the result equals the workspace entry
+    point's bit for bit."""
+    from gpu_util import random_bits, to_dev
+    rng = np.random.default_rng(78)
+    Tb, INb, OUTb = 2048, 1536, 1024                       # fills ~4.3 MB of the array with non-zero bytes
+    api.linear_static(api.PASS_FPROP, to_dev(random_bits(rng, Tb, INb, 2)), to_dev(random_bits(rng, OUTb, INb, 2)),
+                      Tb, INb, OUTb, api.HADAMARD_NONE, api.ROUND_SR, 5)
+    T, IN, OUT = 200, 416, 328
+    X, W, dY = (to_dev(random_bits(rng, r, c, 2)) for r, c in ((T, IN), (OUT, IN), (T, OUT)))
+    got = api.linear_static(api.PASS_FPROP, X, W, T, IN, OUT, api.HADAMARD_DET, api.ROUND_RNE, 3, api.OUT_FP32)
+    api.check()
+    assert torch.isfinite(got).all()
+    assert torch.equal(got, api.linear_fprop(X, W, api.HADAMARD_DET, api.ROUND_RNE, 3, api.OUT_FP32))
+    got = api.linear_static(api.PASS_DGRAD, dY, W, T, IN, OUT, api.HADAMARD_DET, api.ROUND_RNE, 3, api.OUT_FP32)
+    api.check()
+    assert torch.isfinite(got).all()
+    assert torch.equal(got, api.linear_dgrad(dY, W, api.HADAMARD_DET, api.ROUND_RNE, 3, api.OUT_FP32))
