@@ -75,7 +75,7 @@ def test_ragged_shapes_after_a_call_that_left_other_bytes_everywhere():
     Tb, INb, OUTb = 2048, 1536, 1024                       # fills ~4.3 MB of the array with non-zero bytes
     api.linear_static(api.PASS_FPROP, to_dev(random_bits(rng, Tb, INb, 2)), to_dev(random_bits(rng, OUTb, INb, 2)),
                       Tb, INb, OUTb, api.HADAMARD_NONE, api.ROUND_SR, 5)
-    T, IN, OUT = 200, 416, 328
+    T, IN, OUT = 200, 416, 352
     X, W, dY = (to_dev(random_bits(rng, r, c, 2)) for r, c in ((T, IN), (OUT, IN), (T, OUT)))
     got = api.linear_static(api.PASS_FPROP, X, W, T, IN, OUT, api.HADAMARD_DET, api.ROUND_RNE, 3, api.OUT_FP32)
     api.check()
