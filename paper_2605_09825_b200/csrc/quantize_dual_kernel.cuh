@@ -40,7 +40,6 @@ struct QuantDualSmem {
     alignas(128) uint8_t scale_tile[8][kQScaleTileBytes];
     alignas(8) uint64_t full[kQDStages];
     uint64_t empty[kQDStages];
-    uint64_t stg_free[4];        // per consumer group (single-buffered staging): last trip's stores have read it
     int abort_flag;
 };
 
@@ -85,13 +84,14 @@ __device__ __forceinline__ void load_column_blocks(const uint8_t* stage, int kb,
 // Stage one block's results: codes into the 64-byte-swizzled code tile, the scale byte into the
 // 512-byte scale tile (tiled layout) or straight to global memory (canonical layout).
 __device__ __forceinline__ void stage_block(uint8_t* code_tile, uint8_t* scale_tile, const QuantParams& p, int o,
-                                            int kb, int to, int tk, const uint32_t (&packed)[4], uint32_t byte)
+                                            int kb, int to, int tk, const uint32_t (&packed)[4], uint32_t byte,
+                                            bool ok)
 {
     *reinterpret_cast<uint4*>(code_tile + o * 64 + ((kb ^ ((o >> 1) & 3)) * 16)) =
         make_uint4(packed[0], packed[1], packed[2], packed[3]);
     if (p.scale_layout == 1) {
         scale_tile[(o & 31) * 16 + (o >> 5) * 4 + kb] = static_cast<uint8_t>(byte);
-    } else {
+    } else if (ok) {
         const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
         const int64_t tg = static_cast<int64_t>(tk) * 4 + kb;
         if (og < p.outer && tg < p.nt) p.scales[og * p.nt + tg] = static_cast<uint8_t>(byte);
@@ -118,7 +118,6 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
             mbar_init(&sm.full[s], 1);
             mbar_init(&sm.empty[s], kQDGroupThreads / 32);  // the warps of one consumer group
         }
-        for (int g = 0; g < 4; ++g) mbar_init(&sm.stg_free[g], 1);
         fence_barrier_init();
     }
     __syncthreads();
@@ -163,76 +162,72 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
         const uint32_t round = it / kQDStages;
         const int slot = (grp * kQDBufs + (kQDBufs == 2 ? (trip & 1) : 0)) * 2;   // staging tiles of this trip
         const bool ok = mbar_wait(&sm.full[s], round & 1, &sm.abort_flag);
-
-        // A wait that gave up skips the rest of the tile's work and goes straight to the group's
-        // barrier below -- the only CTA barrier of a trip, so every thread reaches it exactly once
-        // whatever happened before -- where the whole group learns of it and leaves.
-        bool good = ok;
-        if (good) {
-            const uint8_t* stage = &sm.stage[s][0];
-            float2 P0[16], P1[16];
-            uint32_t packed[4], byte;
-#pragma unroll
-            for (int u = 0; u < kQDSub; ++u) {
-                const int tv = t + u * kQDGroupThreads;     // position in the 256-thread layout of a tile
-                const int kbh = tv >> 7;                    // row-wise: blocks kbh and kbh + 2 of source row o
-                const int o = tv & 127;
-                const int kbc = tv >> 6;                    // column-wise: block kbc of source columns 2*jc, 2*jc + 1
-                const int jc = tv & 63;
-                if (!good) break;
-
-                // ---- row-wise operand: operand row = source row, K = columns
-                load_block<1, HMODE>(stage, kbh, o, pr.signs, P0);
-                load_block<1, HMODE>(stage, kbh + 2, o, pr.signs, P1);
-                {
-                    const uint64_t e_row = static_cast<uint64_t>(tr * 128 + o) * static_cast<uint64_t>(pr.K);
-                    uint8_t* ct = &sm.code_tile[slot][0];
-                    uint8_t* st = &sm.scale_tile[slot][0];
-                    quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tc * 4 + kbh) * 32), pr, packed, byte);
-                    if (kQDBufs == 1 && u == 0) {
-                        // single staging buffer: last trip's stores must have read it before anyone
-                        // rewrites it.  The thread that issued them waits for that here -- a whole
-                        // block's arithmetic after issuing them, so it rarely has to -- and tells the
-                        // group through an mbarrier (a bounded wait for everybody else).
-                        if (t == 0) {
-                            bulk_wait_group_read<0>();
-                            mbar_arrive(&sm.stg_free[grp]);
-                        }
-                        good = mbar_wait(&sm.stg_free[grp], trip & 1, &sm.abort_flag);
-                        if (!good) break;
-                    }
-                    stage_block(ct, st, pr, o, kbh, tr, tc, packed, byte);
-                    quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tc * 4 + kbh + 2) * 32), pr, packed, byte);
-                    stage_block(ct, st, pr, o, kbh + 2, tr, tc, packed, byte);
-                }
-
-                // ---- column-wise operand: operand row = source column, K = rows
-                load_column_blocks<HMODE>(stage, kbc, jc, pc.signs, P0, P1);
-                if (u == kQDSub - 1) {
-                    // the stage is in registers now: hand it back to the producer
-                    __syncwarp();
-                    if ((tid & 31) == 0) mbar_arrive(&sm.empty[s]);
-                }
-                {
-                    float amax0 = rotate_and_amax<HMODE>(P0);
-                    float amax1 = rotate_and_amax<HMODE>(P1);
-                    if (pc.block2d) amax0 = amax1 = lanes_max(half_mask, fmaxf(amax0, amax1));
-                    const uint64_t e_blk = static_cast<uint64_t>((tr * 4 + kbc) * 32);
-                    const uint64_t e_row = static_cast<uint64_t>(tc * 128 + 2 * jc) * static_cast<uint64_t>(pc.K);
-                    uint8_t* ct = &sm.code_tile[slot + 1][0];
-                    uint8_t* st = &sm.scale_tile[slot + 1][0];
-                    scale_round_pack<SR>(P0, amax0, e_row + e_blk, pc, packed, byte);
-                    stage_block(ct, st, pc, 2 * jc, kbc, tc, tr, packed, byte);
-                    scale_round_pack<SR>(P1, amax1, e_row + static_cast<uint64_t>(pc.K) + e_blk, pc, packed, byte);
-                    stage_block(ct, st, pc, 2 * jc + 1, kbc, tc, tr, packed, byte);
-                }
-            }
-            fence_proxy_async_smem();
-            // double-buffered staging: the stores this group issued one trip ago must have drained
-            // their buffers before the next trip (which every thread of the group reaches only
-            // through the barrier below) overwrites them
-            if (kQDBufs == 2 && t == 0) bulk_wait_group_read<0>();
+        if (kQDBufs == 1) {
+            // single staging buffer: last trip's stores must have read it before anyone rewrites it
+            if (t == 0) bulk_wait_group_read<0>();
+            asm volatile("barrier.cta.sync %0, %1;" ::"r"(grp + 1), "n"(kQDGroupThreads) : "memory");
         }
+
+        float2 P0[16], P1[16];
+        uint32_t packed[4], byte;
+#pragma unroll
+        for (int u = 0; u < kQDSub; ++u) {
+            const int tv = t + u * kQDGroupThreads;     // position in the 256-thread layout of a tile
+            const int kbh = tv >> 7;                    // row-wise: blocks kbh and kbh + 2 of source row o
+            const int o = tv & 127;
+            const int kbc = tv >> 6;                    // column-wise: block kbc of source columns 2*jc, 2*jc + 1
+            const int jc = tv & 63;
+
+            // ---- row-wise operand: operand row = source row, K = columns
+            if (ok) {
+                load_block<1, HMODE>(&sm.stage[s][0], kbh, o, pr.signs, P0);
+                load_block<1, HMODE>(&sm.stage[s][0], kbh + 2, o, pr.signs, P1);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
+            }
+            {
+                const uint64_t e_row = static_cast<uint64_t>(tr * 128 + o) * static_cast<uint64_t>(pr.K);
+                uint8_t* ct = &sm.code_tile[slot][0];
+                uint8_t* st = &sm.scale_tile[slot][0];
+                quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tc * 4 + kbh) * 32), pr, packed, byte);
+                stage_block(ct, st, pr, o, kbh, tr, tc, packed, byte, ok);
+                quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tc * 4 + kbh + 2) * 32), pr, packed, byte);
+                stage_block(ct, st, pr, o, kbh + 2, tr, tc, packed, byte, ok);
+            }
+
+            // ---- column-wise operand: operand row = source column, K = rows
+            if (ok) {
+                load_column_blocks<HMODE>(&sm.stage[s][0], kbc, jc, pc.signs, P0, P1);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
+            }
+            if (u == kQDSub - 1) {
+                // the stage is in registers now: hand it back to the producer
+                __syncwarp();
+                if ((tid & 31) == 0) mbar_arrive(&sm.empty[s]);
+            }
+            {
+                float amax0 = rotate_and_amax<HMODE>(P0);
+                float amax1 = rotate_and_amax<HMODE>(P1);
+                if (pc.block2d) amax0 = amax1 = lanes_max(half_mask, fmaxf(amax0, amax1));
+                const uint64_t e_blk = static_cast<uint64_t>((tr * 4 + kbc) * 32);
+                const uint64_t e_row = static_cast<uint64_t>(tc * 128 + 2 * jc) * static_cast<uint64_t>(pc.K);
+                uint8_t* ct = &sm.code_tile[slot + 1][0];
+                uint8_t* st = &sm.scale_tile[slot + 1][0];
+                scale_round_pack<SR>(P0, amax0, e_row + e_blk, pc, packed, byte);
+                stage_block(ct, st, pc, 2 * jc, kbc, tc, tr, packed, byte, ok);
+                scale_round_pack<SR>(P1, amax1, e_row + static_cast<uint64_t>(pc.K) + e_blk, pc, packed, byte);
+                stage_block(ct, st, pc, 2 * jc + 1, kbc, tc, tr, packed, byte, ok);
+            }
+        }
+
+        fence_proxy_async_smem();
+        // double-buffered staging: the stores this group issued one trip ago must have drained
+        // their buffers before the next trip (which every thread of the group reaches only
+        // through the barrier below) overwrites them
+        if (kQDBufs == 2 && t == 0) bulk_wait_group_read<0>();
         uint32_t any_fail;
         asm volatile(
             "{\n\t.reg .pred P, Q;\n\t"
@@ -240,7 +235,7 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
             "barrier.cta.red.or.pred P, %2, %3, Q;\n\t"
             "selp.u32 %0, 1, 0, P;\n\t}"
             : "=r"(any_fail)
-            : "r"(good ? 0u : 1u), "r"(grp + 1), "n"(kQDGroupThreads)
+            : "r"(ok ? 0u : 1u), "r"(grp + 1), "n"(kQDGroupThreads)
             : "memory");
         if (any_fail) break;
         if (t == 0) {

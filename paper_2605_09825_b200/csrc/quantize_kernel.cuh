@@ -42,7 +42,6 @@ struct QuantSmem {
     alignas(128) uint8_t scale_tile[4][kQScaleTileBytes];
     alignas(8) uint64_t full[kQStages];
     uint64_t empty[kQStages];
-    uint64_t stg_free[4];        // per consumer group: last trip's store has read the group's staging tile
     int abort_flag;
 };
 
@@ -333,68 +332,58 @@ __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p
     tile_coords<AXIS>(p, tile, to, tk);
 
     const bool ok = mbar_wait(&sm.full[s], round & 1, &sm.abort_flag);
+    if (Shape::kBufs == 1) {
+        // single staging buffer: last trip's store must have read it before anyone rewrites it
+        if (t == 0) bulk_wait_group_read<0>();
+        asm volatile("barrier.cta.sync %0, %1;" ::"r"(grp + 1), "n"(Shape::kGroupThreads) : "memory");
+    }
 
-    // A wait that gave up skips the rest of the tile's work and goes straight to the group's barrier
-    // below -- the only CTA barrier of a trip, so every thread reaches it exactly once whatever
-    // happened before -- where the whole group learns of it and leaves.
-    bool good = ok;
-    if (good) {
 #pragma unroll
-        for (int u = 0; u < Shape::kSub; ++u) {
-            const int tv = t + u * Shape::kGroupThreads;   // position in the 256-thread layout of a tile
-            const int kbh = tv >> 7;                       // this thread's blocks along K: kbh and kbh + 2
-            const int o = tv & 127;                        // operand row inside the tile
-            if (!good) break;
-            float2 P0[16], P1[16];
+    for (int u = 0; u < Shape::kSub; ++u) {
+        const int tv = t + u * Shape::kGroupThreads;   // position in the 256-thread layout of a tile
+        const int kbh = tv >> 7;                       // this thread's blocks along K: kbh and kbh + 2
+        const int o = tv & 127;                        // operand row inside the tile
+        float2 P0[16], P1[16];
+        if (ok) {
             load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.signs, P0);
             load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.signs, P1);
-            if (u == Shape::kSub - 1) {
-                // the stage is in registers now: hand it back to the producer
-                __syncwarp();
-                if ((t & 31) == 0) mbar_arrive(&sm.empty[s]);
-            }
-
-            const uint64_t e_row = static_cast<uint64_t>(to * kQTileO + o) * static_cast<uint64_t>(p.K);
-            uint32_t packed0[4], packed1[4], byte0, byte1;
-            quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tk * 4 + kbh) * 32), p, packed0, byte0);
-            quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tk * 4 + kbh + 2) * 32), p, packed1, byte1);
-
-            if (Shape::kBufs == 1 && u == 0) {
-                // single staging buffer: last trip's store must have read it before anyone rewrites
-                // it.  The thread that issued the store waits for that here -- two blocks' arithmetic
-                // after issuing it, so it rarely has to -- and tells the group through an mbarrier
-                // (a bounded wait for everybody else).
-                if (t == 0) {
-                    bulk_wait_group_read<0>();
-                    mbar_arrive(&sm.stg_free[grp]);
-                }
-                good = mbar_wait(&sm.stg_free[grp], trip & 1, &sm.abort_flag);
-                if (!good) break;
-            }
-
-            // stage the results: codes in the 64-byte swizzle the TMA store expects
-            uint8_t* ct = &sm.code_tile[slot][o * 64];
-            *reinterpret_cast<uint4*>(ct + ((kbh ^ ((o >> 1) & 3)) * 16)) =
-                make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]);
-            *reinterpret_cast<uint4*>(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16)) =
-                make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]);
-            if (p.scale_layout == 1) {
-                uint8_t* st = &sm.scale_tile[slot][(o & 31) * 16 + (o >> 5) * 4];
-                st[kbh] = static_cast<uint8_t>(byte0);
-                st[kbh + 2] = static_cast<uint8_t>(byte1);
-            } else {
-                const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
-                const int64_t tg = static_cast<int64_t>(tk) * 4 + kbh;
-                if (og < p.outer && tg < p.nt) p.scales[og * p.nt + tg] = static_cast<uint8_t>(byte0);
-                if (og < p.outer && tg + 2 < p.nt) p.scales[og * p.nt + tg + 2] = static_cast<uint8_t>(byte1);
-            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
         }
-        fence_proxy_async_smem();
-        // double-buffered staging: the store this group issued one trip ago must have drained its
-        // buffer before the next trip (which every thread of the group reaches only through the
-        // barrier below) overwrites it
-        if (Shape::kBufs == 2 && t == 0) bulk_wait_group_read<0>();
+        if (u == Shape::kSub - 1) {
+            // the stage is in registers now: hand it back to the producer
+            __syncwarp();
+            if ((t & 31) == 0) mbar_arrive(&sm.empty[s]);
+        }
+
+        const uint64_t e_row = static_cast<uint64_t>(to * kQTileO + o) * static_cast<uint64_t>(p.K);
+        uint32_t packed0[4], packed1[4], byte0, byte1;
+        quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tk * 4 + kbh) * 32), p, packed0, byte0);
+        quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tk * 4 + kbh + 2) * 32), p, packed1, byte1);
+
+        // stage the results: codes in the 64-byte swizzle the TMA store expects
+        uint8_t* ct = &sm.code_tile[slot][o * 64];
+        *reinterpret_cast<uint4*>(ct + ((kbh ^ ((o >> 1) & 3)) * 16)) =
+            make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]);
+        *reinterpret_cast<uint4*>(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16)) =
+            make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]);
+        if (p.scale_layout == 1) {
+            uint8_t* st = &sm.scale_tile[slot][(o & 31) * 16 + (o >> 5) * 4];
+            st[kbh] = static_cast<uint8_t>(byte0);
+            st[kbh + 2] = static_cast<uint8_t>(byte1);
+        } else if (ok) {
+            const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
+            const int64_t tg = static_cast<int64_t>(tk) * 4 + kbh;
+            if (og < p.outer && tg < p.nt) p.scales[og * p.nt + tg] = static_cast<uint8_t>(byte0);
+            if (og < p.outer && tg + 2 < p.nt) p.scales[og * p.nt + tg + 2] = static_cast<uint8_t>(byte1);
+        }
     }
+    fence_proxy_async_smem();
+    // double-buffered staging: the store this group issued one trip ago must have drained its
+    // buffer before the next trip (which every thread of the group reaches only through the
+    // barrier below) overwrites it
+    if (Shape::kBufs == 2 && t == 0) bulk_wait_group_read<0>();
     uint32_t any_fail;
     asm volatile(
         "{\n\t.reg .pred P, Q;\n\t"
@@ -402,7 +391,7 @@ __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p
         "barrier.cta.red.or.pred P, %2, %3, Q;\n\t"
         "selp.u32 %0, 1, 0, P;\n\t}"
         : "=r"(any_fail)
-        : "r"(good ? 0u : 1u), "r"(grp + 1), "n"(Shape::kGroupThreads)
+        : "r"(ok ? 0u : 1u), "r"(grp + 1), "n"(Shape::kGroupThreads)
         : "memory");
     if (any_fail) return false;
     if (t == 0) {
@@ -434,7 +423,6 @@ quantize_kernel(const __grid_constant__ QuantJobs jobs)
             mbar_init(&sm.full[s], 1);
             mbar_init(&sm.empty[s], Shape::kGroupThreads / 32);   // the warps of one consumer group
         }
-        for (int g = 0; g < 4; ++g) mbar_init(&sm.stg_free[g], 1);
         fence_barrier_init();
     }
     __syncthreads();
