@@ -639,16 +639,42 @@ def run_ours(args):
         e2e_step = e2e_step_layer if layer else e2e_step_per_pass
 
         e2e_step()
-        n_e2e = max(1, min(args.steps, 3))
+        n_e2e = max(1, min(args.steps, 6))
         sync_all()
         t0 = time.perf_counter()
         for _ in range(n_e2e):
             e2e_step()
         sync_all()
         e2e_ms = aggregate_over_ranks((time.perf_counter() - t0) * 1e3, world)
+        # what the bus itself gives with both directions busy: plain pinned copies of 1 GiB each way
+        # at the same time on two streams (the end-to-end step moves h2d and d2h bytes concurrently)
+        bus = None
+        try:
+            nb = 1 << 30
+            hb_in, hb_out = torch.empty(nb, dtype=torch.uint8).pin_memory(), torch.empty(nb, dtype=torch.uint8).pin_memory()
+            db_in, db_out = torch.empty(nb, dtype=torch.uint8, device="cuda"), torch.empty(nb, dtype=torch.uint8, device="cuda")
+            s_up, s_down = torch.cuda.Stream(), torch.cuda.Stream()
+            best = 0.0
+            for rep in range(3):
+                torch.cuda.synchronize()
+                tb = time.perf_counter()
+                with torch.cuda.stream(s_up):
+                    db_in.copy_(hb_in, non_blocking=True)
+                with torch.cuda.stream(s_down):
+                    hb_out.copy_(db_out, non_blocking=True)
+                torch.cuda.synchronize()
+                best = max(best, nb / (time.perf_counter() - tb) / 1e9)
+            bus = best
+            del hb_in, hb_out, db_in, db_out
+        except Exception:
+            bus = None
+        e2e_gbs = max(h2d, d2h) / (e2e_ms / n_e2e * 1e-3) / 1e9
         e2e = {"value": world * flops_per_step * n_e2e / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
                "ms_per_step": e2e_ms / n_e2e,
+               "bus": {"bound": "pcie", "achieved_gbs_each_way": e2e_gbs, "peak_gbs_each_way": bus,
+                       "frac": (e2e_gbs / bus) if bus else None,
+                       "peak_source": "measured in this run: 1 GiB pinned copies, both directions at once"},
                "note": ("mxfp4_linear_layer_host per linear: pinned X, W, dY copied in once each, Y, dX, dW "
                         "copied out to their own host buffers, copies overlapped with each other, with the kernels and "
                         "across the linears of a step, drained once per step"

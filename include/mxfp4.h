@@ -310,11 +310,13 @@ int mxfp4_linear_host(int pass, const void* a_host, const void* b_host, void* ou
  * copy stream, each as soon as its GEMM has finished, so results flow out while dY still flows
  * in.  With drain != 0 the call returns after everything has drained: the three host outputs are
  * valid.  With drain == 0 it returns as soon as the work is queued, so that the next layer's
- * inputs travel while this layer's results are still on their way back (the next call orders
- * itself after this one wherever the two share a staging buffer, provided both use the same
- * `stream`); the host outputs of all
- * undrained calls are valid after mxfp4_linear_layer_host_drain(stream), and the host inputs must
- * stay untouched until then.
+ * inputs travel while this layer's kernels run and its results are still on their way back.
+ * Consecutive calls order themselves buffer by buffer, assuming that they pass the same staging
+ * buffers in the same roles and the same `stream`: an input staging buffer is overwritten once the
+ * previous call's quantize launch has read it, an output staging buffer once the previous call's
+ * copy to the host has left it.  No other work may use the staging buffers while such calls are
+ * in flight.  The host outputs of all undrained calls are valid after
+ * mxfp4_linear_layer_host_drain(stream), and the host inputs must stay untouched until then.
  *   dev_x, dev_w, dev_dy    device staging for the bf16 inputs ([T x in], [out x in], [T x out]);
  *   dev_y, dev_dx, dev_dw   device staging for the outputs; all six distinct;
  *   saved, workspace        as for forward / backward; workspace must cover the larger of

@@ -111,11 +111,27 @@ __device__ __forceinline__ uint32_t make_idesc_mx_pair(uint32_t a_sf_id, uint32_
     d |= b_sf_id << 4;                 // bits 4..5   B scale-factor id
     d |= (KIND == 0 ? 1u : 0u) << 7;   // bits 7..9   A format: E2M1 (mxf4) / E4M3 (mxf8f6f4)
     d |= (KIND == 0 ? 1u : 0u) << 10;  // bits 10..12 B format
-    d |= (kPMmaN >> 3) << 17;          // bits 17..22 N / 8
+    //                                    bits 17..22 N / 8: added per MMA (idesc_n), see below
     d |= 1u << 23;                     // bit 23      scale format: E8M0
     d |= (kPTileM >> 4) << 24;         // bits 24..28 M / 16
     d |= a_sf_id << 29;                // bits 29..30 A scale-factor id
     return d;
+}
+
+// N field of the instruction descriptor.  N is 192 for every MMA except in a matrix's last tile
+// column, where it shrinks to the columns that exist (rounded up to the instruction's granule of
+// 16): an MMA's issue time is proportional to N, so e.g. the 256 columns that N = 4096 leaves for
+// its eleventh tile cost 192 + 64 instead of 2 x 192.
+__device__ __forceinline__ uint32_t idesc_n(int n) { return static_cast<uint32_t>(n >> 3) << 17; }
+
+// Columns the two MMAs of a tile in tile column `tn` compute: n0 for accumulator columns 0..191,
+// n1 (possibly 0: no MMA) for columns 192..383.  CTA r of the pair supplies rows
+// [r * n / 2, (r + 1) * n / 2) of the MMA's n rows of B, so the producer needs the same numbers.
+__device__ __forceinline__ void tile_mma_widths(int N, int tn, int& n0, int& n1)
+{
+    const int nv = min(kPTileN, N - tn * kPTileN);
+    n0 = min(kPMmaN, (nv + 15) & ~15);
+    n1 = nv > kPMmaN ? min(kPMmaN, (nv - kPMmaN + 15) & ~15) : 0;
 }
 
 // The kernel body for both operand widths.  A stage is 128 bytes of codes per operand row either
@@ -168,11 +184,11 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
     griddep_launch_dependents();
     griddep_wait();
 
-    // register budget per role (whole warpgroups): 4*32*(56 + 2*192 + 56) = 63488 <= 65536;
-    // every warp of a warpgroup executes the same setmaxnreg at the top of its role
+    // register budget per role (whole warpgroups): 4*32*(56 + 2*192 + 72) = 65536, all of the register
+    // file; every warp of a warpgroup executes the same setmaxnreg at the top of its role
     if (warp == kPProducerWarp) {
         // ------------------------------------------------------------ TMA producer
-        setmaxnreg_dec<56>();
+        setmaxnreg_dec<72>();
         if (lane == 0) {
             tma_prefetch_desc(&tm_a);
             tma_prefetch_desc(&tm_b);
@@ -183,6 +199,12 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
             const int tile = cluster_id + t * n_clusters;
             const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
             const int a_row_tile = tm * 2 + static_cast<int>(rank);     // 128-row scale tile of A
+            int n0, n1;
+            tile_mma_widths(p.N, tn, n0, n1);
+            // this CTA's share of B: rows [rank * n / 2, ...) of each MMA's n rows (the box is always 96
+            // rows: what lies beyond the share is not read by the MMA, what lies beyond N arrives as zeros)
+            const int32_t yb0 = tn * kPTileN + static_cast<int>(rank) * (n0 >> 1);
+            const int32_t yb1 = tn * kPTileN + kPMmaN + static_cast<int>(rank) * (n1 >> 1);
             for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
                 const int s = it % kPStages;
                 const uint32_t round = it / kPStages;
@@ -196,10 +218,9 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
                     mbar_arrive_expect_tx_cluster(full_leader, kPABytes + 2 * kPBSubBytes);
                     const int32_t x = ks * 128;                          // bytes along the code row
                     const int32_t ya = tm * kPTileM + rank * kPHalfM;
-                    const int32_t yb = tn * kPTileN + rank * kPSubN;
                     tma_load_2d_pair(sm.a[s], &tm_a, full_leader, x, ya);
-                    tma_load_2d_pair(sm.b[s][0], &tm_b, full_leader, x, yb);
-                    tma_load_2d_pair(sm.b[s][1], &tm_b, full_leader, x, yb + kPMmaN);
+                    tma_load_2d_pair(sm.b[s][0], &tm_b, full_leader, x, yb0);
+                    tma_load_2d_pair(sm.b[s][1], &tm_b, full_leader, x, yb1);
                     // scales: local barrier
                     const int kt0 = ks * kSfTilesPerStage;
                     const int nkt = min(kSfTilesPerStage, p.sf_tiles_k - kt0);
@@ -222,7 +243,7 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
         }
     } else if (warp == kPMmaWarp) {
         // ------------------------------------------------------------ MMA issuer (leader only)
-        setmaxnreg_dec<56>();
+        setmaxnreg_dec<72>();
         if (rank == 0 && total_it > 0) {
             int it = 0;
             bool alive = true;
@@ -237,6 +258,9 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
             int s = 0;
             uint32_t parity = 0;
             for (int tile_it = 0; alive && tile_it < my_tiles; ++tile_it) {
+                int n0, n1;
+                tile_mma_widths(p.N, (cluster_id + tile_it * n_clusters) / p.tiles_m, n0, n1);
+                const uint32_t idn0 = idesc_n(n0), idn1 = idesc_n(n1);
                 if (tile_it > 0 && !mbar_wait(&sm.tmem_empty, (tile_it - 1) & 1, &sm.abort_flag)) break;
                 for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
                     // codes landed in both CTAs' shared memory; scales landed in both CTAs' TMEM
@@ -267,11 +291,12 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
                                                                  : (j == 0 ? idesc0 : j == 1 ? idesc1 : j == 2 ? idesc2 : idesc3);
                                 const uint32_t sfa = sf_tmem + (KIND == 0 ? (j >> 1) * 4 : 0);
                                 const uint32_t sfb = sf_tmem + 8 + (KIND == 0 ? (j >> 1) * 12 : 0);
-                                tcgen05_mma_mx_pair_collect<KIND, 0>(tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, sfa, sfb,
-                                                                     (ks > 0 || j > 0) ? 1u : 0u);
-                                tcgen05_mma_mx_pair_collect<KIND, 1>(tmem + kPMmaN, a_desc + 2 * j,
-                                                                     b_desc + 2 * j + (kPBSubBytes >> 4), idesc, sfa,
-                                                                     sfb + 6, (ks > 0 || j > 0) ? 1u : 0u);
+                                tcgen05_mma_mx_pair_collect<KIND, 0>(tmem, a_desc + 2 * j, b_desc + 2 * j, idesc | idn0, sfa,
+                                                                     sfb, (ks > 0 || j > 0) ? 1u : 0u);
+                                if (n1 > 0)
+                                    tcgen05_mma_mx_pair_collect<KIND, 1>(tmem + kPMmaN, a_desc + 2 * j,
+                                                                         b_desc + 2 * j + (kPBSubBytes >> 4), idesc | idn1,
+                                                                         sfa, sfb + 6, (ks > 0 || j > 0) ? 1u : 0u);
                             }
                         }
                         // frees the shared-memory stage and its TMEM scale columns in both CTAs
@@ -441,7 +466,7 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
         }
         if (lane == 0) bulk_wait_group<0>();
     } else {
-        setmaxnreg_dec<56>();   // idle warps of the producer/MMA warpgroup
+        setmaxnreg_dec<72>();   // idle warps of the producer/MMA warpgroup
     }
 
     // neither CTA may leave (or free TMEM) while its peer can still signal it or read its memory

@@ -616,9 +616,31 @@ static float rotation_alpha(int hmode)
     return hmode == MXFP4_HADAMARD_NONE ? 1.0f : (hmode <= MXFP4_HADAMARD_RAND ? 0.03125f : 0.0625f);
 }
 
-int mxfp4_linear_forward(const void* X, const void* W, void* Y, int64_t T, int64_t in_features,
-                         int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int out_dtype,
-                         void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream)
+// Optional stream ordering around the three launches of a forward or backward call, used by the
+// host-buffer form to tie each launch to the copy that feeds it or drains it: `wait[i]` (if set)
+// is waited for on the stream before launch i, `done[i]` (if set) is recorded after it.
+struct LaunchHooks {
+    cudaEvent_t wait[3];
+    cudaEvent_t done[3];
+};
+
+static int hook_wait(const LaunchHooks* h, int i, cudaStream_t st)
+{
+    if (h && h->wait[i] && cudaStreamWaitEvent(st, h->wait[i], 0) != cudaSuccess) return MXFP4_ERR_CUDA;
+    return MXFP4_OK;
+}
+
+static int hook_done(const LaunchHooks* h, int i, cudaStream_t st)
+{
+    if (h && h->done[i] && cudaEventRecord(h->done[i], st) != cudaSuccess) return MXFP4_ERR_CUDA;
+    return MXFP4_OK;
+}
+
+// mxfp4_linear_forward; launches: 0 = quantize X, 1 = quantize W, 2 = Fprop GEMM.
+static int linear_forward_impl(const void* X, const void* W, void* Y, int64_t T, int64_t in_features,
+                               int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int out_dtype,
+                               void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream,
+                               const LaunchHooks* hooks)
 {
     if (!X || !W || !Y) return MXFP4_ERR_NULL;
     if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
@@ -626,6 +648,7 @@ int mxfp4_linear_forward(const void* X, const void* W, void* Y, int64_t T, int64
     int rc = layer_args_ok(T, in_features, out_features, hadamard_mode, rounding, saved, saved_bytes, workspace,
                            workspace_bytes, MXFP4_LAYER_FORWARD);
     if (rc != MXFP4_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     uint8_t* x_codes = ws;
     uint8_t* x_scales = x_codes + round_up(mxfp4_codes_bytes(T, in_features), 256);
@@ -637,21 +660,34 @@ int mxfp4_linear_forward(const void* X, const void* W, void* Y, int64_t T, int64
     uint8_t* wt_codes = sv + operand_bytes(in_features, T);
     uint8_t* wt_scales = wt_codes + round_up(mxfp4_codes_bytes(in_features, out_features), 256);
     // tags as in the per-pass entry points: A operands 0, B operands 1 (X^T is Wgrad's B, W^T Dgrad's B)
+    if ((rc = hook_wait(hooks, 0, st)) != MXFP4_OK) return rc;
     rc = mxfp4_quantize_dual(X, T, in_features, in_features, hadamard_mode, rounding, seed, 0u, 1u,
                              MXFP4_BLOCK_1X32, x_codes, x_scales, xt_codes, xt_scales, MXFP4_SCALES_TILED, stream);
     if (rc != MXFP4_OK) return rc;
+    if ((rc = hook_done(hooks, 0, st)) != MXFP4_OK || (rc = hook_wait(hooks, 1, st)) != MXFP4_OK) return rc;
     rc = mxfp4_quantize_dual(W, out_features, in_features, in_features, hadamard_mode, rounding, seed, 1u, 1u,
                              MXFP4_BLOCK_1X32, w_codes, w_scales, wt_codes, wt_scales, MXFP4_SCALES_TILED, stream);
     if (rc != MXFP4_OK) return rc;
-    return mxfp4_gemm(x_codes, x_scales, w_codes, w_scales, T, out_features, in_features,
-                      rotation_alpha(hadamard_mode), Y, out_dtype, out_features, nullptr, 0, stream);
+    if ((rc = hook_done(hooks, 1, st)) != MXFP4_OK || (rc = hook_wait(hooks, 2, st)) != MXFP4_OK) return rc;
+    rc = mxfp4_gemm(x_codes, x_scales, w_codes, w_scales, T, out_features, in_features,
+                    rotation_alpha(hadamard_mode), Y, out_dtype, out_features, nullptr, 0, stream);
+    if (rc != MXFP4_OK) return rc;
+    return hook_done(hooks, 2, st);
 }
 
-// mxfp4_linear_backward; `after_dx` (optional) is recorded between the two GEMMs.
+int mxfp4_linear_forward(const void* X, const void* W, void* Y, int64_t T, int64_t in_features,
+                         int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int out_dtype,
+                         void* saved, size_t saved_bytes, void* workspace, size_t workspace_bytes, void* stream)
+{
+    return linear_forward_impl(X, W, Y, T, in_features, out_features, hadamard_mode, rounding, seed, out_dtype, saved,
+                               saved_bytes, workspace, workspace_bytes, stream, nullptr);
+}
+
+// mxfp4_linear_backward; launches: 0 = quantize dY, 1 = Dgrad GEMM, 2 = Wgrad GEMM.
 static int linear_backward_impl(const void* dY, void* dX, void* dW, int64_t T, int64_t in_features,
                                 int64_t out_features, int hadamard_mode, int rounding, uint64_t seed, int dx_dtype,
                                 int dw_dtype, const void* saved, size_t saved_bytes, void* workspace,
-                                size_t workspace_bytes, void* stream, cudaEvent_t after_dx)
+                                size_t workspace_bytes, void* stream, const LaunchHooks* hooks)
 {
     if (!dY || !dX || !dW) return MXFP4_ERR_NULL;
     for (int d : {dx_dtype, dw_dtype})
@@ -670,18 +706,23 @@ static int linear_backward_impl(const void* dY, void* dX, void* dW, int64_t T, i
     const uint8_t* xt_scales = xt_codes + round_up(mxfp4_codes_bytes(in_features, T), 256);
     const uint8_t* wt_codes = sv + operand_bytes(in_features, T);
     const uint8_t* wt_scales = wt_codes + round_up(mxfp4_codes_bytes(in_features, out_features), 256);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((rc = hook_wait(hooks, 0, st)) != MXFP4_OK) return rc;
     rc = mxfp4_quantize_dual(dY, T, out_features, out_features, hadamard_mode, rounding, seed, 0u, 0u,
                              MXFP4_BLOCK_1X32, dy_codes, dy_scales, dyt_codes, dyt_scales, MXFP4_SCALES_TILED, stream);
     if (rc != MXFP4_OK) return rc;
+    if ((rc = hook_done(hooks, 0, st)) != MXFP4_OK || (rc = hook_wait(hooks, 1, st)) != MXFP4_OK) return rc;
     const float alpha = rotation_alpha(hadamard_mode);
     // dX [T x in] = dY [T x out] . (W^T operand [in x out])^T
     rc = mxfp4_gemm(dy_codes, dy_scales, wt_codes, wt_scales, T, in_features, out_features, alpha, dX, dx_dtype,
                     in_features, nullptr, 0, stream);
     if (rc != MXFP4_OK) return rc;
-    if (after_dx && cudaEventRecord(after_dx, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MXFP4_ERR_CUDA;
+    if ((rc = hook_done(hooks, 1, st)) != MXFP4_OK || (rc = hook_wait(hooks, 2, st)) != MXFP4_OK) return rc;
     // dW [out x in] = dY^T [out x T] . (X^T operand [in x T])^T
-    return mxfp4_gemm(dyt_codes, dyt_scales, xt_codes, xt_scales, out_features, in_features, T, alpha, dW, dw_dtype,
-                      in_features, nullptr, 0, stream);
+    rc = mxfp4_gemm(dyt_codes, dyt_scales, xt_codes, xt_scales, out_features, in_features, T, alpha, dW, dw_dtype,
+                    in_features, nullptr, 0, stream);
+    if (rc != MXFP4_OK) return rc;
+    return hook_done(hooks, 2, st);
 }
 
 int mxfp4_linear_backward(const void* dY, void* dX, void* dW, int64_t T, int64_t in_features,
@@ -697,8 +738,12 @@ int mxfp4_linear_backward(const void* dY, void* dX, void* dW, int64_t T, int64_t
 // use and kept for the life of the process.
 struct HostPipe {
     cudaStream_t h2d, d2h;
-    cudaEvent_t start, xw, dy, y, dx, dw, done;
-    bool ready;
+    // per tensor t in (X, W, dY): in[t] = its copy to the device has landed, read[t] = the quantize
+    // launch that reads its staging buffer is done (the buffer may be overwritten);
+    // per result r in (Y, dX, dW): ready[r] = its GEMM is done, out[r] = its copy to the host is
+    // done (the staging buffer may be overwritten)
+    cudaEvent_t in[3], read[3], ready[3], out[3];
+    bool ok;
 };
 
 static int host_pipe(HostPipe** out)
@@ -713,10 +758,10 @@ static int host_pipe(HostPipe** out)
         if (cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking) != cudaSuccess ||
             cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking) != cudaSuccess)
             return MXFP4_ERR_CUDA;
-        cudaEvent_t* evs[7] = {&p.start, &p.xw, &p.dy, &p.y, &p.dx, &p.dw, &p.done};
-        for (cudaEvent_t* e : evs)
-            if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return MXFP4_ERR_CUDA;
-        p.ready = true;
+        for (cudaEvent_t* set : {p.in, p.read, p.ready, p.out})
+            for (int i = 0; i < 3; ++i)
+                if (cudaEventCreateWithFlags(&set[i], cudaEventDisableTiming) != cudaSuccess) return MXFP4_ERR_CUDA;
+        p.ok = true;
         return MXFP4_OK;
     });
 }
@@ -754,36 +799,37 @@ int mxfp4_linear_layer_host(const void* X_host, const void* W_host, const void* 
     const size_t dx_out = static_cast<size_t>(T) * in_features * (dx_dtype == MXFP4_OUT_BF16 ? 2 : 4);
     const size_t dw_out = static_cast<size_t>(out_features) * in_features * (dw_dtype == MXFP4_OUT_BF16 ? 2 : 4);
 #define MXFP4_TRY(call) do { if ((call) != cudaSuccess) return MXFP4_ERR_CUDA; } while (0)
-    // inputs travel on their own stream, in the order they are needed; they start once the work
-    // already queued on the caller's stream (which may still use the staging buffers) is done
-    MXFP4_TRY(cudaEventRecord(hp->start, st));
-    MXFP4_TRY(cudaStreamWaitEvent(hp->h2d, hp->start, 0));
-    MXFP4_TRY(cudaMemcpyAsync(dev_x, X_host, x_bytes, cudaMemcpyHostToDevice, hp->h2d));
-    MXFP4_TRY(cudaMemcpyAsync(dev_w, W_host, w_bytes, cudaMemcpyHostToDevice, hp->h2d));
-    MXFP4_TRY(cudaEventRecord(hp->xw, hp->h2d));
-    MXFP4_TRY(cudaMemcpyAsync(dev_dy, dY_host, dy_bytes, cudaMemcpyHostToDevice, hp->h2d));
-    MXFP4_TRY(cudaEventRecord(hp->dy, hp->h2d));
-    // compute on the caller's stream; the output staging buffers may still be on their way to the
-    // host from the previous call (a no-op wait the first time)
-    MXFP4_TRY(cudaStreamWaitEvent(st, hp->xw, 0));
-    MXFP4_TRY(cudaStreamWaitEvent(st, hp->done, 0));
-    rc = mxfp4_linear_forward(dev_x, dev_w, dev_y, T, in_features, out_features, hadamard_mode, rounding, seed,
-                              y_dtype, saved, saved_bytes, workspace, workspace_bytes, stream);
+    // Inputs travel on their own stream in the order they are needed.  A staging buffer is
+    // overwritten as soon as the quantize launch of the PREVIOUS call that read it is done -- not
+    // when that whole call is -- so the next layer's inputs flow in while this layer's GEMMs run
+    // (waiting on an event that was never recorded is a no-op: the first call).
+    const void* src[3] = {X_host, W_host, dY_host};
+    void* stg_in[3] = {dev_x, dev_w, dev_dy};
+    const size_t in_bytes[3] = {x_bytes, w_bytes, dy_bytes};
+    for (int i = 0; i < 3; ++i) {
+        MXFP4_TRY(cudaStreamWaitEvent(hp->h2d, hp->read[i], 0));
+        MXFP4_TRY(cudaMemcpyAsync(stg_in[i], src[i], in_bytes[i], cudaMemcpyHostToDevice, hp->h2d));
+        MXFP4_TRY(cudaEventRecord(hp->in[i], hp->h2d));
+    }
+    // Compute on the caller's stream: each quantize launch waits for its tensor, each GEMM for the
+    // previous call's copy out of the staging buffer it is about to overwrite.
+    const LaunchHooks fwd = {{hp->in[0], hp->in[1], hp->out[0]}, {hp->read[0], hp->read[1], hp->ready[0]}};
+    rc = linear_forward_impl(dev_x, dev_w, dev_y, T, in_features, out_features, hadamard_mode, rounding, seed, y_dtype,
+                             saved, saved_bytes, workspace, workspace_bytes, stream, &fwd);
     if (rc != MXFP4_OK) return rc;
-    MXFP4_TRY(cudaEventRecord(hp->y, st));
-    MXFP4_TRY(cudaStreamWaitEvent(st, hp->dy, 0));
+    const LaunchHooks bwd = {{hp->in[2], hp->out[1], hp->out[2]}, {hp->read[2], hp->ready[1], hp->ready[2]}};
     rc = linear_backward_impl(dev_dy, dev_dx, dev_dw, T, in_features, out_features, hadamard_mode, rounding, seed,
-                              dx_dtype, dw_dtype, saved, saved_bytes, workspace, workspace_bytes, stream, hp->dx);
+                              dx_dtype, dw_dtype, saved, saved_bytes, workspace, workspace_bytes, stream, &bwd);
     if (rc != MXFP4_OK) return rc;
-    MXFP4_TRY(cudaEventRecord(hp->dw, st));
     // results leave on a third stream, each as soon as its GEMM is done, while later inputs still arrive
-    MXFP4_TRY(cudaStreamWaitEvent(hp->d2h, hp->y, 0));
-    MXFP4_TRY(cudaMemcpyAsync(Y_host, dev_y, y_out, cudaMemcpyDeviceToHost, hp->d2h));
-    MXFP4_TRY(cudaStreamWaitEvent(hp->d2h, hp->dx, 0));
-    MXFP4_TRY(cudaMemcpyAsync(dX_host, dev_dx, dx_out, cudaMemcpyDeviceToHost, hp->d2h));
-    MXFP4_TRY(cudaStreamWaitEvent(hp->d2h, hp->dw, 0));
-    MXFP4_TRY(cudaMemcpyAsync(dW_host, dev_dw, dw_out, cudaMemcpyDeviceToHost, hp->d2h));
-    MXFP4_TRY(cudaEventRecord(hp->done, hp->d2h));
+    void* dst[3] = {Y_host, dX_host, dW_host};
+    const void* stg_out[3] = {dev_y, dev_dx, dev_dw};
+    const size_t out_bytes[3] = {y_out, dx_out, dw_out};
+    for (int i = 0; i < 3; ++i) {
+        MXFP4_TRY(cudaStreamWaitEvent(hp->d2h, hp->ready[i], 0));
+        MXFP4_TRY(cudaMemcpyAsync(dst[i], stg_out[i], out_bytes[i], cudaMemcpyDeviceToHost, hp->d2h));
+        MXFP4_TRY(cudaEventRecord(hp->out[i], hp->d2h));
+    }
 #undef MXFP4_TRY
     return drain ? mxfp4_linear_layer_host_drain(stream) : MXFP4_OK;
 }
