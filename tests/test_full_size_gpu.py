@@ -1,13 +1,18 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times (fused
 passes, bf16 outputs, deterministic H32 + RNE and the config-4 variants): quantized operands
-bit-exact against the oracle on whole tensors, GEMM outputs on sampled rows the oracle computes
-one by one, all columns of each.  The sample holds one seeded row out of EVERY 128-row slab of
-the output plus the slab-edge rows, so every 256 x 384 tile of the persistent grid, every wave
-of it and both CTAs of every pair meet the oracle."""
+bit-exact against the oracle on whole tensors; GEMM outputs checked twice --
+  * against the CPU oracle on sampled rows it computes one by one, all columns of each: one
+    seeded row out of EVERY 128-row slab of the output plus the slab-edge rows, so every
+    256 x 384 tile of the persistent grid, every wave of it and both CTAs of every pair meet
+    the oracle;
+  * EVERY element against a slow fp64 CUDA checker (tests/gemm_checker: one thread per output,
+    integer products, fp64 sums, nothing shared with the library) that multiplies the ORACLE's
+    quantized operands and is itself first held against the oracle on those sampled rows."""
 import numpy as np
 import pytest
 import torch
 
+import gemm_checker
 import oracle
 from gpu_util import assert_gemm_close, to_dev
 from paper_2605_09825_b200 import api, synth
@@ -24,17 +29,41 @@ def _rows(M, seed, stride=128):
     return np.unique(np.concatenate([np.array(fixed), per_slab])).astype(np.int64)
 
 
+ALPHA = {0: 1.0, 1: 1.0 / 32, 2: 1.0 / 32, 3: 1.0 / 16, 4: 1.0 / 16}     # exact factor that undoes H H^T = n I
+AXES = ((1, 1), (1, 0), (0, 0))                                          # operand orientation per pass (Appendix C)
+
+
+def _check_output(out, pass_, a_bits, b_bits, hmode, rnd, seed, what, rows_seed):
+    """`out` (CUDA tensor, whole GEMM result of the product path) against the oracle on sampled
+    rows and against the fp64 checker on every element."""
+    qa = oracle.quantize(a_bits, AXES[pass_][0], hmode, rnd, seed, 0)
+    qb = oracle.quantize(b_bits, AXES[pass_][1], hmode, rnd, seed, 1)
+    M = out.shape[0]
+    rows = _rows(M, rows_seed)
+    ref, S = oracle.gemm(*qa, *qb, alpha=ALPHA[hmode], rows=rows)
+    bf16 = out.dtype == torch.bfloat16
+    got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy()
+    assert_gemm_close(got, ref, S, bf16, what)
+    # the checker on the same rows of the oracle's operands: must reproduce the oracle (both sum
+    # exact block products in fp64; only the order of the last additions may differ)
+    _, _, _, cref, cS = gemm_checker.check(qa[0][rows], qa[1][rows], qb[0], qb[1], ALPHA[hmode], None, want_ref=True)
+    cref, cS = cref.cpu().numpy(), cS.cpu().numpy()
+    assert np.all(np.abs(cref - ref) <= 1e-12 * S + 1e-300), f"{what}: checker differs from the oracle"
+    assert np.all(np.abs(cS - S) <= 1e-12 * S + 1e-300), f"{what}: checker's tolerance base differs from the oracle's"
+    # every element of the product path's output against the checker
+    n_bad, first, worst, _, _ = gemm_checker.check(*qa, *qb, ALPHA[hmode], out)
+    assert n_bad == 0, (f"{what}: {n_bad} of {out.numel()} elements out of tolerance, first at "
+                        f"[{first // out.shape[1]}, {first % out.shape[1]}], worst error / tolerance {worst:.3g}")
+    assert worst <= 1.0
+
+
 def _check_pass(pass_, a_bits, b_bits, hmode, rnd, seed, what):
     a, b = to_dev(a_bits), to_dev(b_bits)
     fn = (api.linear_fprop, api.linear_dgrad, api.linear_wgrad)[pass_]
-    ofn = (oracle.linear_fprop, oracle.linear_dgrad, oracle.linear_wgrad)[pass_]
     out = fn(a, b, hmode, rnd, seed, api.OUT_BF16)
     api.check()
-    M = out.shape[0]
-    rows = _rows(M, 1234 + pass_)
-    ref, S = ofn(a_bits, b_bits, hmode, rnd, seed, rows=rows)
-    got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy()
-    assert_gemm_close(got, ref, S, True, what)
+    del a, b
+    _check_output(out, pass_, a_bits, b_bits, hmode, rnd, seed, what, 1234 + pass_)
     del out
 
 
@@ -86,13 +115,9 @@ def test_config5_layer_schedule_16384_tokens(name):
     Y, saved = api.linear_forward(X, W, 1, 0, 0)
     dX, dW = api.linear_backward(dY, saved, in_f, 1, 0, 0)
     api.check()
-    for out, ofn, a, b, what in ((Y, oracle.linear_fprop, t["X"], t["W"], "fprop"),
-                                 (dX, oracle.linear_dgrad, t["dY"], t["W"], "dgrad"),
-                                 (dW, oracle.linear_wgrad, t["dY"], t["X"], "wgrad")):
-        rows = _rows(out.shape[0], 4321)
-        ref, S = ofn(a, b, 1, 0, 0, rows=rows)
-        got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy()
-        assert_gemm_close(got, ref, S, True, f"config 5 {name} layer schedule {what}")
+    for out, pass_, a, b, what in ((Y, 0, t["X"], t["W"], "fprop"), (dX, 1, t["dY"], t["W"], "dgrad"),
+                                   (dW, 2, t["dY"], t["X"], "wgrad")):
+        _check_output(out, pass_, a, b, 1, 0, 0, f"config 5 {name} layer schedule {what}", 4321)
     if name == "o":
         raw = saved.cpu().numpy()
         r256 = lambda n: (n + 255) // 256 * 256
@@ -137,12 +162,8 @@ def test_eight_times_the_benchmark_token_count():
     Y, saved = api.linear_forward(X, W, 1, 0, 0)
     dX, dW = api.linear_backward(dY, saved, in_f, 1, 0, 0, api.OUT_BF16, api.OUT_FP32)
     api.check()
-    rows = _rows(T, 99)
-    ref, S = oracle.linear_fprop(Xb, Wb, 1, 0, 0, rows=rows)
-    assert_gemm_close(Y[torch.from_numpy(rows).cuda()].float().cpu().numpy(), ref, S, True, "fprop at 131072 tokens")
-    rows = _rows(out_f, 98)
-    ref, S = oracle.linear_wgrad(dYb, Xb, 1, 0, 0, rows=rows)
-    assert_gemm_close(dW[torch.from_numpy(rows).cuda()].cpu().numpy(), ref, S, False, "wgrad over 131072 tokens")
+    _check_output(Y, 0, Xb, Wb, 1, 0, 0, "fprop at 131072 tokens", 99)
+    _check_output(dW, 2, dYb, Xb, 1, 0, 0, "wgrad over 131072 tokens", 98)
 
 
 @pytest.mark.parametrize("hmode,rnd", [(1, 0), (2, 0), (0, 1)])
