@@ -51,6 +51,8 @@ extern "C" {
 #define MXFP4_ERR_TIMEOUT (-7)   /* a bounded device-side wait expired (reported by check)    */
 #define MXFP4_ERR_DEVICE (-8)    /* not an sm_100 device                                      */
 #define MXFP4_ERR_STATIC_LIMIT (-9) /* mxfp4_linear_static: problem exceeds the built-in scratch */
+#define MXFP4_ERR_BOUNDS (-10)   /* bounds-checking debug build only: a kernel computed an address outside
+                                    its buffer (reported by check; the access was skipped)              */
 
 /* enums (plain ints in the ABI) */
 #define MXFP4_AXIS_ROWS 0 /* 32-blocks run down the rows (column-wise 32x1); operand = src^T */
@@ -378,6 +380,19 @@ int mxfp4_check(void* stream);
  * or hangs -- so the next mxfp4_check(stream) returns MXFP4_ERR_TIMEOUT (and clears it).
  */
 int mxfp4_selftest_wait_timeout(void* stream);
+
+/*
+ * The library can be built with -DMXFP4_BOUNDS (no counterpart in the paper): a debug build that
+ * stands in for a memory sanitizer.  Every shared-memory access whose address a kernel computes is
+ * then checked against the buffer it belongs to (range and natural alignment); a miss is skipped
+ * and recorded, and the next mxfp4_check returns MXFP4_ERR_BOUNDS.  Results are bit-identical to
+ * the normal build.  mxfp4_bounds_checked() tells which build is loaded (1 / 0);
+ * mxfp4_selftest_bounds enqueues a one-thread kernel that hands the checker an address one
+ * element past a buffer -- the address is only tested, never dereferenced, in either build -- so
+ * that the next mxfp4_check(stream) returns MXFP4_ERR_BOUNDS (and clears it).
+ */
+int mxfp4_bounds_checked(void);
+int mxfp4_selftest_bounds(void* stream);
 
 #ifdef __cplusplus
 }

@@ -29,7 +29,7 @@ EXPORTS = (
     "mxfp4_linear_dgrad", "mxfp4_linear_wgrad", "mxfp4_linear_layer_bytes", "mxfp4_linear_forward",
     "mxfp4_linear_backward", "mxfp4_linear_layer_host", "mxfp4_linear_layer_host_drain", "mxfp4_quantize_fp8", "mxfp4_gemm_fp8",
     "mxfp4_linear_pass_workspace_bytes", "mxfp4_linear_pass", "mxfp4_linear_host", "mxfp4_linear_static",
-    "mxfp4_check", "mxfp4_selftest_wait_timeout",
+    "mxfp4_check", "mxfp4_selftest_wait_timeout", "mxfp4_bounds_checked", "mxfp4_selftest_bounds",
 )
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
@@ -111,6 +111,8 @@ def load_library() -> ctypes.CDLL:
     lib.mxfp4_linear_static.restype = ci
     lib.mxfp4_check.argtypes, lib.mxfp4_check.restype = [vp], ci
     lib.mxfp4_selftest_wait_timeout.argtypes, lib.mxfp4_selftest_wait_timeout.restype = [vp], ci
+    lib.mxfp4_selftest_bounds.argtypes, lib.mxfp4_selftest_bounds.restype = [vp], ci
+    lib.mxfp4_bounds_checked.argtypes, lib.mxfp4_bounds_checked.restype = [], ci
     _lib = lib
     return lib
 
@@ -474,6 +476,16 @@ def linear_static(pass_: int, a: torch.Tensor, b: torch.Tensor, T: int, in_f: in
                                             _stream())
     _raise(rc, "mxfp4_linear_static")
     return out
+
+
+def bounds_checked() -> bool:
+    """True when the loaded library is the bounds-checking debug build (``-DMXFP4_BOUNDS``)."""
+    return bool(load_library().mxfp4_bounds_checked())
+
+
+def selftest_bounds() -> None:
+    """``mxfp4_selftest_bounds``: the next :func:`check` raises with status -10 (and clears it)."""
+    _raise(load_library().mxfp4_selftest_bounds(_stream()), "mxfp4_selftest_bounds")
 
 
 def selftest_wait_timeout() -> None:

@@ -326,11 +326,12 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
             const uint32_t t = tmem + lane_base + kPTmemSfBase + s * kPTmemSfPerBuf;
             const uint8_t* sa = &sm.sfa[s][lane * 16];
             const uint8_t* sb = &sm.sfb[s][lane * 16];           // [row block nb][K-tile kt] at nb*1024 + kt*512
-            auto ld = [](const uint8_t* q) { return *reinterpret_cast<const uint4*>(q); };
-            tmem_st_32x32b_x8(t, ld(sa), ld(sa + 512));                       // SFA kt0 | kt1
-            tmem_st_32x32b_x8(t + 8, ld(sb), ld(sb + 1024));                  // SFB kt0: nb0 | nb1
-            tmem_st_32x32b_x8(t + 16, ld(sb + 2048), ld(sb + 512));           // SFB kt0: nb2 | kt1: nb0
-            tmem_st_32x32b_x8(t + 24, ld(sb + 1024 + 512), ld(sb + 2048 + 512));  // SFB kt1: nb1 | nb2
+            auto lda = [&](const uint8_t* q) { return smem_load<uint4>(q, sm.sfa[s], kPSfaBytes); };
+            auto ldb = [&](const uint8_t* q) { return smem_load<uint4>(q, sm.sfb[s], kPSfbBytes); };
+            tmem_st_32x32b_x8(t, lda(sa), lda(sa + 512));                       // SFA kt0 | kt1
+            tmem_st_32x32b_x8(t + 8, ldb(sb), ldb(sb + 1024));                  // SFB kt0: nb0 | nb1
+            tmem_st_32x32b_x8(t + 16, ldb(sb + 2048), ldb(sb + 512));           // SFB kt0: nb2 | kt1: nb0
+            tmem_st_32x32b_x8(t + 24, ldb(sb + 1024 + 512), ldb(sb + 2048 + 512));  // SFB kt1: nb1 | nb2
             tmem_st_wait();
             tcgen05_fence_before();
             __syncwarp();
@@ -376,10 +377,12 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
                         __syncwarp();
 #pragma unroll
                         for (int q = 0; q < 8; ++q)
-                            *reinterpret_cast<float4*>(stg + lane * 128 + ((q ^ (lane & 7)) * 16)) =
-                                make_float4(__uint_as_float(r[c][4 * q]) * p.alpha, __uint_as_float(r[c][4 * q + 1]) * p.alpha,
-                                            __uint_as_float(r[c][4 * q + 2]) * p.alpha,
-                                            __uint_as_float(r[c][4 * q + 3]) * p.alpha);
+                            smem_store(stg + lane * 128 + ((q ^ (lane & 7)) * 16),
+                                       make_float4(__uint_as_float(r[c][4 * q]) * p.alpha,
+                                                   __uint_as_float(r[c][4 * q + 1]) * p.alpha,
+                                                   __uint_as_float(r[c][4 * q + 2]) * p.alpha,
+                                                   __uint_as_float(r[c][4 * q + 3]) * p.alpha),
+                                       stg, 32 * 128);
                         fence_proxy_async_smem();
                         __syncwarp();
                         if (p.n_tma < p.N) {
@@ -388,7 +391,7 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
                             const int64_t rc = p.n_tma - col0;
                             if (rc >= 0 && rc < 32 && row < p.M) {
                                 const int q = static_cast<int>(rc >> 2);
-                                const float4 v = *reinterpret_cast<const float4*>(stg + lane * 128 + ((q ^ (lane & 7)) * 16));
+                                const float4 v = smem_load<float4>(stg + lane * 128 + ((q ^ (lane & 7)) * 16), stg, 32 * 128);
                                 const float e[4] = {v.x, v.y, v.z, v.w};
                                 float* dst = static_cast<float*>(p.out) + row * p.ld_out + p.n_tma;
                                 for (int k = 0; k < 3; ++k)
@@ -436,9 +439,10 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
                     __syncwarp();
 #pragma unroll
                     for (int q = 0; q < 8; ++q)
-                        *reinterpret_cast<uint4*>(stg + lane * 128 + ((q ^ (lane & 7)) * 16)) =
-                            make_uint4(w[c * 32 + q * 4], w[c * 32 + q * 4 + 1], w[c * 32 + q * 4 + 2],
-                                       w[c * 32 + q * 4 + 3]);
+                        smem_store(stg + lane * 128 + ((q ^ (lane & 7)) * 16),
+                                   make_uint4(w[c * 32 + q * 4], w[c * 32 + q * 4 + 1], w[c * 32 + q * 4 + 2],
+                                              w[c * 32 + q * 4 + 3]),
+                                   stg, 32 * 128);
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (p.n_tma < p.N) {
@@ -449,7 +453,7 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
                         const int64_t row = row0 + lane;
                         if (rc >= 0 && rc < 64 && row < p.M) {
                             const int q = static_cast<int>(rc >> 3);
-                            const uint4 v = *reinterpret_cast<const uint4*>(stg + lane * 128 + ((q ^ (lane & 7)) * 16));
+                            const uint4 v = smem_load<uint4>(stg + lane * 128 + ((q ^ (lane & 7)) * 16), stg, 32 * 128);
                             const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
                             __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.out) + row * p.ld_out + p.n_tma;
                             for (int k = 0; k < 8; ++k)

@@ -267,6 +267,15 @@ __global__ void selftest_wait_timeout_kernel()
     mbar_wait(&bar, 0, &abort_flag, 256u);
 }
 
+// Self-test of the bounds discipline: the checker is handed an address one element past a
+// shared array.  It refuses (the store never happens) and records the status.
+__global__ void selftest_bounds_kernel()
+{
+    __shared__ uint32_t buf[8];
+    uint32_t* past = buf + 8;
+    if (bounds_ok(past, sizeof(uint32_t), buf, sizeof(buf))) *past = 1u;
+}
+
 }  // namespace mxfp4
 
 using namespace mxfp4;
@@ -309,6 +318,7 @@ const char* mxfp4_status_string(int status)
         case MXFP4_ERR_TIMEOUT: return "device-side wait timed out";
         case MXFP4_ERR_DEVICE: return "not an sm_100 device";
         case MXFP4_ERR_STATIC_LIMIT: return "problem needs more scratch than the built-in array holds";
+        case MXFP4_ERR_BOUNDS: return "a kernel computed an address outside its buffer (debug build)";
         default: return "unknown status";
     }
 }
@@ -929,6 +939,24 @@ int mxfp4_selftest_wait_timeout(void* stream)
     if (!dev.ok) return MXFP4_ERR_CUDA;
     if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
     selftest_wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>();
+    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+int mxfp4_bounds_checked(void)
+{
+#ifdef MXFP4_BOUNDS
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int mxfp4_selftest_bounds(void* stream)
+{
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return MXFP4_ERR_CUDA;
+    if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
+    selftest_bounds_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>();
     return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 

@@ -14,6 +14,39 @@ namespace mxfp4 {
 __device__ int g_device_status = 0;
 
 constexpr int kDevErrTimeout = -7;
+constexpr int kDevErrBounds = -10;
+
+// Bounds discipline of the debug build (-DMXFP4_BOUNDS), the stand-in for a memory sanitizer: every
+// access whose address a kernel COMPUTES (shared-memory stages, staging tiles, scale tiles) goes
+// through smem_load / smem_store, which in that build check that the address lies inside the
+// buffer it was derived from and is naturally aligned; a miss records kDevErrBounds in the status
+// word and the access is skipped (a load returns zeros) -- nothing traps.  In the normal build the
+// helpers are plain loads and stores.
+__device__ __forceinline__ bool bounds_ok(const void* p, size_t bytes, const void* base, size_t size)
+{
+    const uintptr_t a = reinterpret_cast<uintptr_t>(p), b = reinterpret_cast<uintptr_t>(base);
+    if (a >= b && a + bytes <= b + size && a % bytes == 0) return true;
+    atomicCAS(&g_device_status, 0, kDevErrBounds);
+    return false;
+}
+
+template <class T>
+__device__ __forceinline__ T smem_load(const void* p, const void* base, size_t size)
+{
+#ifdef MXFP4_BOUNDS
+    if (!bounds_ok(p, sizeof(T), base, size)) return T{};
+#endif
+    return *static_cast<const T*>(p);
+}
+
+template <class T>
+__device__ __forceinline__ void smem_store(void* p, const T& v, const void* base, size_t size)
+{
+#ifdef MXFP4_BOUNDS
+    if (!bounds_ok(p, sizeof(T), base, size)) return;
+#endif
+    *static_cast<T*>(p) = v;
+}
 
 // Spin limit for one wait.  A try_wait suspends for a hardware-defined slice, so this many
 // attempts is on the order of a second -- far longer than any legitimate wait here.

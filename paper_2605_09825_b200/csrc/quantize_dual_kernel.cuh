@@ -65,8 +65,8 @@ __device__ __forceinline__ void load_column_blocks(const uint8_t* stage, int kb,
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
         const int r0 = 2 * i, r1 = 2 * i + 1;               // rows of the block; (kb*32 + r) % 8 == r % 8
-        uint32_t w0 = *reinterpret_cast<const uint32_t*>(stage + ((base ^ ((r0 & 7) << 4)) + r0 * 128));
-        uint32_t w1 = *reinterpret_cast<const uint32_t*>(stage + ((base ^ ((r1 & 7) << 4)) + r1 * 128));
+        uint32_t w0 = smem_load<uint32_t>(stage + ((base ^ ((r0 & 7) << 4)) + r0 * 128), stage, kQStageBytes);
+        uint32_t w1 = smem_load<uint32_t>(stage + ((base ^ ((r1 & 7) << 4)) + r1 * 128), stage, kQStageBytes);
         if (HMODE == 2 || HMODE == 4) {                     // element r of both columns shares its sign
             w0 ^= sg.word[r0];
             w1 ^= sg.word[r1];
@@ -87,10 +87,11 @@ __device__ __forceinline__ void stage_block(uint8_t* code_tile, uint8_t* scale_t
                                             int kb, int to, int tk, const uint32_t (&packed)[4], uint32_t byte,
                                             bool ok)
 {
-    *reinterpret_cast<uint4*>(code_tile + o * 64 + ((kb ^ ((o >> 1) & 3)) * 16)) =
-        make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    smem_store(code_tile + o * 64 + ((kb ^ ((o >> 1) & 3)) * 16), make_uint4(packed[0], packed[1], packed[2], packed[3]),
+               code_tile, kQCodeTileBytes);
     if (p.scale_layout == 1) {
-        scale_tile[(o & 31) * 16 + (o >> 5) * 4 + kb] = static_cast<uint8_t>(byte);
+        smem_store(scale_tile + (o & 31) * 16 + (o >> 5) * 4 + kb, static_cast<uint8_t>(byte), scale_tile,
+                   kQScaleTileBytes);
     } else if (ok) {
         const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
         const int64_t tg = static_cast<int64_t>(tk) * 4 + kb;

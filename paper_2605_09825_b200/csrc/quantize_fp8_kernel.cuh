@@ -82,14 +82,15 @@ __device__ __forceinline__ bool consume_tile_fp8(QuantFp8Smem& sm, const QuantPa
     // codes: row o of the tile is 128 bytes = 8 chunks of 16, chunk c stored at c ^ (o % 8)
     uint8_t* ct = &sm.code_tile[grp][buf][o * 128];
     const int sw = o & 7;
-    *reinterpret_cast<uint4*>(ct + (((2 * kbh) ^ sw) * 16)) = make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]);
-    *reinterpret_cast<uint4*>(ct + (((2 * kbh + 1) ^ sw) * 16)) = make_uint4(packed0[4], packed0[5], packed0[6], packed0[7]);
-    *reinterpret_cast<uint4*>(ct + (((2 * kbh + 4) ^ sw) * 16)) = make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]);
-    *reinterpret_cast<uint4*>(ct + (((2 * kbh + 5) ^ sw) * 16)) = make_uint4(packed1[4], packed1[5], packed1[6], packed1[7]);
+    const void* ctb = sm.code_tile[grp][buf];
+    smem_store(ct + (((2 * kbh) ^ sw) * 16), make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]), ctb, 128 * 128);
+    smem_store(ct + (((2 * kbh + 1) ^ sw) * 16), make_uint4(packed0[4], packed0[5], packed0[6], packed0[7]), ctb, 128 * 128);
+    smem_store(ct + (((2 * kbh + 4) ^ sw) * 16), make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]), ctb, 128 * 128);
+    smem_store(ct + (((2 * kbh + 5) ^ sw) * 16), make_uint4(packed1[4], packed1[5], packed1[6], packed1[7]), ctb, 128 * 128);
     if (p.scale_layout == 1) {
         uint8_t* st = &sm.scale_tile[grp][buf][(o & 31) * 16 + (o >> 5) * 4];
-        st[kbh] = static_cast<uint8_t>(byte0);
-        st[kbh + 2] = static_cast<uint8_t>(byte1);
+        smem_store(st + kbh, static_cast<uint8_t>(byte0), sm.scale_tile[grp][buf], kQScaleTileBytes);
+        smem_store(st + kbh + 2, static_cast<uint8_t>(byte1), sm.scale_tile[grp][buf], kQScaleTileBytes);
     } else if (ok) {
         const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
         const int64_t tg = static_cast<int64_t>(tk) * 4 + kbh;

@@ -175,7 +175,7 @@ __device__ __forceinline__ void load_block(const uint8_t* stage, int kb, int o, 
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int chunk = (((kb & 1) * 4 + j) ^ (o & 7)) * 16;
-            const uint4 q = *reinterpret_cast<const uint4*>(base + chunk);
+            const uint4 q = smem_load<uint4>(base + chunk, stage, kQStageBytes);
             const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -189,7 +189,8 @@ __device__ __forceinline__ void load_block(const uint8_t* stage, int kb, int o, 
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
             // zero-extended elements; the flip word's upper half falls off in the shift / the 16-bit operand
-            uint32_t a = base[(2 * i) * 128], b = base[(2 * i + 1) * 128];
+            uint32_t a = smem_load<uint16_t>(base + (2 * i) * 128, stage, kQStageBytes);
+            uint32_t b = smem_load<uint16_t>(base + (2 * i + 1) * 128, stage, kQStageBytes);
             if (kRand) {
                 a ^= sg.word[2 * i];
                 b ^= sg.word[2 * i + 1];
@@ -364,14 +365,14 @@ __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p
 
         // stage the results: codes in the 64-byte swizzle the TMA store expects
         uint8_t* ct = &sm.code_tile[slot][o * 64];
-        *reinterpret_cast<uint4*>(ct + ((kbh ^ ((o >> 1) & 3)) * 16)) =
-            make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]);
-        *reinterpret_cast<uint4*>(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16)) =
-            make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]);
+        smem_store(ct + ((kbh ^ ((o >> 1) & 3)) * 16), make_uint4(packed0[0], packed0[1], packed0[2], packed0[3]),
+                   sm.code_tile[slot], kQCodeTileBytes);
+        smem_store(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16), make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]),
+                   sm.code_tile[slot], kQCodeTileBytes);
         if (p.scale_layout == 1) {
             uint8_t* st = &sm.scale_tile[slot][(o & 31) * 16 + (o >> 5) * 4];
-            st[kbh] = static_cast<uint8_t>(byte0);
-            st[kbh + 2] = static_cast<uint8_t>(byte1);
+            smem_store(st + kbh, static_cast<uint8_t>(byte0), sm.scale_tile[slot], kQScaleTileBytes);
+            smem_store(st + kbh + 2, static_cast<uint8_t>(byte1), sm.scale_tile[slot], kQScaleTileBytes);
         } else if (ok) {
             const int64_t og = static_cast<int64_t>(to) * kQTileO + o;
             const int64_t tg = static_cast<int64_t>(tk) * 4 + kbh;
