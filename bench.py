@@ -516,6 +516,28 @@ def run_ours(args):
         del flush
         api.check()
 
+    # ---- ceiling of the tensor pipe itself on this device, in this run: the GEMM's own pair MMAs on
+    # operands that stay in shared memory (no loads, no epilogue), constant and random operand bits
+    mma_only = None
+    if not args.no_mma_probe:
+        def mma_rate(random_operands, launches):
+            api.probe_mma_rate(10000, random_operands)
+            torch.cuda.synchronize()
+            m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            m0.record(stream)
+            fl = 0.0
+            for _ in range(launches):
+                fl += api.probe_mma_rate(10000, random_operands)
+            m1.record(stream)
+            torch.cuda.synchronize()
+            return fl / (m0.elapsed_time(m1) * 1e-3) / 1e12
+        mma_only = {"constant_operands_tflops": mma_rate(False, 10), "random_operands_burst_tflops": mma_rate(True, 5),
+                    "random_operands_sustained_tflops": mma_rate(True, 60),
+                    "note": "mxfp4_probe_mma_rate: 256x192x64 pair MMAs, eight per iteration as in one K-step of the "
+                            "GEMM, operands resident in shared memory; 10 / 5 / 60 launches of ~5 ms; with random "
+                            "operand bits the tensor pipe alone reaches the power limit"}
+        api.check()
+
     fp8_info = None
     if ladder:
         f8_ms = sum(a0.elapsed_time(a1) for a0, a1, _ in fp8_evs)
@@ -549,12 +571,14 @@ def run_ours(args):
         # ncu, one launch of the 8192 x 6144 x 4096 GEMM (QKV Fprop at 8192 tokens; profiles/): DRAM
         # bytes of THAT launch, not scaled to this step's shapes (operands are re-read from L2 and
         # part of the output is still in L2 at kernel end, so traffic does not follow the flops)
-        "traffic": 81.3e6,
+        "traffic": 78.6e6,
         "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one captured 8192x6144x4096 launch "
                         "(algorithmic bytes of that launch 130.1e6); not scaled to the 12 shapes of this step",
         "flops_per_launch": gemm_flops / n_gemm, "avg_launch_ms": gemm_ms / n_gemm,
         "launch_timing": f"median of {n_dec - 1} repetitions per launch, CUDA events on the launching stream",
         "tflops_by_launch": gemm_by_shape,
+        "mma_only_ceiling": mma_only,
+        "frac_of_mma_only_random_sustained": (gemm_tflops / mma_only["random_operands_sustained_tflops"]) if mma_only else None,
         "fused_path": {"tflops": step_tflops, "frac_of_nominal_fp4": step_tflops / 9000.0,
                        "frac_of_4x_burst_bf16": step_tflops / fp4_peak,
                        "frac_of_4x_sustained_bf16": step_tflops / fp4_peak_sustained,
@@ -765,6 +789,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the per-variant quantize table")
+    ap.add_argument("--no-mma-probe", action="store_true", help="skip the shared-memory-resident MMA ceiling")
     ap.add_argument("--decomposed-reps", type=int, default=20,
                     help="repetitions of the per-launch timed step (medians feed the roofline)")
     args = ap.parse_args()

@@ -394,6 +394,18 @@ int mxfp4_selftest_wait_timeout(void* stream);
 int mxfp4_bounds_checked(void);
 int mxfp4_selftest_bounds(void* stream);
 
+/*
+ * Diagnostic (no counterpart in the paper): enqueues one launch of a kernel that issues the GEMM's
+ * own pair MMAs (256 x 192 x 64, kind::mxf4.block_scale, eight per iteration = one K-step) on
+ * operands resident in shared memory -- no loads, no epilogue -- on every CTA pair of the device.
+ * Timed by the caller (CUDA events around a few launches) it gives the ceiling the tensor pipe
+ * sets for MXFP4 on this device: with constant operand bits the clock-bound rate, with
+ * random_operands != 0 the rate the power limit allows once operands toggle.  *flops (host, may
+ * be NULL) receives the floating-point operations of the launch.  iterations: 1..20000 (a launch
+ * of 10000 takes about 5 ms).  Every wait inside is bounded.
+ */
+int mxfp4_probe_mma_rate(int iterations, int random_operands, void* stream, double* flops);
+
 #ifdef __cplusplus
 }
 #endif

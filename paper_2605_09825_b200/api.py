@@ -30,6 +30,7 @@ EXPORTS = (
     "mxfp4_linear_backward", "mxfp4_linear_layer_host", "mxfp4_linear_layer_host_drain", "mxfp4_quantize_fp8", "mxfp4_gemm_fp8",
     "mxfp4_linear_pass_workspace_bytes", "mxfp4_linear_pass", "mxfp4_linear_host", "mxfp4_linear_static",
     "mxfp4_check", "mxfp4_selftest_wait_timeout", "mxfp4_bounds_checked", "mxfp4_selftest_bounds",
+    "mxfp4_probe_mma_rate",
 )
 STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
 
@@ -113,6 +114,8 @@ def load_library() -> ctypes.CDLL:
     lib.mxfp4_selftest_wait_timeout.argtypes, lib.mxfp4_selftest_wait_timeout.restype = [vp], ci
     lib.mxfp4_selftest_bounds.argtypes, lib.mxfp4_selftest_bounds.restype = [vp], ci
     lib.mxfp4_bounds_checked.argtypes, lib.mxfp4_bounds_checked.restype = [], ci
+    lib.mxfp4_probe_mma_rate.argtypes = [ci, ci, vp, ctypes.POINTER(ctypes.c_double)]
+    lib.mxfp4_probe_mma_rate.restype = ci
     _lib = lib
     return lib
 
@@ -476,6 +479,15 @@ def linear_static(pass_: int, a: torch.Tensor, b: torch.Tensor, T: int, in_f: in
                                             _stream())
     _raise(rc, "mxfp4_linear_static")
     return out
+
+
+def probe_mma_rate(iterations: int = 10000, random_operands: bool = True) -> float:
+    """``mxfp4_probe_mma_rate``: enqueue one launch of the shared-memory-resident MMA loop on the
+    current stream; returns the floating-point operations it performs (time it with CUDA events)."""
+    fl = ctypes.c_double(0.0)
+    _raise(load_library().mxfp4_probe_mma_rate(iterations, int(random_operands), _stream(), ctypes.byref(fl)),
+           "mxfp4_probe_mma_rate")
+    return fl.value
 
 
 def bounds_checked() -> bool:

@@ -15,6 +15,7 @@
 #include "quantize_dual_kernel.cuh"
 #include "quantize_fp8_kernel.cuh"
 #include "gemm_pair_kernel.cuh"
+#include "mma_rate_probe.cuh"
 
 namespace mxfp4 {
 
@@ -940,6 +941,24 @@ int mxfp4_selftest_wait_timeout(void* stream)
     if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
     selftest_wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>();
     return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+int mxfp4_probe_mma_rate(int iterations, int random_operands, void* stream, double* flops)
+{
+    if (iterations <= 0 || iterations > 20000) return MXFP4_ERR_SHAPE;   // a launch stays within ~10 ms
+    const DeviceInfo& dev = device_info();
+    if (!dev.ok) return MXFP4_ERR_CUDA;
+    if (dev.cc_major != 10) return MXFP4_ERR_DEVICE;
+    const size_t smem = sizeof(MmaProbeSmem) + 1024;
+    static PerDeviceOnce once;
+    const int rc = ensure_smem_attribute(once, mma_rate_probe_kernel, smem);
+    if (rc != MXFP4_OK) return rc;
+    const int clusters = dev.sm_count / 2;
+    mma_rate_probe_kernel<<<2 * clusters, kMmaProbeThreads, smem, static_cast<cudaStream_t>(stream)>>>(
+        iterations, random_operands ? 1 : 0);
+    if (cudaGetLastError() != cudaSuccess) return MXFP4_ERR_CUDA;
+    if (flops) *flops = 2.0 * kPTileM * kPMmaN * 64.0 * 8.0 * iterations * clusters;
+    return MXFP4_OK;
 }
 
 int mxfp4_bounds_checked(void)

@@ -187,3 +187,15 @@ def test_plain_stream_order_launches_still_work():
     res = subprocess.run([sys.executable, "-c", "import __graft_entry__ as g; g.smoke()"], cwd=root,
                          env=dict(os.environ, MXFP4_PDL="0"), capture_output=True, text=True, timeout=600)
     assert res.returncode == 0, res.stdout + res.stderr
+
+
+def test_mma_rate_probe_runs_and_reports_its_flops():
+    """The diagnostic that measures the tensor pipe's own ceiling: a short launch completes, leaves
+    the status word clean and reports 2 * 256 * 192 * 64 * 8 flops per iteration and CTA pair."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for rnd in (False, True):
+        fl = api.probe_mma_rate(200, rnd)
+        api.check()
+        assert fl == 2.0 * 256 * 192 * 64 * 8 * 200 * (sms // 2)
+    with pytest.raises(api.Mxfp4Error):
+        api.probe_mma_rate(0, True)
