@@ -142,8 +142,10 @@ static void fill_quant_params(QuantParams* pp, int64_t outer, int64_t K, int had
     p.nt = K / 32;
     p.tiles_o = static_cast<int32_t>((outer + kQTileO - 1) / kQTileO);
     p.tiles_k = static_cast<int32_t>((K + kQTileK - 1) / kQTileK);
-    p.seed_lo = static_cast<uint32_t>(seed);
-    p.seed_hi = static_cast<uint32_t>(seed >> 32);
+    for (int r = 0; r < 10; ++r) {          // key schedule of Philox4x32-10: key + r * Weyl constant
+        p.rk.k0[r] = static_cast<uint32_t>(seed) + static_cast<uint32_t>(r) * 0x9E3779B9u;
+        p.rk.k1[r] = static_cast<uint32_t>(seed >> 32) + static_cast<uint32_t>(r) * 0xBB67AE85u;
+    }
     p.tag = operand_tag;
     p.sign_mask = 0u;
     if (hadamard_mode == MXFP4_HADAMARD_RAND) p.sign_mask = host_sign_mask(seed);

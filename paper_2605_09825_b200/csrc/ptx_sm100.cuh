@@ -313,21 +313,42 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
 
 // ---------------------------------------------------------------- Philox4x32-10
 // Counter-based generator of the stochastic-rounding variant: same inputs, same outputs on
-// any thread, so the stream is a pure function of (seed, counter).
+// any thread, so the stream is a pure function of (seed, counter).  The ten round keys
+// (key + r * Weyl constant, the published key schedule) depend on the seed only, so the host
+// computes them once per call and the kernel reads them as constant-bank operands of the XORs;
+// each round is then two 32 x 32 -> 64-bit multiplies and two three-input XORs.
+struct PhiloxRoundKeys {
+    uint32_t k0[10], k1[10];
+};
+
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              uint32_t k0, uint32_t k1, uint32_t (&out)[4])
+                                              const PhiloxRoundKeys& rk, uint32_t (&out)[4])
 {
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-        const uint32_t n0 = hi1 ^ c1 ^ k0;
-        const uint32_t n2 = hi0 ^ c3 ^ k1;
-        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-        k0 += 0x9E3779B9u;
-        k1 += 0xBB67AE85u;
+        const uint64_t p0 = static_cast<uint64_t>(0xD2511F53u) * c0;
+        const uint64_t p1 = static_cast<uint64_t>(0xCD9E8D57u) * c2;
+        const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ rk.k0[r];
+        const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ rk.k1[r];
+        c0 = n0; c1 = static_cast<uint32_t>(p1); c2 = n2; c3 = static_cast<uint32_t>(p0);
     }
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// byte permute: byte i of the result is byte (selector nibble i) of the eight bytes {a, b}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t selector)
+{
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(selector));
+    return r;
+}
+
+// minimum of the two unsigned 16-bit halves
+__device__ __forceinline__ uint32_t min_u16x2(uint32_t a, uint32_t b)
+{
+    uint32_t r;
+    asm("min.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
 }
 
 }  // namespace mxfp4

@@ -61,7 +61,8 @@ struct QuantParams {
     int64_t outer, K;        // operand view
     int64_t nt;              // K / 32
     int32_t tiles_o, tiles_k;
-    uint32_t seed_lo, seed_hi, tag, sign_mask;
+    PhiloxRoundKeys rk;      // round keys of the stochastic-rounding stream (from the seed)
+    uint32_t tag, sign_mask;
     int32_t scale_layout;    // 0 canonical, 1 tiled
     int32_t block2d;         // 0: 1 x 32 blocks, 1: 32 x 32 blocks (scale shared by 32 operand rows)
 };
@@ -137,16 +138,29 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(float v0, float v1, float v2, flo
     return r;
 }
 
-// Stochastic rounding of one scaled value with 8 random bits.  |s| * 2^-126 re-biases the value
-// so that bits 22.. of its fp32 pattern are the E2M1 magnitude code below it and bits 0..21 the
-// position between the two neighbouring grid points; rounding the product toward +inf keeps
-// every strict comparison against the (integer) thresholds intact.
-__device__ __forceinline__ uint32_t sr_e2m1(float s, uint32_t u8)
+// Stochastic rounding (8 random bits per element, round up iff (u8 + 1/2) / 256 < frac) of two
+// scaled values at a time.  |s| * 2^-126 re-biases a value so that bits 22.. of its fp32 pattern
+// are the E2M1 magnitude code below it and bits 0..21 the position x between the two neighbouring
+// grid points (the product is rounded toward +inf, so nothing below the pattern's last bit is
+// lost to the strict comparison).  The rule compares x with T = (2 u8 + 1) * 2^13, and
+// x > T  <=>  ceil(x / 2^13) > 2 u8 + 1, so a 13-bit number y = ceil(pattern / 2^13) = code * 512 +
+// position-in-512ths carries everything the decision needs: the rounded code is
+// (y + 510 - 2 u8) >> 9.  Two such numbers fit the halves of one register: z = 8 * pattern +
+// 0x01FEFFF8 has y + 510 in its upper half, one byte permute packs the upper halves of two z,
+// one multiply-add subtracts twice the two random bytes (spread to the halves by another
+// permute; no borrow crosses the halves because y + 510 >= 2 u8), and shift, mask and a
+// two-way minimum with 7 (values in [6, 8) may step to 8) give both codes.  Returns the codes in
+// bits 0..3 and 16..19, sign bits included; `rbytes` holds the two random bytes in its bytes 0 and 2.
+__device__ __forceinline__ uint32_t sr_e2m1_pair(float sa, float sb, uint32_t rbytes)
 {
-    const float a = fminf(fabsf(s), 6.0f);
-    const uint32_t bits = __float_as_uint(__fmul_ru(a, 1.1754943508222875e-38f));
-    const uint32_t r = bits + (0x3FFFFFu - ((2u * u8 + 1u) << 13));
-    return (r >> 22) | ((__float_as_uint(s) >> 28) & 8u);
+    const uint32_t za = __float_as_uint(__fmul_ru(fabsf(sa), 1.1754943508222875e-38f)) * 8u + 0x01FEFFF8u;
+    const uint32_t zb = __float_as_uint(__fmul_ru(fabsf(sb), 1.1754943508222875e-38f)) * 8u + 0x01FEFFF8u;
+    const uint32_t y2 = prmt(za, zb, 0x7632u);                       // (y_b + 510) << 16 | (y_a + 510)
+    const uint32_t r2 = rbytes * 0xFFFFFFFEu + y2;                    // minus 2 u8 in each half
+    const uint32_t mag = min_u16x2((r2 >> 9) & 0x000F000Fu, 0x00070007u);
+    // bytes 0 and 2 = the top bytes of sa and sb with their sign bit replicated (selector nibble 8 | index)
+    const uint32_t sg = prmt(__float_as_uint(sa), __float_as_uint(sb), 0xFFBBu);
+    return mag | (sg & 0x00080008u);
 }
 
 // h = 1 butterfly of the deterministic rotation straight from bf16: (a + b, a - b) with a the
@@ -252,18 +266,23 @@ __device__ __forceinline__ void scale_round_pack(const float2 (&P)[16], float am
         for (int half = 0; half < 2; ++half) {
             uint32_t r[4];
             const uint64_t gg = g + half;
-            philox4x32_10(static_cast<uint32_t>(gg), static_cast<uint32_t>(gg >> 32), p.tag, 0u, p.seed_lo,
-                          p.seed_hi, r);
+            philox4x32_10(static_cast<uint32_t>(gg), static_cast<uint32_t>(gg >> 32), p.tag, 0u, p.rk, r);
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
-                uint32_t w = 0;
+                // eight elements = four pairs -> one word of packed codes; element e of the 16-group
+                // draws byte (e & 3) of word (e >> 2): pair j of this word uses bytes 0, 1 or 2, 3 of
+                // word 2q + j / 2
+                uint32_t c2[4];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int e = q * 8 + i;                   // element in the 16-group
-                    const uint32_t u8 = (r[e >> 2] >> (8 * (e & 3))) & 0xFFu;
-                    w |= sr_e2m1(v[half * 16 + e], u8) << (4 * i);
+                for (int j = 0; j < 4; ++j) {
+                    const int e = q * 8 + 2 * j;             // even element of the pair in the 16-group
+                    const uint32_t rb = prmt(r[e >> 2], 0u, (j & 1) ? 0x4342u : 0x4140u);   // [u8_a, 0, u8_b, 0]
+                    c2[j] = sr_e2m1_pair(v[half * 16 + e], v[half * 16 + e + 1], rb);
                 }
-                packed[half * 2 + q] = w;
+                // bytes: codes of the even elements in the lower halves, of the odd ones in the upper
+                const uint32_t u01 = c2[1] * 256u + c2[0], u23 = c2[3] * 256u + c2[2];
+                const uint32_t even4 = prmt(u01, u23, 0x5410u), odd4 = prmt(u01, u23, 0x7632u);
+                packed[half * 2 + q] = odd4 * 16u + even4;   // element k even in the low nibble
             }
         }
     }
