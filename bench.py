@@ -538,6 +538,49 @@ def run_ours(args):
                             "operand bits the tensor pipe alone reaches the power limit"}
         api.check()
 
+    # ---- the GEMM kernel's own steady state: 148 tiles of K = 65536 (tile switches, epilogue and partial
+    # waves negligible), quantized-activation-like codes.  It does not depend on the operand bits (constant
+    # bits give the same rate), i.e. it is the L2 -> shared-memory operand feed, not power, that sets it;
+    # bytes moved per K-step of a CTA pair: codes 2 x (16 + 24) KB + scale tiles 2 x (1 + 3) KB.
+    l2_feed = None
+    if not args.no_mma_probe and not ladder:
+        Ms, Ns, Ks = 1024, 37 * 384, 65536
+        gen = torch.Generator(device="cuda").manual_seed(11)
+
+        def like_codes(rows):
+            mag = torch.clamp((torch.randn(rows, Ks, device="cuda", generator=gen).abs() * 2.0).round(), 0, 7).to(torch.uint8)
+            sgn = (torch.rand(rows, Ks, device="cuda", generator=gen) < 0.5).to(torch.uint8) << 3
+            c = mag | sgn
+            return (c[:, 0::2] | (c[:, 1::2] << 4)).contiguous()
+
+        a_c, b_c = like_codes(Ms), like_codes(Ns)
+        a_s = torch.randint(124, 130, (api.scales_bytes(Ms, Ks),), dtype=torch.uint8, device="cuda", generator=gen)
+        b_s = torch.randint(124, 130, (api.scales_bytes(Ns, Ks),), dtype=torch.uint8, device="cuda", generator=gen)
+        o_s = torch.empty((Ms, Ns), dtype=torch.bfloat16, device="cuda")
+        for _ in range(3):
+            api.gemm(a_c, a_s, b_c, b_s, 1.0, api.OUT_BF16, out=o_s)
+        torch.cuda.synchronize()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        for _ in range(20):
+            api.gemm(a_c, a_s, b_c, b_s, 1.0, api.OUT_BF16, out=o_s)
+        s1.record(stream)
+        torch.cuda.synchronize()
+        steady = 2.0 * Ms * Ns * Ks * 20 / (s0.elapsed_time(s1) * 1e-3) / 1e12
+        del a_c, b_c, a_s, b_s, o_s
+        pair_kstep_bytes = 2 * (16384 + 24576) + 2 * (1024 + 3072)
+        pair_kstep_flops = 2.0 * 256 * 384 * 256
+        feed_peak = steady * 1e12 * pair_kstep_bytes / pair_kstep_flops / 1e12          # TB/s at the steady state
+        step_bytes = 0.0
+        for (_, _, _, _, M, N, K) in passes:
+            tiles = ((M + 255) // 256) * ((N + 383) // 384)
+            step_bytes += tiles * ((K + 255) // 256) * pair_kstep_bytes + M * N * 2     # operand feed + bf16 output
+        l2_feed = {"steady_state_tflops": steady, "peak_tbs": feed_peak, "bytes_per_step": step_bytes,
+                   "note": "the GEMM is bound by L2 <-> SM traffic: peak = what the kernel's steady state (148 tiles of "
+                           "K = 65536, measured in this run) moves from L2 to shared memory; bytes_per_step = operand "
+                           "codes and scale tiles of every tile and K-step plus the bf16 outputs of the 12 GEMMs"}
+        api.check()
+
     fp8_info = None
     if ladder:
         f8_ms = sum(a0.elapsed_time(a1) for a0, a1, _ in fp8_evs)
@@ -578,6 +621,10 @@ def run_ours(args):
         "launch_timing": f"median of {n_dec - 1} repetitions per launch, CUDA events on the launching stream",
         "tflops_by_launch": gemm_by_shape,
         "mma_only_ceiling": mma_only,
+        "l2_feed": (dict(l2_feed, achieved_tbs=l2_feed["bytes_per_step"] / (gemm_ms * 1e-3) / 1e12,
+                         frac=l2_feed["bytes_per_step"] / (gemm_ms * 1e-3) / 1e12 / l2_feed["peak_tbs"],
+                         frac_of_steady_state_tflops=gemm_tflops / l2_feed["steady_state_tflops"])
+                    if l2_feed else None),
         "frac_of_mma_only_random_sustained": (gemm_tflops / mma_only["random_operands_sustained_tflops"]) if mma_only else None,
         "fused_path": {"tflops": step_tflops, "frac_of_nominal_fp4": step_tflops / 9000.0,
                        "frac_of_4x_burst_bf16": step_tflops / fp4_peak,
