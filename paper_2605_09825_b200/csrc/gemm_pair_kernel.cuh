@@ -8,8 +8,8 @@
 // 2 x 96 rows of B: 40 KB per K-step of 256 elements for 128 x 384 outputs, against the 48 KB a
 // lone 128 x 256 tile needs for two thirds of that -- the L2 -> shared-memory operand feed
 // (about 10.5 TB/s on this part), not the tensor pipe, is what bounds an FP4 GEMM here, and the
-// 512 TMEM columns are exactly used up: 384 accumulator + 4 x 32 scale columns.  No TMA
-// multicast is used: every CTA fetches its own operands; only barrier signals cross the pair.
+// 512 TMEM columns are exactly used up: 384 accumulator + 4 x 32 scale columns.  Every CTA
+// fetches its own operands with plain TMA loads; only barrier signals cross the pair.
 //
 // Roles per CTA (512 threads, four warpgroups; registers rebalanced with setmaxnreg):
 //   warps 0..3   scale warps (one per TMEM lane quadrant): shared memory -> this CTA's TMEM scale

@@ -395,7 +395,7 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 }
 
 // 2-D tiled load whose completion is counted on a barrier that may live in the peer CTA of the
-// pair (no multicast: the data lands only in the executing CTA's shared memory).
+// pair (the data lands only in the executing CTA's shared memory).
 __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* tmap, uint32_t bar_cluster_addr,
                                                  int32_t x, int32_t y)
 {
