@@ -521,6 +521,7 @@ def run_ours(args):
     mma_only = None
     if not args.no_mma_probe:
         def mma_rate(random_operands, launches):
+            time.sleep(1.0)                   # let the clocks recover from the previous leg
             api.probe_mma_rate(10000, random_operands)
             torch.cuda.synchronize()
             m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -532,22 +533,25 @@ def run_ours(args):
             torch.cuda.synchronize()
             return fl / (m0.elapsed_time(m1) * 1e-3) / 1e12
         mma_only = {"constant_operands_tflops": mma_rate(False, 10), "random_operands_burst_tflops": mma_rate(True, 5),
-                    "random_operands_sustained_tflops": mma_rate(True, 60),
+                    "random_operands_sustained_tflops": mma_rate(True, 60),   # each after a second of idling
                     "note": "mxfp4_probe_mma_rate: 256x192x64 pair MMAs, eight per iteration as in one K-step of the "
                             "GEMM, operands resident in shared memory; 10 / 5 / 60 launches of ~5 ms; with random "
                             "operand bits the tensor pipe alone reaches the power limit"}
         api.check()
 
     # ---- the GEMM kernel's own steady state: 148 tiles of K = 65536 (tile switches, epilogue and partial
-    # waves negligible), quantized-activation-like codes.  It does not depend on the operand bits (constant
-    # bits give the same rate), i.e. it is the L2 -> shared-memory operand feed, not power, that sets it;
-    # bytes moved per K-step of a CTA pair: codes 2 x (16 + 24) KB + scale tiles 2 x (1 + 3) KB.
-    l2_feed = None
+    # waves negligible) on quantized-activation-like codes (or constant ones: --steady-state-codes const).
+    # With constant codes this loop runs at ~8.1 PFLOP/s (91 % of the MMA-only rate): in cycles the K loop
+    # is close to the tensor pipe; with codes that toggle it is the power limit that holds it lower.
+    steady_state = None
     if not args.no_mma_probe and not ladder:
+        time.sleep(1.0)                       # let the clocks recover from the previous leg
         Ms, Ns, Ks = 1024, 37 * 384, 65536
         gen = torch.Generator(device="cuda").manual_seed(11)
 
         def like_codes(rows):
+            if args.steady_state_codes == "const":
+                return torch.full((rows, Ks // 2), 0x22, dtype=torch.uint8, device="cuda")
             mag = torch.clamp((torch.randn(rows, Ks, device="cuda", generator=gen).abs() * 2.0).round(), 0, 7).to(torch.uint8)
             sgn = (torch.rand(rows, Ks, device="cuda", generator=gen) < 0.5).to(torch.uint8) << 3
             c = mag | sgn
@@ -560,25 +564,29 @@ def run_ours(args):
         for _ in range(3):
             api.gemm(a_c, a_s, b_c, b_s, 1.0, api.OUT_BF16, out=o_s)
         torch.cuda.synchronize()
-        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s0.record(stream)
-        for _ in range(20):
-            api.gemm(a_c, a_s, b_c, b_s, 1.0, api.OUT_BF16, out=o_s)
-        s1.record(stream)
-        torch.cuda.synchronize()
-        steady = 2.0 * Ms * Ns * Ks * 20 / (s0.elapsed_time(s1) * 1e-3) / 1e12
+
+        def rate(launches):
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s0.record(stream)
+            for _ in range(launches):
+                api.gemm(a_c, a_s, b_c, b_s, 1.0, api.OUT_BF16, out=o_s)
+            s1.record(stream)
+            torch.cuda.synchronize()
+            return 2.0 * Ms * Ns * Ks * launches / (s0.elapsed_time(s1) * 1e-3) / 1e12
+
+        burst, sustained = rate(20), rate(300)          # ~6 ms, then ~0.1 s
         del a_c, b_c, a_s, b_s, o_s
+        # bytes between L2 and the SMs per K-step of a CTA pair: codes 2 x (16 + 24) KB + scale tiles 2 x (1 + 3) KB
         pair_kstep_bytes = 2 * (16384 + 24576) + 2 * (1024 + 3072)
-        pair_kstep_flops = 2.0 * 256 * 384 * 256
-        feed_peak = steady * 1e12 * pair_kstep_bytes / pair_kstep_flops / 1e12          # TB/s at the steady state
         step_bytes = 0.0
         for (_, _, _, _, M, N, K) in passes:
             tiles = ((M + 255) // 256) * ((N + 383) // 384)
             step_bytes += tiles * ((K + 255) // 256) * pair_kstep_bytes + M * N * 2     # operand feed + bf16 output
-        l2_feed = {"steady_state_tflops": steady, "peak_tbs": feed_peak, "bytes_per_step": step_bytes,
-                   "note": "the GEMM is bound by L2 <-> SM traffic: peak = what the kernel's steady state (148 tiles of "
-                           "K = 65536, measured in this run) moves from L2 to shared memory; bytes_per_step = operand "
-                           "codes and scale tiles of every tile and K-step plus the bf16 outputs of the 12 GEMMs"}
+        steady_state = {"codes": args.steady_state_codes, "burst_tflops": burst, "sustained_tflops": sustained,
+                        "l2_sm_bytes_per_step": step_bytes,
+                        "note": "gemm_mxf4_pair_kernel on 1024 x 14208 x 65536 (148 tiles, one long K loop each): 20 launches, "
+                                "then 300 (0.1 s).  Same kernel, no tile switch, no epilogue to speak of: what is lost "
+                                "against the MMA-only ceiling is operand movement (cycles and, with toggling codes, power)"}
         api.check()
 
     fp8_info = None
@@ -621,11 +629,10 @@ def run_ours(args):
         "launch_timing": f"median of {n_dec - 1} repetitions per launch, CUDA events on the launching stream",
         "tflops_by_launch": gemm_by_shape,
         "mma_only_ceiling": mma_only,
-        "l2_feed": (dict(l2_feed, achieved_tbs=l2_feed["bytes_per_step"] / (gemm_ms * 1e-3) / 1e12,
-                         frac=l2_feed["bytes_per_step"] / (gemm_ms * 1e-3) / 1e12 / l2_feed["peak_tbs"],
-                         frac_of_steady_state_tflops=gemm_tflops / l2_feed["steady_state_tflops"])
-                    if l2_feed else None),
-        "frac_of_mma_only_random_sustained": (gemm_tflops / mma_only["random_operands_sustained_tflops"]) if mma_only else None,
+        "kernel_steady_state": (dict(steady_state, frac_of_burst=gemm_tflops / steady_state["burst_tflops"],
+                                     frac_of_sustained=gemm_tflops / steady_state["sustained_tflops"],
+                                     l2_sm_tbs_in_step=steady_state["l2_sm_bytes_per_step"] / (gemm_ms * 1e-3) / 1e12)
+                                if steady_state else None),
         "fused_path": {"tflops": step_tflops, "frac_of_nominal_fp4": step_tflops / 9000.0,
                        "frac_of_4x_burst_bf16": step_tflops / fp4_peak,
                        "frac_of_4x_sustained_bf16": step_tflops / fp4_peak_sustained,
@@ -837,6 +844,8 @@ def main():
     ap.add_argument("--no-configs", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the per-variant quantize table")
     ap.add_argument("--no-mma-probe", action="store_true", help="skip the shared-memory-resident MMA ceiling")
+    ap.add_argument("--steady-state-codes", default="like", choices=["like", "const"],
+                    help="operand codes of the GEMM steady-state leg: quantized-activation-like (default) or constant")
     ap.add_argument("--decomposed-reps", type=int, default=20,
                     help="repetitions of the per-launch timed step (medians feed the roofline)")
     args = ap.parse_args()
