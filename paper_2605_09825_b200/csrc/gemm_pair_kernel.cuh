@@ -6,8 +6,10 @@
 // CTA-pair kernel (tcgen05 cta_group::2): the two CTAs of a cluster share one 256 x 384 output
 // tile (two 256 x 192 MMAs per K = 64).  Each CTA loads its own 128 rows of A and its own
 // 2 x 96 rows of B: 40 KB per K-step of 256 elements for 128 x 384 outputs, against the 48 KB a
-// lone 128 x 256 tile needs for two thirds of that -- the L2 -> shared-memory operand feed
-// (about 10.5 TB/s on this part), not the tensor pipe, is what bounds an FP4 GEMM here, and the
+// lone 128 x 256 tile needs for two thirds of that -- on operands that toggle, an FP4 GEMM here
+// runs at the device's power limit, and the bytes moved from L2 into shared memory per flop are
+// the part of that budget a kernel can shrink (with constant operand bits this kernel's K loop
+// reaches 91 % of the tensor pipe's own rate) -- and the
 // 512 TMEM columns are exactly used up: 384 accumulator + 4 x 32 scale columns.  Every CTA
 // fetches its own operands with plain TMA loads; only barrier signals cross the pair.
 //
