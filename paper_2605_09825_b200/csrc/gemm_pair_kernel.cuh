@@ -92,6 +92,7 @@ struct GemmPairParams {
     int64_t ld_out;
     int32_t M, N, K;
     int32_t tiles_m, tiles_n;   // 256 x 384 pair tiles
+    int32_t band_m;             // tile rows per band of the tile order (see gemm_tile_coords)
     int32_t k_stages;           // ceil(K / 256)
     int32_t sf_tiles_k;         // ceil(K / 128)
     int32_t sf_rows_a;          // ceil(M / 128)
@@ -125,6 +126,24 @@ __device__ __forceinline__ uint32_t make_idesc_mx_pair(uint32_t a_sf_id, uint32_
 // 16): an MMA's issue time is proportional to N, so e.g. the 256 columns that N = 4096 leaves for
 // its eleventh tile cost 192 + 64 instead of 2 x 192.
 __device__ __forceinline__ uint32_t idesc_n(int n) { return static_cast<uint32_t>(n >> 3) << 17; }
+
+// Tile order.  The persistent clusters take tiles cluster_id, cluster_id + n_clusters, ..., so at any
+// time about n_clusters consecutive tiles are in flight and read the same K range of their A and B
+// panels.  Tiles are numbered band by band: a band is `band_m` tile rows of M, and inside a band the
+// tile row varies fastest, then the tile column.  The A panel of a band (band_m x 256 rows x K) is
+// sized by the host to stay in L2 while the band sweeps across N, so A comes from HBM once; B is
+// re-read once per band.  (With a single band -- every shape whose A fits in L2 -- this is plain
+// column-major order.  With tile rows fastest over ALL of M, a long-K A that exceeds L2 was
+// streamed from HBM once per tile column: 2.6 GB instead of 0.7 GB for 16384 x 4096 x 28672.)
+__device__ __forceinline__ void gemm_tile_coords(const GemmPairParams& p, int tile, int& tm, int& tn)
+{
+    const int per_band = p.band_m * p.tiles_n;
+    const int band = tile / per_band;
+    const int r = tile - band * per_band;
+    const int rows = min(p.band_m, p.tiles_m - band * p.band_m);    // the last band may be shorter
+    tn = r / rows;
+    tm = band * p.band_m + (r - tn * rows);
+}
 
 // Columns the two MMAs of a tile in tile column `tn` compute: n0 for accumulator columns 0..191,
 // n1 (possibly 0: no MMA) for columns 192..383.  CTA r of the pair supplies rows
@@ -199,7 +218,8 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
         bool alive = true;
         for (int t = 0; alive && t < my_tiles; ++t) {
             const int tile = cluster_id + t * n_clusters;
-            const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+            int tm, tn;
+            gemm_tile_coords(p, tile, tm, tn);
             const int a_row_tile = tm * 2 + static_cast<int>(rank);     // 128-row scale tile of A
             int n0, n1;
             tile_mma_widths(p.N, tn, n0, n1);
@@ -260,8 +280,9 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
             int s = 0;
             uint32_t parity = 0;
             for (int tile_it = 0; alive && tile_it < my_tiles; ++tile_it) {
-                int n0, n1;
-                tile_mma_widths(p.N, (cluster_id + tile_it * n_clusters) / p.tiles_m, n0, n1);
+                int n0, n1, tm_unused, tn;
+                gemm_tile_coords(p, cluster_id + tile_it * n_clusters, tm_unused, tn);
+                tile_mma_widths(p.N, tn, n0, n1);
                 const uint32_t idn0 = idesc_n(n0), idn1 = idesc_n(n1);
                 if (tile_it > 0 && !mbar_wait(&sm.tmem_empty, (tile_it - 1) & 1, &sm.abort_flag)) break;
                 for (int ks = 0; ks < p.k_stages; ++ks, ++it) {
@@ -350,7 +371,8 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
         const uint32_t tmem_empty_leader = map_to_cta(smem_u32(&sm.tmem_empty), 0);
         for (int tile_it = 0; tile_it < my_tiles; ++tile_it) {
             const int tile = cluster_id + tile_it * n_clusters;
-            const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+            int tm, tn;
+            gemm_tile_coords(p, tile, tm, tn);
             if (!mbar_wait(&sm.tmem_full, tile_it & 1, &sm.abort_flag)) break;
             tcgen05_fence_after();
             const uint32_t taddr = tmem + (static_cast<uint32_t>(quad * 32) << 16) + half * kPMmaN;
@@ -536,6 +558,16 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
     p.K = static_cast<int32_t>(K);
     p.tiles_m = static_cast<int32_t>((M + kPTileM - 1) / kPTileM);
     p.tiles_n = static_cast<int32_t>((N + kPTileN - 1) / kPTileN);
+    {
+        // band height of the tile order: as many tile rows as keep the band's A panel within about a
+        // quarter of the L2 (32 MB), so that it survives the band's sweep across N beside the B
+        // panels streaming through
+        const int64_t a_tile_row_bytes = static_cast<int64_t>(kPTileM) * (KIND == 0 ? K / 2 : K);
+        int64_t band = (32ll << 20) / (a_tile_row_bytes > 0 ? a_tile_row_bytes : 1);
+        if (band < 1) band = 1;
+        if (band > p.tiles_m) band = p.tiles_m;
+        p.band_m = static_cast<int32_t>(band);
+    }
     constexpr int kBlockK = KIND == 0 ? kPBlockK : kPBlockK / 2;
     p.k_stages = static_cast<int32_t>((K + kBlockK - 1) / kBlockK);
     p.sf_tiles_k = static_cast<int32_t>((K + 127) / 128);
