@@ -629,6 +629,7 @@ def run_ours(args):
         "launch_timing": f"median of {n_dec - 1} repetitions per launch, CUDA events on the launching stream",
         "tflops_by_launch": gemm_by_shape,
         "mma_only_ceiling": mma_only,
+        "frac_of_mma_only_random_sustained": (gemm_tflops / mma_only["random_operands_sustained_tflops"]) if mma_only else None,
         "kernel_steady_state": (dict(steady_state, frac_of_burst=gemm_tflops / steady_state["burst_tflops"],
                                      frac_of_sustained=gemm_tflops / steady_state["sustained_tflops"],
                                      l2_sm_tbs_in_step=steady_state["l2_sm_bytes_per_step"] / (gemm_ms * 1e-3) / 1e12)
