@@ -199,3 +199,24 @@ def test_mma_rate_probe_runs_and_reports_its_flops():
         assert fl == 2.0 * 256 * 192 * 64 * 8 * 200 * (sms // 2)
     with pytest.raises(api.Mxfp4Error):
         api.probe_mma_rate(0, True)
+
+
+def test_band_order_with_a_ragged_last_band():
+    """K = 65536 makes a 256-row tile of A 8 MB, so the tile order uses bands of four tile rows:
+    M = 2304 + 40 gives bands of 4, 4 and 2 tile rows (the last one ragged in rows as well), N = 900
+    three tile columns with a narrow last one.  Whole output against the fp64 checker on the same
+    codes and scales, sampled rows of every band against the CPU oracle."""
+    import gemm_checker
+    rng = np.random.default_rng(65536)
+    M, N, K = 2344, 900, 65536
+    ac, asc, bc, bsc = _random_operands(rng, M, N, K, lo=122, hi=132)
+    out = api.gemm(_dev(ac), _dev(oracle.scales_to_tiled(asc)), _dev(bc), _dev(oracle.scales_to_tiled(bsc)),
+                   0.03125, api.OUT_FP32)
+    api.check()
+    rows = np.array([0, 255, 256, 1023, 1024, 1500, 2047, 2048, 2303, 2304, 2343])
+    ref, S = oracle.gemm(ac, asc, bc, bsc, alpha=0.03125, rows=rows)
+    assert_gemm_close(out[torch.from_numpy(rows).cuda()].cpu().numpy(), ref, S, False, "band order, sampled rows")
+    _, _, _, cref, cS = gemm_checker.check(ac[rows], asc[rows], bc, bsc, 0.03125, None, want_ref=True)
+    assert np.all(np.abs(cref.cpu().numpy() - ref) <= 1e-12 * S + 1e-300)
+    n_bad, first, worst, _, _ = gemm_checker.check(ac, asc, bc, bsc, 0.03125, out)
+    assert n_bad == 0 and worst <= 1.0, (n_bad, first // N, first % N, worst)
