@@ -161,7 +161,8 @@ def aggregate_over_ranks(elapsed_ms: float, world: int) -> float:
 
 def sweep_quantize_variants(dev_in, peaks, api, reps: int = 10):
     """GB/s of every quantizer variant -- {no rotation, deterministic H32, randomized H32} x {RNE,
-    stochastic rounding} x {row-wise, column-wise, dual-axis} -- on the activations of config 2
+    stochastic rounding} x {row-wise, column-wise, dual-axis}, plus the 16-point rotation with RNE
+    for its ratio to the 32-point one -- on the activations of config 2
     (X 8192 x 4096), the gradient of config 3 (dY 8192 x 28672) and the activations of config 4
     (X 8192 x 14336): the first 8192 tokens of this step's tensors, which follow those recipes.
     Single launches, CUDA events, a 256 MB buffer rewritten before each so that nothing comes from
@@ -197,8 +198,11 @@ def sweep_quantize_variants(dev_in, peaks, api, reps: int = 10):
                0: (torch.empty((cols, rows // 2), dtype=torch.uint8, device="cuda"),
                    torch.empty(api.scales_bytes(cols, rows), dtype=torch.uint8, device="cuda"))}
         table = {}
-        for hname, hmode in (("none", api.HADAMARD_NONE), ("h32", api.HADAMARD_DET), ("rh32", api.HADAMARD_RAND)):
+        for hname, hmode in (("none", api.HADAMARD_NONE), ("h32", api.HADAMARD_DET), ("rh32", api.HADAMARD_RAND),
+                             ("h16", api.HADAMARD_DET16)):
             for rname, rnd in (("rne", api.ROUND_RNE), ("sr", api.ROUND_SR)):
+                if hname == "h16" and rname == "sr":
+                    continue          # the 16-point variant is listed for its H16 : H32 ratio only
                 for axis, aname in ((1, "row"), (0, "col")):
                     c, sc = buf[axis]
                     ms = timed(lambda: api.quantize(x, axis, hmode, rnd, 7, 0, codes=c, scales=sc))
@@ -209,6 +213,9 @@ def sweep_quantize_variants(dev_in, peaks, api, reps: int = 10):
                 gbs = n * 3.0625 / (ms * 1e-3) / 1e9
                 table[f"dual {hname} {rname}"] = {"us": round(ms * 1e3, 1), "gbs": round(gbs, 1),
                                                   "frac": round(gbs / hbm, 3)}
+        # the paper's one kernel-level number is the H16 : H32 throughput ratio (1.08 on its hardware)
+        table["h16_to_h32_ratio"] = {ax: round(table[f"{ax} h16 rne"]["gbs"] / table[f"{ax} h32 rne"]["gbs"], 3)
+                                     for ax in ("row", "col", "dual")}
         out["cases"][tname] = table
         del buf
     del flush
