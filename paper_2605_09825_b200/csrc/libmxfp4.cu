@@ -306,7 +306,7 @@ static int gemm_checked(const void* a_codes, const void* a_scales, const void* b
 
 extern "C" {
 
-int mxfp4_version(void) { return 104; }   // 1.4: thread-safe first calls, argument checks before any enqueue
+int mxfp4_version(void) { return 105; }   // 1.5: band-ordered GEMM tiles, bounds-checking build, diagnostics
 
 const char* mxfp4_status_string(int status)
 {
