@@ -194,6 +194,9 @@ int mxfp4_quantize_pair(const mxfp4_quant_desc* a, const mxfp4_quant_desc* b, in
  *   out[m][n] = alpha * sum_t 2^(sa[m][t]-127) * 2^(sb[n][t]-127) * sum_{k in block t} A[m][k]*B[n][k]
  * A: [M x K], B: [N x K], both K-major codes with TILED scales (as mxfp4_quantize writes
  * them).  K multiple of 32.  Products are exact; accumulation is fp32 on the tensor cores.
+ * Scale bytes of tile rows past M (or N) are never used for a stored element and may hold
+ * anything; the bytes of blocks past K/32 inside the last 128-element tile are multiplied with
+ * zero codes and must not be 0xFF (mxfp4_quantize writes 0 there).
  *   alpha        exact power of two in the intended use (2^-5 undoes H*H^T = 32*I).
  *   out          [M x N] row-major, leading dimension ld_out (elements), bf16 (RNE) or fp32;
  *                16-byte aligned, ld_out*sizeof(elem) a multiple of 16.

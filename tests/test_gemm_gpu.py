@@ -178,6 +178,27 @@ def test_ragged_n_with_padded_leading_dimension(M, N, K, ld, out_dtype):
     assert (big[:, N:] == 7.0).all()
 
 
+def test_scale_bytes_of_rows_that_do_not_exist_never_reach_an_output():
+    """The tiled scale buffers hold whole tiles of 128 rows; what stands in the rows past M (or N)
+    belongs to accumulator rows (columns) that are never stored.  With 0xFF -- the E8M0 NaN -- in
+    all of them the result is the same and finite."""
+    rng = np.random.default_rng(77)
+    M, N, K = 200, 304, 256
+    ac, asc, bc, bsc = _random_operands(rng, M, N, K)
+    ref, S = oracle.gemm(ac, asc, bc, bsc, alpha=1.0)
+    a_pad = np.full((256, K // 32), 0xFF, dtype=np.uint8)
+    b_pad = np.full((384, K // 32), 0xFF, dtype=np.uint8)
+    a_pad[:M], b_pad[:N] = asc, bsc
+    a_t, b_t = oracle.scales_to_tiled(a_pad), oracle.scales_to_tiled(b_pad)
+    assert a_t.size == api.scales_bytes(M, K, api.SCALES_TILED) and b_t.size == api.scales_bytes(N, K, api.SCALES_TILED)
+    for out_dtype in (api.OUT_FP32, api.OUT_BF16):
+        out = api.gemm(_dev(ac), _dev(a_t), _dev(bc), _dev(b_t), 1.0, out_dtype)
+        api.check()
+        got = out.float().cpu().numpy()
+        assert np.isfinite(got).all()
+        assert_gemm_close(got, ref, S, out_dtype == api.OUT_BF16, "0xFF in the padding rows")
+
+
 def test_plain_stream_order_launches_still_work():
     """MXFP4_PDL=0 turns the programmatic-dependent-launch attribute off; same results."""
     import os
