@@ -160,6 +160,22 @@ static void fill_quant_params(QuantParams* pp, int64_t outer, int64_t K, int had
     p.block2d = block2d;
 }
 
+// Size limits of the kernels' 32-bit tile arithmetic, checked on the host before anything else is
+// done with a shape: a quantizer walks at most 2^30 source tiles of 128 x 128, a GEMM at most 2^30
+// output tiles of 256 x 384 and fewer than 2^31 (output tile, K-step of 256 elements) pairs.
+static bool quant_tiles_fit(int64_t rows, int64_t cols)
+{
+    return ((rows + 127) / 128) * ((cols + 127) / 128) <= 0x3FFFFFFF;
+}
+
+static bool gemm_tiles_fit(int64_t M, int64_t N, int64_t K)
+{
+    const int64_t tiles = ((M + kPTileM - 1) / kPTileM) * ((N + kPTileN - 1) / kPTileN);
+    if (tiles > 0x3FFFFFFF) return false;
+    const int64_t k_steps = (K + 127) / 128;              // the 8-bit kernel's K-step; the 4-bit one's is 256
+    return tiles <= 0x7FFFFFFF / k_steps;
+}
+
 // Validates one tensor's arguments and fills its job (tensor maps + parameters).
 static int build_quant_job(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld_src, int axis,
                            int hadamard_mode, int rounding, uint64_t seed, uint32_t operand_tag,
@@ -174,7 +190,7 @@ static int build_quant_job(const void* src_bf16, int64_t rows, int64_t cols, int
     const int64_t outer = axis ? rows : cols;
     const int64_t K = axis ? cols : rows;
     if (K % 32 != 0) return MXFP4_ERR_SHAPE;
-    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF || !quant_tiles_fit(rows, cols)) return MXFP4_ERR_SHAPE;
     if (!aligned16(src_bf16) || !aligned16(codes) || !aligned16(scales)) return MXFP4_ERR_ALIGN;
     if (ld_src % 8 != 0) return MXFP4_ERR_ALIGN;
     const DeviceInfo& dev = device_info();
@@ -291,7 +307,7 @@ static int gemm_checked(const void* a_codes, const void* a_scales, const void* b
     if (!a_codes || !a_scales || !b_codes || !b_scales || !out) return MXFP4_ERR_NULL;
     if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
     if (M <= 0 || N <= 0 || K <= 0 || K % 32 != 0 || ld_out < N) return MXFP4_ERR_SHAPE;
-    if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF || !gemm_tiles_fit(M, N, K)) return MXFP4_ERR_SHAPE;
     if (!aligned16(a_codes) || !aligned16(a_scales) || !aligned16(b_codes) || !aligned16(b_scales) ||
         !aligned16(out))
         return MXFP4_ERR_ALIGN;
@@ -377,7 +393,7 @@ int mxfp4_quantize_dual(const void* src_bf16, int64_t rows, int64_t cols, int64_
     if (block_shape != MXFP4_BLOCK_1X32 && block_shape != MXFP4_BLOCK_32X32) return MXFP4_ERR_ENUM;
     if (rows <= 0 || cols <= 0 || ld_src < cols) return MXFP4_ERR_SHAPE;
     if (rows % 32 != 0 || cols % 32 != 0) return MXFP4_ERR_SHAPE;      // both axes are reduction axes here
-    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF || !quant_tiles_fit(rows, cols)) return MXFP4_ERR_SHAPE;
     if (!aligned16(src_bf16) || !aligned16(codes_rowwise) || !aligned16(scales_rowwise) ||
         !aligned16(codes_colwise) || !aligned16(scales_colwise))
         return MXFP4_ERR_ALIGN;
@@ -509,6 +525,7 @@ static int linear_pass(int pass, const void* a_src, const void* b_src, void* out
     // everything the GEMM would reject is checked here, before the quantize launch
     if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_ENUM;
     if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (!gemm_tiles_fit(M, N, K) || !quant_tiles_fit(M, K) || !quant_tiles_fit(N, K)) return MXFP4_ERR_SHAPE;
     const size_t need = pass_workspace_bytes(T, in_f, out_f, pass, precision);
     if (!workspace || workspace_bytes < need) return MXFP4_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MXFP4_ERR_ALIGN;
@@ -615,6 +632,10 @@ static int layer_args_ok(int64_t T, int64_t in_f, int64_t out_f, int hmode, int 
 {
     if (T <= 0 || in_f <= 0 || out_f <= 0) return MXFP4_ERR_SHAPE;
     if (T % 32 != 0 || in_f % 32 != 0 || out_f % 32 != 0) return MXFP4_ERR_SHAPE;
+    if (T > 0x7FFFFFFF || in_f > 0x7FFFFFFF || out_f > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (!quant_tiles_fit(T, in_f) || !quant_tiles_fit(out_f, in_f) || !quant_tiles_fit(T, out_f) ||
+        !gemm_tiles_fit(T, out_f, in_f) || !gemm_tiles_fit(T, in_f, out_f) || !gemm_tiles_fit(out_f, in_f, T))
+        return MXFP4_ERR_SHAPE;
     if (hmode < 0 || hmode > 4 || rounding < 0 || rounding > 1) return MXFP4_ERR_ENUM;
     if (!saved || saved_bytes < mxfp4_linear_layer_bytes(T, in_f, out_f, MXFP4_LAYER_SAVED)) return MXFP4_ERR_WORKSPACE;
     if (!workspace || workspace_bytes < mxfp4_linear_layer_bytes(T, in_f, out_f, ws_kind)) return MXFP4_ERR_WORKSPACE;

@@ -99,3 +99,33 @@ def test_output_errors_are_found_before_the_quantize_launch(lib):
     bw = lib.mxfp4_linear_backward
     assert bw(p, p, p + 6, 64, 64, 64, 1, 0, 0, 0, 0, p, big, p, big, None) == -3
     assert bw(p, p, p, 64, 64, 64, 1, 0, 0, 0, 3, p, big, p, big, None) == -4
+
+
+def test_empty_and_oversized_shapes_are_shape_errors(lib):
+    """Zero-sized tensors and sizes past the kernels' 32-bit tile arithmetic (a dimension of 2^31 or
+    more, more than 2^30 tiles, 2^31 or more tile K-steps) are refused on the host, before the
+    device is looked at."""
+    buf = ctypes.create_string_buffer(1 << 12)
+    p = (ctypes.addressof(buf) + 255) & ~255
+    big = 0x7FFFFFE0                                    # the largest multiple of 32 below 2^31
+    q, g, d = lib.mxfp4_quantize, lib.mxfp4_gemm, lib.mxfp4_quantize_dual
+    for axis in (0, 1):
+        assert q(p, 0, 32, 32, axis, 0, 0, 0, 0, p, p, 1, None) == -2
+        assert q(p, 32, 0, 0, axis, 0, 0, 0, 0, p, p, 1, None) == -2
+        assert q(p, 1 << 31, 32, 32, axis, 0, 0, 0, 0, p, p, 1, None) == -2
+        assert q(p, 32, 1 << 31, 1 << 31, axis, 0, 0, 0, 0, p, p, 1, None) == -2
+        assert q(p, big, big, big, axis, 0, 0, 0, 0, p, p, 1, None) == -2            # 2^48 tiles
+    assert d(p, 0, 32, 32, 1, 0, 0, 0, 1, 0, p, p, p, p, 1, None) == -2
+    assert d(p, big, big, big, 1, 0, 0, 0, 1, 0, p, p, p, p, 1, None) == -2
+    assert g(p, p, p, p, 0, 128, 128, 1.0, p, 0, 128, None, 0, None) == -2
+    assert g(p, p, p, p, 128, 0, 128, 1.0, p, 0, 128, None, 0, None) == -2
+    assert g(p, p, p, p, 128, 128, 0, 1.0, p, 0, 128, None, 0, None) == -2
+    assert g(p, p, p, p, 1 << 31, 128, 128, 1.0, p, 0, 128, None, 0, None) == -2
+    assert g(p, p, p, p, big, big, 32, 1.0, p, 0, big, None, 0, None) == -2          # 2^45 tiles
+    assert g(p, p, p, p, 1 << 20, 1 << 20, 1 << 30, 1.0, p, 0, 1 << 20, None, 0, None) == -2   # tiles x K-steps
+    f = lib.mxfp4_linear_fprop
+    assert f(p, p, p, 0, 128, 128, 1, 0, 0, 0, p, 1 << 15, None) == -2
+    assert f(p, p, p, big, big, big, 1, 0, 0, 0, p, 1 << 15, None) == -2
+    fw = lib.mxfp4_linear_forward
+    assert fw(p, p, p, 0, 64, 64, 1, 0, 0, 0, p, 1 << 16, p, 1 << 16, None) == -2
+    assert fw(p, p, p, big, big, big, 1, 0, 0, 0, p, 1 << 16, p, 1 << 16, None) == -2
