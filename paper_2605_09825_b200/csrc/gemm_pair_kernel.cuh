@@ -168,8 +168,7 @@ __device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tm_a, const CU
     constexpr int kMmaK = KIND == 0 ? 64 : 32;                     // elements per MMA
     constexpr int kSfTilesPerStage = KIND == 0 ? 2 : 1;
     extern __shared__ uint8_t smem_raw[];
-    GemmPairSmem& sm = *reinterpret_cast<GemmPairSmem*>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    GemmPairSmem& sm = *reinterpret_cast<GemmPairSmem*>(smem_align_1024(smem_raw));
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();

@@ -257,15 +257,24 @@ static int launch_quant_jobs_fp8(const QuantJob& j0, const QuantJob& j1, int axi
     return MXFP4_ERR_ENUM;
 }
 
-template <int HMODE, int SR>
-static int launch_quantize_dual(const QuantDualJob& job, int grid, cudaStream_t stream)
+template <int HMODE, int SR, bool PLAIN>
+static int launch_quantize_dual_as(const QuantDualJob& job, int grid, cudaStream_t stream)
 {
     const size_t smem = sizeof(QuantDualSmem) + 1024;
     static PerDeviceOnce once;               // the attribute is per device
-    const int rc = ensure_smem_attribute(once, quantize_dual_kernel<HMODE, SR>, smem);
+    const int rc = ensure_smem_attribute(once, quantize_dual_kernel<HMODE, SR, PLAIN>, smem);
     if (rc != MXFP4_OK) return rc;
-    return launch_kernel_pdl(quantize_dual_kernel<HMODE, SR>, grid, kQThreads, smem, stream, job) == cudaSuccess
+    return launch_kernel_pdl(quantize_dual_kernel<HMODE, SR, PLAIN>, grid, kQThreads, smem, stream, job) == cudaSuccess
                ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+template <int HMODE, int SR>
+static int launch_quantize_dual(const QuantDualJob& job, int grid, cudaStream_t stream)
+{
+    // the layer-level path (tiled scales, 1 x 32 blocks) has an instantiation of its own
+    if (job.pr.scale_layout == MXFP4_SCALES_TILED && !job.pr.block2d)
+        return launch_quantize_dual_as<HMODE, SR, true>(job, grid, stream);
+    return launch_quantize_dual_as<HMODE, SR, false>(job, grid, stream);
 }
 
 static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -24,8 +24,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMmaProbeThreads, 1)
 mma_rate_probe_kernel(int iterations, int random_operands)
 {
     extern __shared__ uint8_t smem_raw[];
-    MmaProbeSmem& sm = *reinterpret_cast<MmaProbeSmem*>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    MmaProbeSmem& sm = *reinterpret_cast<MmaProbeSmem*>(smem_align_1024(smem_raw));
     // operand bits: a constant pattern, or a per-thread linear congruential sequence
     uint32_t x = 1234567u + blockIdx.x * 7919u + threadIdx.x * 104729u;
     constexpr int kWords = (kPStages * kPABytes + kPStages * 2 * kPBSubBytes) / 4;

@@ -57,6 +57,16 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p)
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// Start of a kernel's dynamic shared memory rounded up to 1024 bytes (what the 128-byte swizzle
+// wants).  The padding is added to the POINTER: rounding the address up as an integer and casting
+// back hides the address space from the compiler, and every access through such a pointer becomes
+// a generic load or store (global-path latency, 64-bit address arithmetic) instead of
+// ld.shared / st.shared.
+__device__ __forceinline__ uint8_t* smem_align_1024(uint8_t* smem_raw)
+{
+    return smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+}
+
 // Programmatic dependent launch: every kernel of the library is launched with the
 // programmatic-stream-serialization attribute, so its CTAs may start (barrier set-up, TMEM
 // allocation, descriptor prefetch) while the previous kernel in the stream is still draining.
@@ -172,6 +182,15 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const void* tmap, ui
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)),
         "r"(x), "r"(y)
         : "memory");
+}
+
+// 2-D tiled prefetch global -> L2: the box a later tma_load_2d will fetch, so that load finds its
+// data in L2 (same alignment rule for x).
+__device__ __forceinline__ void tma_prefetch_l2_2d(const void* tmap, int32_t x, int32_t y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];"
+                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y)
+                 : "memory");
 }
 
 // 2-D tiled store shared -> global (bulk async-group completion).

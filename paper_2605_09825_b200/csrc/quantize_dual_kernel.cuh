@@ -83,13 +83,14 @@ __device__ __forceinline__ void load_column_blocks(const uint8_t* stage, int kb,
 
 // Stage one block's results: codes into the 64-byte-swizzled code tile, the scale byte into the
 // 512-byte scale tile (tiled layout) or straight to global memory (canonical layout).
+template <bool TILED = false>
 __device__ __forceinline__ void stage_block(uint8_t* code_tile, uint8_t* scale_tile, const QuantParams& p, int o,
                                             int kb, int to, int tk, const uint32_t (&packed)[4], uint32_t byte,
                                             bool ok)
 {
     smem_store(code_tile + o * 64 + ((kb ^ ((o >> 1) & 3)) * 16), make_uint4(packed[0], packed[1], packed[2], packed[3]),
                code_tile, kQCodeTileBytes);
-    if (p.scale_layout == 1) {
+    if (TILED || p.scale_layout == 1) {
         smem_store(scale_tile + (o & 31) * 16 + (o >> 5) * 4 + kb, static_cast<uint8_t>(byte), scale_tile,
                    kQScaleTileBytes);
     } else if (ok) {
@@ -99,7 +100,9 @@ __device__ __forceinline__ void stage_block(uint8_t* code_tile, uint8_t* scale_t
     }
 }
 
-template <int HMODE, int SR>
+// PLAIN: the tiled scale layout and 1 x 32 blocks are known at compile time (the layer-level path);
+// otherwise both are read from the job.
+template <int HMODE, int SR, bool PLAIN>
 __global__ void __launch_bounds__(kQThreads, 1)
 quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
 {
@@ -107,8 +110,7 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
     constexpr int kQDGroupThreads = Shape::kGroupThreads, kQDGroups = Shape::kGroups, kQDSub = Shape::kSub,
                   kQDBufs = Shape::kBufs;
     extern __shared__ uint8_t smem_raw[];
-    QuantDualSmem& sm = *reinterpret_cast<QuantDualSmem*>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    QuantDualSmem& sm = *reinterpret_cast<QuantDualSmem*>(smem_align_1024(smem_raw));
     const int tid = threadIdx.x;
     const int total_tiles = job.tiles_r * job.tiles_c;
     const int my_tiles = blockIdx.x < total_tiles ? (total_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
@@ -138,6 +140,15 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
                 mbar_arrive_expect_tx(&sm.full[s], kQStageBytes);
                 tma_load_2d(&sm.stage[s][0], &job.tm_src, &sm.full[s], tc * 128, tr * 128);
                 tma_load_2d(&sm.stage[s][kQStageBytes / 2], &job.tm_src, &sm.full[s], tc * 128 + 64, tr * 128);
+                // the tile this stage takes next goes to L2 now: its load is issued only when the
+                // stage comes back, three quarters into the tile after this one of its group, and
+                // would otherwise wait for HBM with a quarter of a tile's time to hide it in
+                if (it + kQDStages < my_tiles) {
+                    const int nt = tile + kQDStages * gridDim.x;
+                    const int ntr = nt / job.tiles_c, ntc = nt % job.tiles_c;
+                    tma_prefetch_l2_2d(&job.tm_src, ntc * 128, ntr * 128);
+                    tma_prefetch_l2_2d(&job.tm_src, ntc * 128 + 64, ntr * 128);
+                }
             }
         }
         return;
@@ -180,30 +191,22 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
             const int jc = tv & 63;
 
             // ---- row-wise operand: operand row = source row, K = columns
-            if (ok) {
-                load_block<1, HMODE>(&sm.stage[s][0], kbh, o, pr.signs, P0);
-                load_block<1, HMODE>(&sm.stage[s][0], kbh + 2, o, pr.signs, P1);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
-            }
+            // (after a failed wait the stage holds whatever it held: the blocks are still worked
+            // through, nothing computed from them leaves the CTA)
+            load_block<1, HMODE>(&sm.stage[s][0], kbh, o, pr.signs, P0);
+            load_block<1, HMODE>(&sm.stage[s][0], kbh + 2, o, pr.signs, P1);
             {
                 const uint64_t e_row = static_cast<uint64_t>(tr * 128 + o) * static_cast<uint64_t>(pr.K);
                 uint8_t* ct = &sm.code_tile[slot][0];
                 uint8_t* st = &sm.scale_tile[slot][0];
-                quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tc * 4 + kbh) * 32), pr, packed, byte);
-                stage_block(ct, st, pr, o, kbh, tr, tc, packed, byte, ok);
-                quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tc * 4 + kbh + 2) * 32), pr, packed, byte);
-                stage_block(ct, st, pr, o, kbh + 2, tr, tc, packed, byte, ok);
+                quantize_block<HMODE, SR, PLAIN>(P0, e_row + static_cast<uint64_t>((tc * 4 + kbh) * 32), pr, packed, byte);
+                stage_block<PLAIN>(ct, st, pr, o, kbh, tr, tc, packed, byte, ok);
+                quantize_block<HMODE, SR, PLAIN>(P1, e_row + static_cast<uint64_t>((tc * 4 + kbh + 2) * 32), pr, packed, byte);
+                stage_block<PLAIN>(ct, st, pr, o, kbh + 2, tr, tc, packed, byte, ok);
             }
 
             // ---- column-wise operand: operand row = source column, K = rows
-            if (ok) {
-                load_column_blocks<HMODE>(&sm.stage[s][0], kbc, jc, pc.signs, P0, P1);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
-            }
+            load_column_blocks<HMODE>(&sm.stage[s][0], kbc, jc, pc.signs, P0, P1);
             if (u == kQDSub - 1) {
                 // the stage is in registers now: hand it back to the producer
                 __syncwarp();
@@ -212,15 +215,15 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
             {
                 float amax0 = rotate_and_amax<HMODE>(P0);
                 float amax1 = rotate_and_amax<HMODE>(P1);
-                if (pc.block2d) amax0 = amax1 = lanes_max(half_mask, fmaxf(amax0, amax1));
+                if (!PLAIN && pc.block2d) amax0 = amax1 = lanes_max(half_mask, fmaxf(amax0, amax1));
                 const uint64_t e_blk = static_cast<uint64_t>((tr * 4 + kbc) * 32);
                 const uint64_t e_row = static_cast<uint64_t>(tc * 128 + 2 * jc) * static_cast<uint64_t>(pc.K);
                 uint8_t* ct = &sm.code_tile[slot + 1][0];
                 uint8_t* st = &sm.scale_tile[slot + 1][0];
                 scale_round_pack<SR>(P0, amax0, e_row + e_blk, pc, packed, byte);
-                stage_block(ct, st, pc, 2 * jc, kbc, tc, tr, packed, byte, ok);
+                stage_block<PLAIN>(ct, st, pc, 2 * jc, kbc, tc, tr, packed, byte, ok);
                 scale_round_pack<SR>(P1, amax1, e_row + static_cast<uint64_t>(pc.K) + e_blk, pc, packed, byte);
-                stage_block(ct, st, pc, 2 * jc + 1, kbc, tc, tr, packed, byte, ok);
+                stage_block<PLAIN>(ct, st, pc, 2 * jc + 1, kbc, tc, tr, packed, byte, ok);
             }
         }
 
@@ -242,7 +245,7 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
         if (t == 0) {
             tma_store_2d(&job.tm_codes_row, &sm.code_tile[slot][0], tc * 64, tr * 128);
             tma_store_2d(&job.tm_codes_col, &sm.code_tile[slot + 1][0], tr * 64, tc * 128);
-            if (pr.scale_layout == 1) {
+            if (PLAIN || pr.scale_layout == 1) {
                 bulk_store_1d(pr.scales + (static_cast<int64_t>(tr) * pr.tiles_k + tc) * kQScaleTileBytes,
                               &sm.scale_tile[slot][0], kQScaleTileBytes);
                 bulk_store_1d(pc.scales + (static_cast<int64_t>(tc) * pc.tiles_k + tr) * kQScaleTileBytes,

@@ -124,8 +124,7 @@ __global__ void __launch_bounds__(kQThreads, 1)
 quantize_fp8_kernel(const __grid_constant__ QuantJobs jobs)
 {
     extern __shared__ uint8_t smem_raw[];
-    QuantFp8Smem& sm = *reinterpret_cast<QuantFp8Smem*>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    QuantFp8Smem& sm = *reinterpret_cast<QuantFp8Smem*>(smem_align_1024(smem_raw));
     const int tid = threadIdx.x;
     const int tiles0 = jobs.j[0].tiles;
     const int total_tiles = tiles0 + jobs.j[1].tiles;

@@ -290,12 +290,12 @@ __device__ __forceinline__ void scale_round_pack(const float2 (&P)[16], float am
 
 // One block owned by one thread, whose warp holds 32 consecutive operand rows of the same block
 // column: with 32 x 32 blocks (Appendix D) the maximum is taken over the warp.
-template <int HMODE, int SR>
+template <int HMODE, int SR, bool PLAIN = false>
 __device__ __forceinline__ void quantize_block(float2 (&P)[16], uint64_t e0, const QuantParams& p,
                                                uint32_t (&packed)[4], uint32_t& byte)
 {
     float amax = rotate_and_amax<HMODE>(P);
-    if (p.block2d) amax = lanes_max(0xFFFFFFFFu, amax);
+    if (!PLAIN && p.block2d) amax = lanes_max(0xFFFFFFFFu, amax);
     scale_round_pack<SR>(P, amax, e0, p, packed, byte);
 }
 
@@ -430,8 +430,7 @@ quantize_kernel(const __grid_constant__ QuantJobs jobs)
 {
     using Shape = QuantShape<HMODE, SR>;
     extern __shared__ uint8_t smem_raw[];
-    QuantSmem& sm = *reinterpret_cast<QuantSmem*>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    QuantSmem& sm = *reinterpret_cast<QuantSmem*>(smem_align_1024(smem_raw));
     const int tid = threadIdx.x;
     const int tiles0 = jobs.j[0].tiles;
     const int total_tiles = tiles0 + jobs.j[1].tiles;
