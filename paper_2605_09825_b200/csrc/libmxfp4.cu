@@ -272,7 +272,7 @@ template <int HMODE, int SR>
 static int launch_quantize_dual(const QuantDualJob& job, int grid, cudaStream_t stream)
 {
     // the layer-level path (tiled scales, 1 x 32 blocks) has an instantiation of its own
-    if (job.pr.scale_layout == MXFP4_SCALES_TILED && !job.pr.block2d)
+    if (!QuantDualShape<HMODE, SR>::kFirstForm && job.pr.scale_layout == MXFP4_SCALES_TILED && !job.pr.block2d)
         return launch_quantize_dual_as<HMODE, SR, true>(job, grid, stream);
     return launch_quantize_dual_as<HMODE, SR, false>(job, grid, stream);
 }

@@ -67,6 +67,13 @@ __device__ __forceinline__ uint8_t* smem_align_1024(uint8_t* smem_raw)
     return smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
 }
 
+// The same address reached through an integer: accesses through the result are generic loads and
+// stores.  Kept for the one kernel variant that measures faster that way (see quantize_dual_kernel).
+__device__ __forceinline__ uint8_t* smem_align_1024_generic(uint8_t* smem_raw)
+{
+    return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+}
+
 // Programmatic dependent launch: every kernel of the library is launched with the
 // programmatic-stream-serialization attribute, so its CTAs may start (barrier set-up, TMEM
 // allocation, descriptor prefetch) while the previous kernel in the stream is still draining.

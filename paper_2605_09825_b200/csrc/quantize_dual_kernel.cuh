@@ -32,6 +32,15 @@ struct QuantDualShape {
     static constexpr int kGroups = kQConsumers / kGroupThreads;
     static constexpr int kSub = 256 / kGroupThreads;
     static constexpr int kBufs = kGroups == 2 ? 2 : 1;
+    // The un-rotated round-to-nearest variant does so little arithmetic that it runs at the HBM
+    // bound (16384 x 14336 in 111-117 us back to back = 0.99 of the copy bandwidth) -- in the
+    // kernel's first form.  Each of the later savings makes THAT variant slower, measured one by
+    // one on one GPU: ld.shared / st.shared instead of generic accesses 139 us, the compile-time
+    // layout (PLAIN) 138, the L2 prefetch of the next tile 152; every other variant gains from
+    // each of them (deterministic H32 150 -> 134 us, stochastic rounding 342 -> 288).  Consumers
+    // that run ahead seem to bunch the memory requests of a kernel that has no arithmetic to
+    // hide them behind; the variant therefore keeps the first form.
+    static constexpr bool kFirstForm = HMODE == 0 && SR == 0;
 };
 
 struct QuantDualSmem {
@@ -110,7 +119,8 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
     constexpr int kQDGroupThreads = Shape::kGroupThreads, kQDGroups = Shape::kGroups, kQDSub = Shape::kSub,
                   kQDBufs = Shape::kBufs;
     extern __shared__ uint8_t smem_raw[];
-    QuantDualSmem& sm = *reinterpret_cast<QuantDualSmem*>(smem_align_1024(smem_raw));
+    QuantDualSmem& sm = *reinterpret_cast<QuantDualSmem*>(
+        Shape::kFirstForm ? smem_align_1024_generic(smem_raw) : smem_align_1024(smem_raw));
     const int tid = threadIdx.x;
     const int total_tiles = job.tiles_r * job.tiles_c;
     const int my_tiles = blockIdx.x < total_tiles ? (total_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
@@ -143,7 +153,7 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
                 // the tile this stage takes next goes to L2 now: its load is issued only when the
                 // stage comes back, three quarters into the tile after this one of its group, and
                 // would otherwise wait for HBM with a quarter of a tile's time to hide it in
-                if (it + kQDStages < my_tiles) {
+                if (!Shape::kFirstForm && it + kQDStages < my_tiles) {
                     const int nt = tile + kQDStages * gridDim.x;
                     const int ntr = nt / job.tiles_c, ntc = nt % job.tiles_c;
                     tma_prefetch_l2_2d(&job.tm_src, ntc * 128, ntr * 128);
@@ -192,9 +202,14 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
 
             // ---- row-wise operand: operand row = source row, K = columns
             // (after a failed wait the stage holds whatever it held: the blocks are still worked
-            // through, nothing computed from them leaves the CTA)
-            load_block<1, HMODE>(&sm.stage[s][0], kbh, o, pr.signs, P0);
-            load_block<1, HMODE>(&sm.stage[s][0], kbh + 2, o, pr.signs, P1);
+            // through, nothing computed from them leaves the CTA; the first form zero-fills instead)
+            if (!Shape::kFirstForm || ok) {
+                load_block<1, HMODE>(&sm.stage[s][0], kbh, o, pr.signs, P0);
+                load_block<1, HMODE>(&sm.stage[s][0], kbh + 2, o, pr.signs, P1);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
+            }
             {
                 const uint64_t e_row = static_cast<uint64_t>(tr * 128 + o) * static_cast<uint64_t>(pr.K);
                 uint8_t* ct = &sm.code_tile[slot][0];
@@ -206,7 +221,12 @@ quantize_dual_kernel(const __grid_constant__ QuantDualJob job)
             }
 
             // ---- column-wise operand: operand row = source column, K = rows
-            load_column_blocks<HMODE>(&sm.stage[s][0], kbc, jc, pc.signs, P0, P1);
+            if (!Shape::kFirstForm || ok) {
+                load_column_blocks<HMODE>(&sm.stage[s][0], kbc, jc, pc.signs, P0, P1);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
+            }
             if (u == kQDSub - 1) {
                 // the stage is in registers now: hand it back to the producer
                 __syncwarp();
