@@ -331,7 +331,7 @@ static int gemm_checked(const void* a_codes, const void* a_scales, const void* b
 
 extern "C" {
 
-int mxfp4_version(void) { return 105; }   // 1.5: band-ordered GEMM tiles, bounds-checking build, diagnostics
+int mxfp4_version(void) { return 106; }   // 1.6: shared-space accesses in the quantizers, size limits checked on the host
 
 const char* mxfp4_status_string(int status)
 {
