@@ -100,18 +100,29 @@ static uint32_t host_sign_mask(uint64_t seed)
     return c[0];
 }
 
-template <int AXIS0, int AXIS1, int HMODE, int SR>
-static int launch_quantize(const QuantJob& j0, const QuantJob& j1, int grid, cudaStream_t stream)
+template <int AXIS0, int AXIS1, int HMODE, int SR, bool PLAIN>
+static int launch_quantize_as(const QuantJob& j0, const QuantJob& j1, int grid, cudaStream_t stream)
 {
     const size_t smem = sizeof(QuantSmem) + 1024;
     static PerDeviceOnce once;               // the attribute is per device
-    const int rc = ensure_smem_attribute(once, quantize_kernel<AXIS0, AXIS1, HMODE, SR>, smem);
+    const int rc = ensure_smem_attribute(once, quantize_kernel<AXIS0, AXIS1, HMODE, SR, PLAIN>, smem);
     if (rc != MXFP4_OK) return rc;
     QuantJobs jobs;
     jobs.j[0] = j0;
     jobs.j[1] = j1;
-    return launch_kernel_pdl(quantize_kernel<AXIS0, AXIS1, HMODE, SR>, grid, kQThreads, smem, stream, jobs) == cudaSuccess
+    return launch_kernel_pdl(quantize_kernel<AXIS0, AXIS1, HMODE, SR, PLAIN>, grid, kQThreads, smem, stream, jobs) ==
+                   cudaSuccess
                ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+template <int AXIS0, int AXIS1, int HMODE, int SR>
+static int launch_quantize(const QuantJob& j0, const QuantJob& j1, int grid, cudaStream_t stream)
+{
+    // what the fused passes use (tiled scales, 1 x 32 blocks, in both jobs) has an instantiation of its own
+    const bool plain0 = j0.p.scale_layout == MXFP4_SCALES_TILED && !j0.p.block2d;
+    const bool plain1 = j1.tiles == 0 || (j1.p.scale_layout == MXFP4_SCALES_TILED && !j1.p.block2d);
+    if (plain0 && plain1) return launch_quantize_as<AXIS0, AXIS1, HMODE, SR, true>(j0, j1, grid, stream);
+    return launch_quantize_as<AXIS0, AXIS1, HMODE, SR, false>(j0, j1, grid, stream);
 }
 
 template <int AXIS0, int AXIS1>

@@ -340,7 +340,9 @@ struct QuantShape {
 // thread's blocks (two at a time, two sub-passes), stage codes and scales, and (thread 0 of the
 // group) store them.  `p` and `tm_codes` refer to kernel parameters, so every field is a
 // constant-bank operand.  Returns false when a wait gave up (the group leaves the kernel).
-template <int AXIS, int HMODE, int SR>
+// PLAIN: the tiled scale layout and 1 x 32 blocks are known at compile time (what the fused passes
+// use); otherwise both are read from the parameters.
+template <int AXIS, int HMODE, int SR, bool PLAIN>
 __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p, const CUtensorMap* tm_codes,
                                              int tile, int it, int trip, int grp, int t)
 {
@@ -364,13 +366,10 @@ __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p
         const int kbh = tv >> 7;                       // this thread's blocks along K: kbh and kbh + 2
         const int o = tv & 127;                        // operand row inside the tile
         float2 P0[16], P1[16];
-        if (ok) {
-            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.signs, P0);
-            load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.signs, P1);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) P0[i] = P1[i] = make_float2(0.0f, 0.0f);
-        }
+        // (after a failed wait the stage holds whatever it held: the blocks are still worked
+        // through, nothing computed from them leaves the CTA)
+        load_block<AXIS, HMODE>(&sm.stage[s][0], kbh, o, p.signs, P0);
+        load_block<AXIS, HMODE>(&sm.stage[s][0], kbh + 2, o, p.signs, P1);
         if (u == Shape::kSub - 1) {
             // the stage is in registers now: hand it back to the producer
             __syncwarp();
@@ -379,8 +378,8 @@ __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p
 
         const uint64_t e_row = static_cast<uint64_t>(to * kQTileO + o) * static_cast<uint64_t>(p.K);
         uint32_t packed0[4], packed1[4], byte0, byte1;
-        quantize_block<HMODE, SR>(P0, e_row + static_cast<uint64_t>((tk * 4 + kbh) * 32), p, packed0, byte0);
-        quantize_block<HMODE, SR>(P1, e_row + static_cast<uint64_t>((tk * 4 + kbh + 2) * 32), p, packed1, byte1);
+        quantize_block<HMODE, SR, PLAIN>(P0, e_row + static_cast<uint64_t>((tk * 4 + kbh) * 32), p, packed0, byte0);
+        quantize_block<HMODE, SR, PLAIN>(P1, e_row + static_cast<uint64_t>((tk * 4 + kbh + 2) * 32), p, packed1, byte1);
 
         // stage the results: codes in the 64-byte swizzle the TMA store expects
         uint8_t* ct = &sm.code_tile[slot][o * 64];
@@ -388,7 +387,7 @@ __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p
                    sm.code_tile[slot], kQCodeTileBytes);
         smem_store(ct + (((kbh + 2) ^ ((o >> 1) & 3)) * 16), make_uint4(packed1[0], packed1[1], packed1[2], packed1[3]),
                    sm.code_tile[slot], kQCodeTileBytes);
-        if (p.scale_layout == 1) {
+        if (PLAIN || p.scale_layout == 1) {
             uint8_t* st = &sm.scale_tile[slot][(o & 31) * 16 + (o >> 5) * 4];
             smem_store(st + kbh, static_cast<uint8_t>(byte0), sm.scale_tile[slot], kQScaleTileBytes);
             smem_store(st + kbh + 2, static_cast<uint8_t>(byte1), sm.scale_tile[slot], kQScaleTileBytes);
@@ -416,7 +415,7 @@ __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p
     if (any_fail) return false;
     if (t == 0) {
         tma_store_2d(tm_codes, &sm.code_tile[slot][0], tk * (kQTileK / 2), to * kQTileO);
-        if (p.scale_layout == 1)
+        if (PLAIN || p.scale_layout == 1)
             bulk_store_1d(p.scales + (static_cast<int64_t>(to) * p.tiles_k + tk) * kQScaleTileBytes,
                           &sm.scale_tile[slot][0], kQScaleTileBytes);
         bulk_commit_group();
@@ -424,7 +423,7 @@ __device__ __forceinline__ bool consume_tile(QuantSmem& sm, const QuantParams& p
     return true;
 }
 
-template <int AXIS0, int AXIS1, int HMODE, int SR>
+template <int AXIS0, int AXIS1, int HMODE, int SR, bool PLAIN>
 __global__ void __launch_bounds__(kQThreads, 1)
 quantize_kernel(const __grid_constant__ QuantJobs jobs)
 {
@@ -488,13 +487,13 @@ quantize_kernel(const __grid_constant__ QuantJobs jobs)
     for (; it < my_tiles; it += Shape::kGroups, ++trip) {
         const int gtile = blockIdx.x + it * gridDim.x;
         if (gtile >= tiles0) break;
-        alive = consume_tile<AXIS0, HMODE, SR>(sm, jobs.j[0].p, &jobs.j[0].tm_codes, gtile, it, trip, grp, t);
+        alive = consume_tile<AXIS0, HMODE, SR, PLAIN>(sm, jobs.j[0].p, &jobs.j[0].tm_codes, gtile, it, trip, grp, t);
         if (!alive) break;
     }
     if (alive) {
         for (; it < my_tiles; it += Shape::kGroups, ++trip) {
             const int gtile = blockIdx.x + it * gridDim.x;
-            if (!consume_tile<AXIS1, HMODE, SR>(sm, jobs.j[1].p, &jobs.j[1].tm_codes, gtile - tiles0, it, trip,
+            if (!consume_tile<AXIS1, HMODE, SR, PLAIN>(sm, jobs.j[1].p, &jobs.j[1].tm_codes, gtile - tiles0, it, trip,
                                                 grp, t))
                 break;
         }
