@@ -696,12 +696,17 @@ def run_ours(args):
         "frac_of_nominal_fp4": gemm_tflops / 9000.0, "peak_nominal_fp4": 9000.0,
         "frac_of_tensor_pipe_at_sampled_clock": (gemm_tflops / pipe_peak) if pipe_peak else None,
         "tensor_pipe_peak_at_sampled_clock": pipe_peak, "sampled_sm_mhz": sm_mhz or None,
-        # ncu, one launch of the 8192 x 6144 x 4096 GEMM (QKV Fprop at 8192 tokens; profiles/): DRAM
-        # bytes of THAT launch, not scaled to this step's shapes (operands are re-read from L2 and
-        # part of the output is still in L2 at kernel end, so traffic does not follow the flops)
-        "traffic": 78.6e6,
-        "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one captured 8192x6144x4096 launch "
-                        "(algorithmic bytes of that launch 130.1e6); not scaled to the 12 shapes of this step",
+        # ncu, dram__bytes_read.sum + dram__bytes_write.sum per launch (profiles/).  Full layer stack at
+        # 16384 tokens: mean of the step's 12 launches, one-pass capture of the bench's own launches
+        # (5.73 GB per step; operands + outputs are 4.16 GB: the long-K GEMMs re-read their B panel once
+        # per band of tile rows, and ncu flushes the caches before each launch, which a running step does
+        # not).  Other workloads: one captured 8192 x 6144 x 4096 launch, not scaled.
+        "traffic": 477.5e6 if (args.workload == "layer_stack" and layer and not ladder) else 78.6e6,
+        "traffic_note": ("mean over the step's 12 launches of dram__bytes_read.sum + dram__bytes_write.sum, one-pass ncu "
+                         "capture of this command's launches (algorithmic operand + output bytes: 346.8e6 per launch)"
+                         if (args.workload == "layer_stack" and layer and not ladder) else
+                         "dram__bytes_read.sum + dram__bytes_write.sum of one captured 8192x6144x4096 launch "
+                         "(algorithmic bytes of that launch 130.1e6); not scaled to the shapes of this step"),
         "flops_per_launch": gemm_flops / n_gemm, "avg_launch_ms": gemm_ms_used / n_gemm,
         "launch_timing": gemm_timing,
         "tflops_by_launch": gemm_by_shape,
