@@ -93,6 +93,7 @@ struct GemmPairParams {
     int32_t M, N, K;
     int32_t tiles_m, tiles_n;   // 256 x 384 pair tiles
     int32_t band_m;             // tile rows per band of the tile order (see gemm_tile_coords)
+    int32_t band_n;             // 0, or tile columns per band when the bands run along N instead
     int32_t k_stages;           // ceil(K / 256)
     int32_t sf_tiles_k;         // ceil(K / 128)
     int32_t sf_rows_a;          // ceil(M / 128)
@@ -135,8 +136,20 @@ __device__ __forceinline__ uint32_t idesc_n(int n) { return static_cast<uint32_t
 // re-read once per band.  (With a single band -- every shape whose A fits in L2 -- this is plain
 // column-major order.  With tile rows fastest over ALL of M, a long-K A that exceeds L2 was
 // streamed from HBM once per tile column: 2.6 GB instead of 0.7 GB for 16384 x 4096 x 28672.)
+// When B is the smaller panel the bands run along N instead (`band_n` > 0): a band is `band_n` tile
+// columns whose B panel stays in L2, inside a band the tile column varies fastest, so that all of a
+// tile row's columns are in flight together and A streams from HBM once per band.
 __device__ __forceinline__ void gemm_tile_coords(const GemmPairParams& p, int tile, int& tm, int& tn)
 {
+    if (p.band_n > 0) {
+        const int per_band = p.band_n * p.tiles_m;
+        const int band = tile / per_band;
+        const int r = tile - band * per_band;
+        const int cols = min(p.band_n, p.tiles_n - band * p.band_n);    // the last band may be narrower
+        tm = r / cols;
+        tn = band * p.band_n + (r - tm * cols);
+        return;
+    }
     const int per_band = p.band_m * p.tiles_n;
     const int band = tile / per_band;
     const int r = tile - band * per_band;
@@ -561,11 +574,23 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
         // band height of the tile order: as many tile rows as keep the band's A panel within about a
         // quarter of the L2 (32 MB), so that it survives the band's sweep across N beside the B
         // panels streaming through
-        const int64_t a_tile_row_bytes = static_cast<int64_t>(kPTileM) * (KIND == 0 ? K / 2 : K);
+        const int64_t row_b = KIND == 0 ? K / 2 : K;                     // bytes of codes per operand row
+        const int64_t a_tile_row_bytes = static_cast<int64_t>(kPTileM) * row_b;
         int64_t band = (32ll << 20) / (a_tile_row_bytes > 0 ? a_tile_row_bytes : 1);
         if (band < 1) band = 1;
         if (band > p.tiles_m) band = p.tiles_m;
         p.band_m = static_cast<int32_t>(band);
+        // the same along N (a few MB more of budget, so that eleven tile columns of a 4096-wide B make
+        // one or two bands); the orientation with the smaller estimate of HBM reads wins:
+        // bands along M read A once and B once per band, bands along N the other way round
+        const int64_t b_tile_col_bytes = static_cast<int64_t>(kPTileN) * row_b;
+        int64_t band_n = (36ll << 20) / (b_tile_col_bytes > 0 ? b_tile_col_bytes : 1);
+        if (band_n < 1) band_n = 1;
+        if (band_n > p.tiles_n) band_n = p.tiles_n;
+        const int64_t bands_m = (p.tiles_m + band - 1) / band, bands_n = (p.tiles_n + band_n - 1) / band_n;
+        const int64_t a_bytes = M * row_b, b_bytes = N * row_b;
+        const int64_t cost_m = a_bytes + b_bytes * bands_m, cost_n = b_bytes + a_bytes * bands_n;
+        p.band_n = cost_n < cost_m ? static_cast<int32_t>(band_n) : 0;
     }
     constexpr int kBlockK = KIND == 0 ? kPBlockK : kPBlockK / 2;
     p.k_stages = static_cast<int32_t>((K + kBlockK - 1) / kBlockK);

@@ -222,19 +222,22 @@ def test_mma_rate_probe_runs_and_reports_its_flops():
         api.probe_mma_rate(0, True)
 
 
-def test_band_order_with_a_ragged_last_band():
-    """K = 65536 makes a 256-row tile of A 8 MB, so the tile order uses bands of four tile rows:
-    M = 2304 + 40 gives bands of 4, 4 and 2 tile rows (the last one ragged in rows as well), N = 900
-    three tile columns with a narrow last one.  Whole output against the fp64 checker on the same
-    codes and scales, sampled rows of every band against the CPU oracle."""
+@pytest.mark.parametrize("M,N", [(2344, 900), (2344, 1900), (1300, 1900)])
+def test_band_order_with_a_ragged_last_band(M, N):
+    """K = 65536 makes a 256-row tile of A 8 MB and a 384-row tile of B 12 MB, so the tile order
+    works in bands, along whichever axis the host estimates fewer HBM reads for: (2344, 900) one band
+    of all three tile columns, tile column fastest; (2344, 1900) bands of 2, 2 and 1 tile columns (the
+    last one narrow, the last tile column ragged); (1300, 1900) bands of 4 and 2 tile ROWS (the last
+    tile row ragged).  Whole output against the fp64 checker on the same codes and scales, sampled
+    rows of every band against the CPU oracle."""
     import gemm_checker
-    rng = np.random.default_rng(65536)
-    M, N, K = 2344, 900, 65536
+    rng = np.random.default_rng(65536 + M + N)
+    K = 65536
     ac, asc, bc, bsc = _random_operands(rng, M, N, K, lo=122, hi=132)
     out = api.gemm(_dev(ac), _dev(oracle.scales_to_tiled(asc)), _dev(bc), _dev(oracle.scales_to_tiled(bsc)),
                    0.03125, api.OUT_FP32)
     api.check()
-    rows = np.array([0, 255, 256, 1023, 1024, 1500, 2047, 2048, 2303, 2304, 2343])
+    rows = np.array([r for r in (0, 255, 256, 1023, 1024, 1279, 1280, 1299, 1500, 2047, 2048, 2303, 2304, 2343) if r < M])
     ref, S = oracle.gemm(ac, asc, bc, bsc, alpha=0.03125, rows=rows)
     assert_gemm_close(out[torch.from_numpy(rows).cuda()].cpu().numpy(), ref, S, False, "band order, sampled rows")
     _, _, _, cref, cS = gemm_checker.check(ac[rows], asc[rows], bc, bsc, 0.03125, None, want_ref=True)
