@@ -698,10 +698,10 @@ def run_ours(args):
         "tensor_pipe_peak_at_sampled_clock": pipe_peak, "sampled_sm_mhz": sm_mhz or None,
         # ncu, dram__bytes_read.sum + dram__bytes_write.sum per launch (profiles/).  Full layer stack at
         # 16384 tokens: mean of the step's 12 launches, one-pass capture of the bench's own launches
-        # (5.73 GB per step; operands + outputs are 4.16 GB: the long-K GEMMs re-read their B panel once
-        # per band of tile rows, and ncu flushes the caches before each launch, which a running step does
+        # (4.86 GB per step; operands + outputs are 4.16 GB: the long-K GEMMs re-read the streamed panel once
+        # per band of the tile order, and ncu flushes the caches before each launch, which a running step does
         # not).  Other workloads: one captured 8192 x 6144 x 4096 launch, not scaled.
-        "traffic": 477.5e6 if (args.workload == "layer_stack" and layer and not ladder) else 78.6e6,
+        "traffic": 405.1e6 if (args.workload == "layer_stack" and layer and not ladder) else 78.6e6,
         "traffic_note": ("mean over the step's 12 launches of dram__bytes_read.sum + dram__bytes_write.sum, one-pass ncu "
                          "capture of this command's launches (algorithmic operand + output bytes: 346.8e6 per launch)"
                          if (args.workload == "layer_stack" and layer and not ladder) else
