@@ -581,8 +581,9 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
         if (band > p.tiles_m) band = p.tiles_m;
         p.band_m = static_cast<int32_t>(band);
         // the same along N (a few MB more of budget, so that eleven tile columns of a 4096-wide B make
-        // one or two bands); the orientation with the smaller estimate of HBM reads wins:
-        // bands along M read A once and B once per band, bands along N the other way round
+        // one or two bands); the orientation with the smaller estimate of HBM reads wins (bands along
+        // M read A once and B once per band, bands along N the other way round); a tie -- both panels
+        // fit, one band either way -- goes to N, 1-2 % faster on the 4096 x 4096 projections
         const int64_t b_tile_col_bytes = static_cast<int64_t>(kPTileN) * row_b;
         int64_t band_n = (36ll << 20) / (b_tile_col_bytes > 0 ? b_tile_col_bytes : 1);
         if (band_n < 1) band_n = 1;
@@ -590,7 +591,7 @@ static int launch_gemm_pair(const void* a_codes, const void* a_scales, const voi
         const int64_t bands_m = (p.tiles_m + band - 1) / band, bands_n = (p.tiles_n + band_n - 1) / band_n;
         const int64_t a_bytes = M * row_b, b_bytes = N * row_b;
         const int64_t cost_m = a_bytes + b_bytes * bands_m, cost_n = b_bytes + a_bytes * bands_n;
-        p.band_n = cost_n < cost_m ? static_cast<int32_t>(band_n) : 0;
+        p.band_n = cost_n <= cost_m ? static_cast<int32_t>(band_n) : 0;
     }
     constexpr int kBlockK = KIND == 0 ? kPBlockK : kPBlockK / 2;
     p.k_stages = static_cast<int32_t>((K + kBlockK - 1) / kBlockK);
